@@ -1,0 +1,148 @@
+/* sgc.h -- C ABI of the B200 (sm_100a) implementation of one Sparse Gradient Compression step.
+ *
+ * One SGC step for one flat parameter vector W in R^d with gradient G in R^d (the paper treats every
+ * weight matrix as a vector, Section 3 footnote; the flat row-major element index is the column
+ * index of the measurement matrix A in R^{k x d}):
+ *
+ *   a1  G~ = Sparsify_s(G)                      keep the s largest |g_i|                (Section 3.2)
+ *   a2  p = A G~ ,  q = A G~^2                  Eq. (4) and the equation after it; Algorithm 2 line 1
+ *   a3  M <- b1 M + (1-b1) p ; V <- b2 V + (1-b2) q ; M^ = M/(1-b1^t) ; V^ = V/(1-b2^t)
+ *                                                Algorithm 2 lines 2-5
+ *   a4  x^M = OMP_A(M^) , x^V = OMP_A(V^)       Eq. (7); Appendix B Algorithm 3
+ *   a5  N = alpha x^M / (sqrt(x^V) + eps) ; W <- W - lr N          Eq. (8), Eq. (3); Algorithm 2 line 6
+ *
+ * A is never stored.  A[j][i] = sigma_k * Z(seed, j, i), sigma_k = fl32(1/sqrt(k)), where Z is a
+ * counter-based, approximately standard-normal function of (seed, row, column) evaluated on the fly
+ * (i.i.d. zero-mean entries of standard deviation 1/sqrt(k), Section 3.3).  Two states created with
+ * the same (seed, k) therefore see the same A on their common columns.
+ *
+ * Conventions
+ *   - Every function returns 0 on success, a negative SGC_ERR_* code for a rejected argument and a
+ *     positive value (a cudaError_t) when a CUDA call failed.  Nothing aborts, traps or asserts.
+ *   - "device pointer" = memory of the current CUDA device, "host pointer" = ordinary host memory.
+ *   - All work of sgc_step is enqueued on the caller's stream; the call does not synchronise.
+ *   - A state belongs to the device that was current in sgc_create; calls on one state must not overlap.
+ *   - Data-dependent conditions (non-finite gradient, dependent OMP column, support mismatch) are
+ *     recorded in a device status word that sgc_get(SGC_GET_STATUS) returns; see SGC_STATUS_*.
+ */
+#ifndef SGC_H_
+#define SGC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sgc_state sgc_state;
+
+enum {
+    SGC_OK = 0,
+    SGC_ERR_NULL = -1,        /* a required pointer is NULL                                   */
+    SGC_ERR_DIM = -2,         /* d < 1, k < 1, s < 1, s > k, s > d, d >= 2^32, k or s too large */
+    SGC_ERR_HYPER = -3,       /* beta outside [0,1), eps <= 0, lr or alpha not finite          */
+    SGC_ERR_ALIGN = -4,       /* grad or weight not 16-byte aligned                            */
+    SGC_ERR_WHAT = -5,        /* unknown selector for sgc_get                                  */
+    SGC_ERR_SIZE = -6,        /* destination buffer too small                                  */
+    SGC_ERR_GROUP = -7,       /* states of a group do not share (d, k, s, seed)                */
+    SGC_ERR_NOSTEP = -8       /* a record was requested before the first step                  */
+};
+
+/* bits of the status word (sticky until sgc_clear_status) */
+enum {
+    SGC_STATUS_NONFINITE_INPUT = 1u << 0,  /* the gradient held a NaN or an infinity              */
+    SGC_STATUS_DEPENDENT_COLUMN = 1u << 1, /* OMP stopped early: new column dependent on support  */
+    SGC_STATUS_SUPPORT_MISMATCH = 1u << 2, /* supports of OMP(M^) and OMP(V^) differ (Section 3.3 expects equal) */
+    SGC_STATUS_NEGATIVE_V = 1u << 3,       /* a recovered second-moment entry was <= 0; skipped   */
+    SGC_STATUS_CANDIDATE_OVERFLOW = 1u << 4, /* a bounded candidate buffer overflowed; the step
+                                                fell back to its slower exact path               */
+    SGC_STATUS_SELECT_FALLBACK = 1u << 5   /* the sampled top-s threshold missed; exact fallback ran */
+};
+
+/* selectors for sgc_get: records of the LAST step, copied to a host buffer */
+enum {
+    SGC_GET_T = 0,          /* int64      step counter t                                        */
+    SGC_GET_M = 1,          /* float[k]   first-moment state (not bias corrected)               */
+    SGC_GET_V = 2,          /* float[k]   second-moment state                                   */
+    SGC_GET_SEL_IDX = 3,    /* uint32[s]  support of Sparsify_s(G), ascending                   */
+    SGC_GET_SEL_VAL = 4,    /* float[s]   the kept gradient entries                             */
+    SGC_GET_P = 5,          /* double[k]  p = A G~                                              */
+    SGC_GET_Q = 6,          /* double[k]  q = A G~^2                                            */
+    SGC_GET_LAM_M = 7,      /* uint32[s]  columns picked by OMP(M^), in selection order; 0xFFFFFFFF = not picked */
+    SGC_GET_LAM_V = 8,      /* uint32[s]  same for OMP(V^)                                      */
+    SGC_GET_X_M = 9,        /* double[s]  least-squares coefficients aligned with LAM_M         */
+    SGC_GET_X_V = 10,       /* double[s]  aligned with LAM_V                                    */
+    SGC_GET_UPD_IDX = 11,   /* uint32[s]  positions of W that were updated, ascending; first N_UPD valid */
+    SGC_GET_UPD_VAL = 12,   /* double[s]  lr * N at those positions                             */
+    SGC_GET_N_UPD = 13,     /* int32      number of updated positions                           */
+    SGC_GET_STATUS = 14,    /* uint32     status word                                           */
+    SGC_GET_MISMATCH = 15,  /* int32      entries of LAM_M absent from LAM_V in the last step   */
+    SGC_GET_NEGV = 16,      /* int32      common entries skipped because x^V <= 0               */
+    SGC_GET_DONE_M = 17,    /* int32      completed OMP iterations for M^                       */
+    SGC_GET_DONE_V = 18,    /* int32      completed OMP iterations for V^                       */
+    SGC_GET_RNORM_M = 19,   /* double[s]  residual norm after each OMP(M^) iteration            */
+    SGC_GET_RNORM_V = 20    /* double[s]  same for OMP(V^)                                      */
+};
+
+/* Problem statement of Section 3 (Eq. 3) with the method of Algorithm 2.
+ * Allocates the optimizer state M, V in R^k (zero, Section 3.3: M_0 = V_0 = 0), t = 0 and all
+ * workspace on the current device; the library owns them until sgc_destroy.
+ *   out    host pointer receiving the handle (set to NULL on failure)
+ *   d      length of the flat weight / gradient vector, 1 <= d < 2^32
+ *   k      rows of A (dimension of the compressed space), 1 <= k <= 65536
+ *   s      sparsity, 1 <= s <= min(k, d), s <= 1024
+ *   seed   names the matrix A
+ *   lr     learning rate eta of Eq. (3); beta1, beta2, eps: Algorithm 2 "Require"
+ * The scale alpha of Eq. (8) defaults to 1 (sgc_set_alpha). */
+int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, float beta1,
+               float beta2, float eps);
+
+/* One step of Algorithm 2 followed by Eq. (3): W <- W - lr * SGC(G).
+ *   grad    device pointer, d floats, 16-byte aligned, read only
+ *   weight  device pointer, d floats, 16-byte aligned, modified in place at no more than s positions
+ *   stream  a cudaStream_t (NULL = the default stream)
+ * Returns after enqueueing; the caller keeps grad and weight alive until the stream has drained. */
+int sgc_step(sgc_state* st, const float* grad, float* weight, void* stream);
+
+/* Same result as n independent sgc_step calls, for states that share (d, k, s, seed) and hence the
+ * same A (Section 4.4 lets equal-sized vectors share one A): their 2n residuals are correlated
+ * against each generated tile of A together.
+ *   states, grads, weights   host arrays of n handles / device pointers */
+int sgc_step_group(sgc_state* const* states, const float* const* grads, float* const* weights, int32_t n,
+                   void* stream);
+
+/* Waits for the state's last enqueued work, then frees everything.  NULL is accepted. */
+int sgc_destroy(sgc_state* st);
+
+/* alpha of Eq. (8) ("a scaling factor"); must be finite. */
+int sgc_set_alpha(sgc_state* st, float alpha);
+
+/* Synchronises with the state's last step and copies one record to host memory (selectors above).
+ *   dst    host pointer; bytes = its capacity, must cover the record */
+int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes);
+
+/* Overwrites the optimizer state: M, V host pointers to k floats each, t >= 0 (checkpoint resume). */
+int sgc_set_state(sgc_state* st, const float* M, const float* V, int64_t t);
+
+/* Clears the sticky status word. */
+int sgc_clear_status(sgc_state* st);
+
+/* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
+int sgc_last_launches(sgc_state* st, int32_t* out);
+
+/* Fills a device buffer with Z(seed, row0 + r, col0 + c), r < nrows, c < ncols, row-major
+ * (the A definition above without the scale); for checking the generator.
+ *   out   device pointer, nrows*ncols floats */
+int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out, void* stream);
+
+/* Human-readable text for a return code of this library (static storage). */
+const char* sgc_strerror(int code);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int sgc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGC_H_ */

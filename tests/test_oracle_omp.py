@@ -1,0 +1,163 @@
+"""Pins for the oracle's recovery step a4 (OMP, Eq. 7 / Appendix B) and for the whole step (CPU only)."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+
+
+def dense_A(seed, k, d):
+    return oracle.z_block(seed, 0, k, 0, d).astype(np.float64) * np.float64(oracle.sigma(k))
+
+
+def numpy_omp(A, y, s):
+    """Dense restatement with library routines: argmax of |A^T r| / ||A_i||, numpy lstsq on the support."""
+    k, d = A.shape
+    nrm = np.linalg.norm(A, axis=0)
+    r = y.copy()
+    lam = []
+    for _ in range(s):
+        c = np.abs(A.T @ r) / nrm
+        c[lam] = -1.0
+        lam.append(int(np.argmax(c)))
+        x, *_ = np.linalg.lstsq(A[:, lam], y, rcond=None)
+        r = y - A[:, lam] @ x
+    return lam, x, r
+
+
+def test_exact_recovery_of_planted_sparse_vector():
+    # k comfortably above s*log(d/s): OMP returns the planted support and values (Section 3.3).
+    seed, d, k, s = 11, 4096, 512, 8
+    rng = np.random.default_rng(5)
+    supp = np.sort(rng.choice(d, size=s, replace=False))
+    xs = rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)
+    A = dense_A(seed, k, d)
+    y = A[:, supp] @ xs
+    out = oracle.omp(seed, d, k, s, y)
+    assert out["done"] == s
+    order = np.argsort(out["lam"])
+    assert np.array_equal(out["lam"][order], supp.astype(np.uint32))
+    np.testing.assert_allclose(out["x"][order], xs, rtol=1e-9)
+    assert out["rnorm"][-1] < 1e-10 * np.linalg.norm(y)
+    assert np.all(np.diff(out["rnorm"]) <= 1e-12)                 # residual norm never increases
+    assert np.all(out["top1"] >= out["top2"])
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_brute_force_over_every_support(seed):
+    # On a tiny problem with exact recovery the OMP support is the global least-squares minimiser
+    # over all supports of size s, and x is the least-squares solution on it.
+    d, k, s = 18, 12, 3
+    rng = np.random.default_rng(100 + seed)
+    supp = np.sort(rng.choice(d, size=s, replace=False))
+    xs = rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)
+    A = dense_A(seed, k, d)
+    y = A[:, supp] @ xs
+    best, best_S = np.inf, None
+    for S in itertools.combinations(range(d), s):
+        x, *_ = np.linalg.lstsq(A[:, S], y, rcond=None)
+        res = np.linalg.norm(y - A[:, S] @ x)
+        if res < best:
+            best, best_S = res, S
+    out = oracle.omp(seed, d, k, s, y)
+    lam_np, x_np, _ = numpy_omp(A, y, s)
+    assert out["lam"].tolist() == lam_np                               # same greedy path as the dense restatement
+    if best < 1e-9 and sorted(lam_np) == list(supp):
+        assert sorted(out["lam"].tolist()) == list(best_S)
+    xls, *_ = np.linalg.lstsq(A[:, out["lam"].astype(int)], y, rcond=None)
+    np.testing.assert_allclose(out["x"], xls, rtol=1e-9, atol=1e-12)
+
+
+def test_matches_dense_numpy_restatement_on_noisy_target():
+    # inexact regime: y is not s-sparse in A; every pick, the coefficients and residual norms must still agree
+    seed, d, k, s = 6, 700, 48, 10
+    rng = np.random.default_rng(2)
+    A = dense_A(seed, k, d)
+    y = rng.standard_normal(k)
+    out = oracle.omp(seed, d, k, s, y)
+    lam_np, x_np, r_np = numpy_omp(A, y, s)
+    assert out["lam"].tolist() == lam_np
+    np.testing.assert_allclose(out["x"], x_np, rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(out["rnorm"][-1], np.linalg.norm(r_np), rtol=1e-10)
+    # residual orthogonal to the selected columns
+    r = y - A[:, lam_np] @ out["x"]
+    assert np.abs(A[:, lam_np].T @ r).max() < 1e-12
+    # top1/top2 records are the two largest normalised correlations of the first iteration
+    c = np.sort(np.abs(A.T @ y) / np.linalg.norm(A, axis=0))[::-1]
+    np.testing.assert_allclose([out["top1"][0], out["top2"][0]], c[:2], rtol=1e-12)
+
+
+def test_scale_invariance():
+    seed, d, k, s = 8, 2000, 96, 12
+    rng = np.random.default_rng(9)
+    y = rng.standard_normal(k)
+    a = oracle.omp(seed, d, k, s, y)
+    b = oracle.omp(seed, d, k, s, 37.5 * y)
+    assert np.array_equal(a["lam"], b["lam"])
+    np.testing.assert_allclose(b["x"], 37.5 * a["x"], rtol=1e-10)
+
+
+def test_lowest_index_wins_exact_ties_and_no_reselection():
+    # y = 0 gives all-zero correlations: every pick is an exact tie -> lowest unselected index; the
+    # columns are independent so all s iterations complete with zero coefficients.
+    out = oracle.omp(3, 50, 16, 4, np.zeros(16))
+    assert out["lam"].tolist() == [0, 1, 2, 3] and not out["x"].any()
+
+
+def test_dependent_column_stops_early():
+    # k = 2 rows: a third column is always dependent on two selected ones
+    out = oracle.omp(3, 6, 2, 2, np.array([1.0, -2.0]))
+    assert out["done"] == 2
+    st = oracle.Oracle(6, 2, 2, 3, 1e-3, 0.9, 0.999, 1e-8)
+    st.close()
+
+
+def test_whole_step_constant_sparse_gradient_closed_form():
+    # A gradient with exactly s non-zeros, held constant: Mhat = A g, Vhat = A g^2 for all t, OMP recovers
+    # both exactly, so N = alpha * g / (|g| + eps) = alpha * sign(g) and W_t = W_0 - t*eta*alpha*sign(g).
+    d, k, s, seed = 2048, 256, 6, 21
+    lr, alpha = np.float32(1e-3), 2.0
+    rng = np.random.default_rng(4)
+    supp = np.sort(rng.choice(d, size=s, replace=False))
+    g = np.zeros(d, dtype=np.float32)
+    g[supp] = (rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
+    W0 = rng.standard_normal(d).astype(np.float32)
+    W = W0.copy()
+    st = oracle.Oracle(d, k, s, seed, lr, 0.9, 0.999, 1e-8, alpha=alpha)
+    for t in range(1, 6):
+        st.step(g, W)
+        assert st.get("t") == t
+        assert np.array_equal(st.get("sel_idx"), supp.astype(np.uint32))
+        assert sorted(st.get("lamM").tolist()) == supp.tolist() == sorted(st.get("lamV").tolist())
+        assert st.get("mismatch") == 0 and st.get("negv") == 0 and st.get("n_upd") == s
+        order = np.argsort(st.get("lamM"))
+        np.testing.assert_allclose(st.get("xM")[order], g[supp], rtol=2e-6)      # fp32 state rounding
+        want = W0.astype(np.float64)
+        want[supp] -= t * np.float64(lr) * alpha * np.sign(g[supp])
+        np.testing.assert_allclose(W, want, rtol=0, atol=3e-6)
+        untouched = np.ones(d, dtype=bool)
+        untouched[supp] = False
+        assert np.array_equal(W[untouched], W0[untouched])
+    st.close()
+
+
+def test_step_split_equals_whole_step():
+    d, k, s = 512, 64, 4
+    rng = np.random.default_rng(12)
+    a = oracle.Oracle(d, k, s, 1, 1e-3, 0.9, 0.999, 1e-8)
+    b = oracle.Oracle(d, k, s, 1, 1e-3, 0.9, 0.999, 1e-8)
+    Wa = rng.standard_normal(d).astype(np.float32)
+    Wb = Wa.copy()
+    for _ in range(3):
+        g = rng.standard_normal(d).astype(np.float32)
+        a.step(g, Wa)
+        b.step_compress(g)
+        b.step_recover(Wb)
+    assert np.array_equal(Wa, Wb) and np.array_equal(a.get("M"), b.get("M"))
+
+
+def test_create_rejects_bad_arguments():
+    for (d, k, s) in [(0, 4, 1), (10, 0, 1), (10, 4, 0), (10, 4, 5), (3, 8, 4), (1 << 32, 8, 4)]:
+        with pytest.raises(ValueError):
+            oracle.Oracle(d, k, s, 0, 1e-3, 0.9, 0.999, 1e-8)

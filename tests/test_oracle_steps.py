@@ -1,0 +1,128 @@
+"""Pins for the oracle's steps a1-a3 and a5 (CPU only): plain definitions on dense matrices,
+closed forms and invariants that the paper states."""
+import numpy as np
+import pytest
+
+import oracle
+
+
+def dense_A(seed, k, d):
+    return oracle.z_block(seed, 0, k, 0, d).astype(np.float64) * np.float64(oracle.sigma(k))
+
+
+# ---- a1 Sparsify_s --------------------------------------------------------------------------------
+@pytest.mark.parametrize("d,s", [(1, 1), (17, 5), (1000, 16), (4096, 64), (100003, 256)])
+def test_sparsify_is_full_sort_definition(d, s):
+    rng = np.random.default_rng(d)
+    g = rng.standard_normal(d).astype(np.float32)
+    idx, val = oracle.sparsify(g, s)
+    order = np.argsort(-np.abs(g).astype(np.float64), kind="stable")[:s]   # |g| descending, index ascending
+    assert np.array_equal(idx, np.sort(order).astype(np.uint32))
+    assert np.array_equal(val, g[idx])
+    assert np.all(np.diff(idx.astype(np.int64)) > 0)
+
+
+def test_sparsify_ties_zeros_and_signed_zero():
+    g = np.array([0.5, -0.5, 0.5, 0.0, -0.0, 0.25, -0.5], dtype=np.float32)
+    idx, val = oracle.sparsify(g, 3)
+    assert idx.tolist() == [0, 1, 2]                 # four entries tie at 0.5: the three lowest indices win
+    idx, _ = oracle.sparsify(g, 6)
+    assert idx.tolist() == [0, 1, 2, 3, 5, 6]        # +0 and -0 tie: index 3 before index 4
+    g = np.zeros(10, dtype=np.float32)
+    idx, val = oracle.sparsify(g, 4)
+    assert idx.tolist() == [0, 1, 2, 3] and not val.any()
+
+
+# ---- a2 projection ---------------------------------------------------------------------------------
+def test_projection_equals_dense_matvec():
+    seed, k, d, s = 2, 64, 300, 9
+    rng = np.random.default_rng(1)
+    g = rng.standard_normal(d).astype(np.float32)
+    idx, val = oracle.sparsify(g, s)
+    A = dense_A(seed, k, d)
+    gt = np.zeros(d)
+    gt[idx] = val.astype(np.float64)
+    p, q = oracle.project(seed, k, idx, val)
+    np.testing.assert_allclose(p, A @ gt, rtol=0, atol=1e-14)
+    np.testing.assert_allclose(q, A @ (gt * gt), rtol=0, atol=1e-14)
+
+
+def test_projection_is_linear():
+    seed, k = 9, 128
+    idx = np.array([3, 77, 1000, 50000, 4_000_000_000], dtype=np.uint32)
+    x = np.array([1.0, -2.0, 0.5, 4.0, -0.25], dtype=np.float32)
+    y = np.array([0.5, 0.25, -8.0, 1.0, 2.0], dtype=np.float32)
+    px, _ = oracle.project(seed, k, idx, x)
+    py, _ = oracle.project(seed, k, idx, y)
+    pxy, _ = oracle.project(seed, k, idx, (2 * x + 4 * y).astype(np.float32))   # exact in fp32
+    np.testing.assert_allclose(pxy, 2 * px + 4 * py, rtol=0, atol=1e-13)
+    # q is the projection of the squared entries on the same support
+    _, qx = oracle.project(seed, k, idx, x)
+    px2, _ = oracle.project(seed, k, idx, (x * x).astype(np.float32))
+    np.testing.assert_allclose(qx, px2, rtol=0, atol=1e-14)
+
+
+# ---- a3 Adam in k-space ----------------------------------------------------------------------------
+def test_adam_constant_input_closed_form():
+    # Algorithm 2 lines 2-5 with M_0 = V_0 = 0 and constant p, q:  M_t = (1-b1^t) p,  Mhat_t = p.
+    k, b1, b2 = 50, np.float32(0.9), np.float32(0.999)
+    rng = np.random.default_rng(0)
+    p = rng.standard_normal(k)
+    q = rng.random(k)
+    M = np.zeros(k, dtype=np.float32)
+    V = np.zeros(k, dtype=np.float32)
+    for t in range(1, 40):
+        Mh, Vh = oracle.adam(M, V, p, q, b1, b2, t)
+        np.testing.assert_allclose(M, (1 - np.float64(b1) ** t) * p, rtol=3e-6, atol=0)
+        np.testing.assert_allclose(V, (1 - np.float64(b2) ** t) * q, rtol=2e-5, atol=0)
+        np.testing.assert_allclose(Mh, p, rtol=3e-6, atol=0)
+        np.testing.assert_allclose(Vh, q, rtol=2e-5, atol=0)
+
+
+def test_adam_second_moment_uses_beta2():
+    M = np.zeros(1, dtype=np.float32)
+    V = np.zeros(1, dtype=np.float32)
+    oracle.adam(M, V, np.array([1.0]), np.array([1.0]), np.float32(0.5), np.float32(0.75), 1)
+    assert M[0] == np.float32(0.5) and V[0] == np.float32(0.25)
+    Mh, Vh = oracle.adam(M, V, np.array([1.0]), np.array([1.0]), np.float32(0.5), np.float32(0.75), 2)
+    assert M[0] == np.float32(0.75) and V[0] == np.float32(0.4375)       # stored state is NOT bias corrected
+    assert Mh[0] == 1.0 and Vh[0] == 1.0
+
+
+def test_kspace_ema_is_projection_of_dspace_ema():
+    # Eq. (9): M_t = A sum_i h_i(beta1) G~_i.
+    seed, k, d, s, b1, b2 = 4, 32, 200, 6, np.float32(0.9), np.float32(0.999)
+    A = dense_A(seed, k, d)
+    rng = np.random.default_rng(3)
+    M = np.zeros(k, dtype=np.float32)
+    V = np.zeros(k, dtype=np.float32)
+    Md = np.zeros(d)
+    Vd = np.zeros(d)
+    for t in range(1, 8):
+        g = rng.standard_normal(d).astype(np.float32)
+        idx, val = oracle.sparsify(g, s)
+        gt = np.zeros(d)
+        gt[idx] = val
+        Md = np.float64(b1) * Md + (1 - np.float64(b1)) * gt
+        Vd = np.float64(b2) * Vd + (1 - np.float64(b2)) * gt * gt
+        p, q = oracle.project(seed, k, idx, val)
+        oracle.adam(M, V, p, q, b1, b2, t)
+        np.testing.assert_allclose(M, A @ Md, rtol=0, atol=2e-6 * np.abs(A @ Md).max())
+        np.testing.assert_allclose(V, A @ Vd, rtol=0, atol=2e-6 * np.abs(A @ Vd).max())
+
+
+# ---- a5 combine + scatter --------------------------------------------------------------------------
+def test_combine_scatter_definition_and_guards():
+    W = np.arange(10, dtype=np.float32)
+    lamM = np.array([7, 2, 5, 9], dtype=np.uint32)
+    xM = np.array([1.0, -2.0, 3.0, 4.0])
+    lamV = np.array([2, 7, 9, 4], dtype=np.uint32)
+    xV = np.array([4.0, 0.25, -1.0, 1.0])
+    ui, uv, mis, neg = oracle.combine_scatter(lamM, xM, lamV, xV, np.float32(2.0), np.float32(1e-8), np.float32(0.5),
+                                              W)
+    assert ui.tolist() == [2, 7] and mis == 1 and neg == 1        # 5 is not in Lam_V; x^V at 9 is negative
+    np.testing.assert_allclose(uv, [0.5 * 2.0 * -2.0 / (2.0 + 1e-8), 0.5 * 2.0 * 1.0 / (0.5 + 1e-8)], rtol=1e-12)
+    want = np.arange(10, dtype=np.float64)
+    want[2] -= uv[0]
+    want[7] -= uv[1]
+    assert np.array_equal(W, want.astype(np.float32))
