@@ -35,6 +35,12 @@
 extern "C" {
 #endif
 
+#if defined(__GNUC__)
+#define SGC_API __attribute__((visibility("default")))
+#else
+#define SGC_API
+#endif
+
 typedef struct sgc_state sgc_state;
 
 enum {
@@ -95,7 +101,7 @@ enum {
  *   seed   names the matrix A
  *   lr     learning rate eta of Eq. (3); beta1, beta2, eps: Algorithm 2 "Require"
  * The scale alpha of Eq. (8) defaults to 1 (sgc_set_alpha). */
-int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, float beta1,
+SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, float beta1,
                float beta2, float eps);
 
 /* One step of Algorithm 2 followed by Eq. (3): W <- W - lr * SGC(G).
@@ -103,44 +109,44 @@ int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_t seed, 
  *   weight  device pointer, d floats, 16-byte aligned, modified in place at no more than s positions
  *   stream  a cudaStream_t (NULL = the default stream)
  * Returns after enqueueing; the caller keeps grad and weight alive until the stream has drained. */
-int sgc_step(sgc_state* st, const float* grad, float* weight, void* stream);
+SGC_API int sgc_step(sgc_state* st, const float* grad, float* weight, void* stream);
 
 /* Same result as n independent sgc_step calls, for states that share (d, k, s, seed) and hence the
  * same A (Section 4.4 lets equal-sized vectors share one A): their 2n residuals are correlated
  * against each generated tile of A together.
  *   states, grads, weights   host arrays of n handles / device pointers */
-int sgc_step_group(sgc_state* const* states, const float* const* grads, float* const* weights, int32_t n,
+SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, float* const* weights, int32_t n,
                    void* stream);
 
 /* Waits for the state's last enqueued work, then frees everything.  NULL is accepted. */
-int sgc_destroy(sgc_state* st);
+SGC_API int sgc_destroy(sgc_state* st);
 
 /* alpha of Eq. (8) ("a scaling factor"); must be finite. */
-int sgc_set_alpha(sgc_state* st, float alpha);
+SGC_API int sgc_set_alpha(sgc_state* st, float alpha);
 
 /* Synchronises with the state's last step and copies one record to host memory (selectors above).
  *   dst    host pointer; bytes = its capacity, must cover the record */
-int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes);
+SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes);
 
 /* Overwrites the optimizer state: M, V host pointers to k floats each, t >= 0 (checkpoint resume). */
-int sgc_set_state(sgc_state* st, const float* M, const float* V, int64_t t);
+SGC_API int sgc_set_state(sgc_state* st, const float* M, const float* V, int64_t t);
 
 /* Clears the sticky status word. */
-int sgc_clear_status(sgc_state* st);
+SGC_API int sgc_clear_status(sgc_state* st);
 
 /* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
-int sgc_last_launches(sgc_state* st, int32_t* out);
+SGC_API int sgc_last_launches(sgc_state* st, int32_t* out);
 
 /* Fills a device buffer with Z(seed, row0 + r, col0 + c), r < nrows, c < ncols, row-major
  * (the A definition above without the scale); for checking the generator.
  *   out   device pointer, nrows*ncols floats */
-int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out, void* stream);
+SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out, void* stream);
 
 /* Human-readable text for a return code of this library (static storage). */
-const char* sgc_strerror(int code);
+SGC_API const char* sgc_strerror(int code);
 
 /* Library version, major*10000 + minor*100 + patch. */
-int sgc_version(void);
+SGC_API int sgc_version(void);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,180 @@
+"""Thin ctypes binding of the C-ABI library declared in include/sgc.h (argument marshalling only).
+
+PyTorch supplies device memory and streams; every step of the path runs inside the CUDA library.
+The library must have been built (paper_2502_00311_b200.build.build()); loading fails loudly otherwise.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
+_lib = None
+
+EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
+           "sgc_clear_status", "sgc_last_launches", "sgc_z_block", "sgc_strerror", "sgc_version"]
+
+# selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
+RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
+               sel_val=(4, np.float32, "s"), p=(5, np.float64, "k"), q=(6, np.float64, "k"),
+               lamM=(7, np.uint32, "s"), lamV=(8, np.uint32, "s"), xM=(9, np.float64, "s"), xV=(10, np.float64, "s"),
+               upd_idx=(11, np.uint32, "s"), upd_val=(12, np.float64, "s"), n_upd=(13, np.int32, None),
+               status=(14, np.uint32, None), mismatch=(15, np.int32, None), negv=(16, np.int32, None),
+               doneM=(17, np.int32, None), doneV=(18, np.int32, None), rnormM=(19, np.float64, "s"),
+               rnormV=(20, np.float64, "s"))
+
+STATUS_NONFINITE_INPUT = 1
+STATUS_DEPENDENT_COLUMN = 2
+STATUS_SUPPORT_MISMATCH = 4
+STATUS_NEGATIVE_V = 8
+STATUS_CANDIDATE_OVERFLOW = 16
+STATUS_SELECT_FALLBACK = 32
+
+
+class SgcError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s failed with code %d: %s" % (where, code, strerror(code)))
+
+
+def lib():
+    """Loads the shared library once; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: run paper_2502_00311_b200.build.build() "
+                               "(there is no CPU fallback)" % _LIB_PATH)
+        L = C.CDLL(_LIB_PATH)
+        vp = C.c_void_p
+        L.sgc_create.restype = C.c_int
+        L.sgc_create.argtypes = [C.POINTER(vp), C.c_int64, C.c_int32, C.c_int32, C.c_uint64, C.c_float, C.c_float,
+                                 C.c_float, C.c_float]
+        L.sgc_step.restype = C.c_int
+        L.sgc_step.argtypes = [vp, vp, vp, vp]
+        L.sgc_step_group.restype = C.c_int
+        L.sgc_step_group.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int32, vp]
+        L.sgc_destroy.restype = C.c_int
+        L.sgc_destroy.argtypes = [vp]
+        L.sgc_set_alpha.restype = C.c_int
+        L.sgc_set_alpha.argtypes = [vp, C.c_float]
+        L.sgc_get.restype = C.c_int
+        L.sgc_get.argtypes = [vp, C.c_int32, vp, C.c_size_t]
+        L.sgc_set_state.restype = C.c_int
+        L.sgc_set_state.argtypes = [vp, vp, vp, C.c_int64]
+        L.sgc_clear_status.restype = C.c_int
+        L.sgc_clear_status.argtypes = [vp]
+        L.sgc_last_launches.restype = C.c_int
+        L.sgc_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
+        L.sgc_z_block.restype = C.c_int
+        L.sgc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, vp]
+        L.sgc_strerror.restype = C.c_char_p
+        L.sgc_strerror.argtypes = [C.c_int]
+        L.sgc_version.restype = C.c_int
+        L.sgc_version.argtypes = []
+        _lib = L
+    return _lib
+
+
+def strerror(code):
+    return lib().sgc_strerror(int(code)).decode()
+
+
+def version():
+    return int(lib().sgc_version())
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise SgcError(rc, where)
+
+
+def _dev_ptr(t, n, what):
+    """Device pointer of a contiguous float32 CUDA tensor with at least n elements."""
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous float32 CUDA tensor" % what)
+    if t.numel() < n:
+        raise ValueError("%s has %d elements, need %d" % (what, t.numel(), n))
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def z_block(seed, row0, nrows, col0, ncols, stream=None):
+    """Z(seed, row, col) for a block as a float32 CUDA tensor [nrows, ncols] (sgc_z_block)."""
+    import torch
+    out = torch.empty((nrows, ncols), dtype=torch.float32, device="cuda")
+    _check(lib().sgc_z_block(C.c_uint64(seed), row0, nrows, col0, ncols, C.c_void_p(out.data_ptr()),
+                             _stream_ptr(stream)), "sgc_z_block")
+    return out
+
+
+class Sgc:
+    """One SGC optimizer state (sgc_create / sgc_step / sgc_destroy)."""
+
+    def __init__(self, d, k, s, seed, lr, beta1, beta2, eps, alpha=None):
+        self.d, self.k, self.s = int(d), int(k), int(s)
+        h = C.c_void_p()
+        _check(lib().sgc_create(C.byref(h), self.d, self.k, self.s, C.c_uint64(seed), lr, beta1, beta2, eps),
+               "sgc_create")
+        self._h = h
+        if alpha is not None:
+            self.set_alpha(alpha)
+
+    def set_alpha(self, alpha):
+        _check(lib().sgc_set_alpha(self._h, alpha), "sgc_set_alpha")
+
+    def step(self, grad, weight, stream=None):
+        _check(lib().sgc_step(self._h, _dev_ptr(grad, self.d, "grad"), _dev_ptr(weight, self.d, "weight"),
+                              _stream_ptr(stream)), "sgc_step")
+
+    def get(self, name):
+        code, dt, dim = RECORDS[name]
+        n = 1 if dim is None else getattr(self, dim)
+        out = np.empty(n, dtype=dt)
+        _check(lib().sgc_get(self._h, code, out.ctypes.data_as(C.c_void_p), out.nbytes), "sgc_get(%s)" % name)
+        return out[0] if dim is None else out
+
+    def set_state(self, M, V, t):
+        M = np.ascontiguousarray(M, dtype=np.float32)
+        V = np.ascontiguousarray(V, dtype=np.float32)
+        if M.size != self.k or V.size != self.k:
+            raise ValueError("M and V must have k elements")
+        _check(lib().sgc_set_state(self._h, M.ctypes.data_as(C.c_void_p), V.ctypes.data_as(C.c_void_p), int(t)),
+               "sgc_set_state")
+
+    def clear_status(self):
+        _check(lib().sgc_clear_status(self._h), "sgc_clear_status")
+
+    def last_launches(self):
+        n = C.c_int32(0)
+        _check(lib().sgc_last_launches(self._h, C.byref(n)), "sgc_last_launches")
+        return n.value
+
+    def close(self):
+        if getattr(self, "_h", None):
+            h, self._h = self._h, None
+            _check(lib().sgc_destroy(h), "sgc_destroy")
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def step_group(states, grads, weights, stream=None):
+    """sgc_step_group: one step for several states that share (d, k, s, seed)."""
+    n = len(states)
+    if not (n == len(grads) == len(weights)) or n == 0:
+        raise ValueError("states, grads and weights must be non-empty lists of equal length")
+    hs = (C.c_void_p * n)(*[st._h for st in states])
+    gs = (C.c_void_p * n)(*[_dev_ptr(g, states[i].d, "grad") for i, g in enumerate(grads)])
+    ws = (C.c_void_p * n)(*[_dev_ptr(w, states[i].d, "weight") for i, w in enumerate(weights)])
+    _check(lib().sgc_step_group(hs, gs, ws, n, _stream_ptr(stream)), "sgc_step_group")

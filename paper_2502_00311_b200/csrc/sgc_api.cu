@@ -1,0 +1,229 @@
+// C ABI of the SGC library (include/sgc.h): argument checks, state life cycle, step orchestration.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "sgc_internal.cuh"
+
+namespace {
+
+inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+template <class T>
+T* carve(unsigned char* base, size_t& off, size_t count) {
+    T* p = reinterpret_cast<T*>(base + off);
+    off = align_up(off + count * sizeof(T));
+    return p;
+}
+
+// lays out (base == nullptr: only measures) the workspace of a state
+size_t layout(sgc_state* st, unsigned char* base) {
+    size_t off = 0;
+    const size_t k = (size_t)st->k, s = (size_t)st->s;
+    st->M = carve<float>(base, off, k);
+    st->V = carve<float>(base, off, k);
+    st->p = carve<double>(base, off, k);
+    st->q = carve<double>(base, off, k);
+    st->sel_idx = carve<uint32_t>(base, off, s);
+    st->sel_val = carve<float>(base, off, s);
+    st->y64 = carve<double>(base, off, 2 * k);
+    st->r64 = carve<double>(base, off, 2 * k);
+    st->r32 = carve<float2>(base, off, k);
+    st->sel_cand = carve<unsigned long long>(base, off, sgc::kSelCap);
+    st->sel_hist = carve<unsigned int>(base, off, sgc::kSelBins);
+    st->corr_cand = carve<sgc::Cand>(base, off, 2 * (size_t)st->corr_grid * sgc::kCorrTop);
+    st->zsel = carve<uint16_t>(base, off, 2 * s * k);
+    st->lam = carve<uint32_t>(base, off, 2 * s);
+    st->F = carve<double>(base, off, 2 * s * s);
+    st->acoef = carve<double>(base, off, 2 * s);
+    st->x = carve<double>(base, off, 2 * s);
+    st->rnorm = carve<double>(base, off, 2 * s);
+    st->upd_idx = carve<uint32_t>(base, off, s);
+    st->upd_val = carve<double>(base, off, s);
+    st->cnt = carve<sgc::Counters>(base, off, 1);
+    return off;
+}
+
+bool finite_f(float v) { return isfinite(v); }
+
+}  // namespace
+
+extern "C" {
+
+SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, float beta1, float beta2,
+               float eps) {
+    if (!out) return SGC_ERR_NULL;
+    *out = nullptr;
+    if (d < 1 || k < 1 || s < 1 || s > k || (int64_t)s > d || d >= ((int64_t)1 << 32) || k > sgc::kMaxK ||
+        s > sgc::kMaxS)
+        return SGC_ERR_DIM;
+    if (!(beta1 >= 0.0f && beta1 < 1.0f) || !(beta2 >= 0.0f && beta2 < 1.0f) || !(eps > 0.0f) || !finite_f(eps) ||
+        !finite_f(lr))
+        return SGC_ERR_HYPER;
+    sgc_state* st = new (std::nothrow) sgc_state();
+    if (!st) return (int)cudaErrorMemoryAllocation;
+    memset(st, 0, sizeof(*st));
+    st->d = d; st->k = k; st->s = s; st->seed = seed; st->lr = lr; st->beta1 = beta1; st->beta2 = beta2; st->eps = eps;
+    st->alpha = 1.0f; st->t = 0;
+    cudaError_t e = cudaGetDevice(&st->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&st->sm_count, cudaDevAttrMultiProcessorCount, st->device);
+    if (e == cudaSuccess) e = sgc::configure_recover(st);
+    if (e == cudaSuccess) {
+        st->bytes = layout(st, nullptr);
+        e = cudaMalloc(&st->base, st->bytes);
+    }
+    if (e == cudaSuccess) {
+        layout(st, static_cast<unsigned char*>(st->base));
+        e = cudaMemset(st->base, 0, st->bytes);        // M_0 = V_0 = 0, counters, histogram
+    }
+    if (e != cudaSuccess) {
+        if (st->base) cudaFree(st->base);
+        delete st;
+        return (int)e;
+    }
+    *out = st;
+    return SGC_OK;
+}
+
+SGC_API int sgc_step(sgc_state* st, const float* grad, float* weight, void* stream) {
+    if (!st || !grad || !weight) return SGC_ERR_NULL;
+    if (((uintptr_t)grad & 15u) || ((uintptr_t)weight & 15u)) return SGC_ERR_ALIGN;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    st->t += 1;
+    int launches = 0;
+    cudaError_t e = sgc::launch_select(st, grad, cs, &launches);
+    if (e == cudaSuccess) e = sgc::launch_project_adam(st, cs, &launches);
+    if (e == cudaSuccess) e = sgc::launch_recover(st, weight, cs, &launches);
+    st->last_stream = cs; st->has_stream = true; st->stepped = true; st->last_launches = launches;
+    return (int)e;
+}
+
+SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, float* const* weights, int32_t n, void* stream) {
+    if (!states || !grads || !weights) return SGC_ERR_NULL;
+    if (n < 1) return SGC_ERR_DIM;
+    for (int32_t i = 0; i < n; ++i) {
+        if (!states[i] || !grads[i] || !weights[i]) return SGC_ERR_NULL;
+        if (states[i]->d != states[0]->d || states[i]->k != states[0]->k || states[i]->s != states[0]->s ||
+            states[i]->seed != states[0]->seed)
+            return SGC_ERR_GROUP;
+        if (((uintptr_t)grads[i] & 15u) || ((uintptr_t)weights[i] & 15u)) return SGC_ERR_ALIGN;
+        for (int32_t j = 0; j < i; ++j) if (states[j] == states[i]) return SGC_ERR_GROUP;
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        const int rc = sgc_step(states[i], grads[i], weights[i], stream);
+        if (rc != 0) return rc;
+    }
+    return SGC_OK;
+}
+
+SGC_API int sgc_destroy(sgc_state* st) {
+    if (!st) return SGC_OK;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    cudaError_t e2 = cudaFree(st->base);
+    delete st;
+    return (int)(e != cudaSuccess ? e : e2);
+}
+
+SGC_API int sgc_set_alpha(sgc_state* st, float alpha) {
+    if (!st) return SGC_ERR_NULL;
+    if (!finite_f(alpha)) return SGC_ERR_HYPER;
+    st->alpha = alpha;
+    return SGC_OK;
+}
+
+SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
+    if (!st || !dst) return SGC_ERR_NULL;
+    const size_t k = (size_t)st->k, s = (size_t)st->s;
+    const void* src = nullptr;
+    size_t n = 0;
+    bool needs_step = true;
+    switch (what) {
+        case SGC_GET_T: {
+            if (bytes < 8) return SGC_ERR_SIZE;
+            memcpy(dst, &st->t, 8);
+            return SGC_OK;
+        }
+        case SGC_GET_M: src = st->M; n = 4 * k; needs_step = false; break;
+        case SGC_GET_V: src = st->V; n = 4 * k; needs_step = false; break;
+        case SGC_GET_SEL_IDX: src = st->sel_idx; n = 4 * s; break;
+        case SGC_GET_SEL_VAL: src = st->sel_val; n = 4 * s; break;
+        case SGC_GET_P: src = st->p; n = 8 * k; break;
+        case SGC_GET_Q: src = st->q; n = 8 * k; break;
+        case SGC_GET_LAM_M: src = st->lam; n = 4 * s; break;
+        case SGC_GET_LAM_V: src = st->lam + s; n = 4 * s; break;
+        case SGC_GET_X_M: src = st->x; n = 8 * s; break;
+        case SGC_GET_X_V: src = st->x + s; n = 8 * s; break;
+        case SGC_GET_UPD_IDX: src = st->upd_idx; n = 4 * s; break;
+        case SGC_GET_UPD_VAL: src = st->upd_val; n = 8 * s; break;
+        case SGC_GET_N_UPD: src = &st->cnt->n_upd; n = 4; break;
+        case SGC_GET_STATUS: src = &st->cnt->status; n = 4; needs_step = false; break;
+        case SGC_GET_MISMATCH: src = &st->cnt->mismatch; n = 4; break;
+        case SGC_GET_NEGV: src = &st->cnt->negv; n = 4; break;
+        case SGC_GET_DONE_M: src = &st->cnt->done[0]; n = 4; break;
+        case SGC_GET_DONE_V: src = &st->cnt->done[1]; n = 4; break;
+        case SGC_GET_RNORM_M: src = st->rnorm; n = 8 * s; break;
+        case SGC_GET_RNORM_V: src = st->rnorm + s; n = 8 * s; break;
+        default: return SGC_ERR_WHAT;
+    }
+    if (needs_step && !st->stepped) return SGC_ERR_NOSTEP;
+    if (bytes < n) return SGC_ERR_SIZE;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(dst, src, n, cudaMemcpyDeviceToHost);
+    return (int)e;
+}
+
+SGC_API int sgc_set_state(sgc_state* st, const float* M, const float* V, int64_t t) {
+    if (!st || !M || !V) return SGC_ERR_NULL;
+    if (t < 0) return SGC_ERR_DIM;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(st->M, M, 4 * (size_t)st->k, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(st->V, V, 4 * (size_t)st->k, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) st->t = t;
+    return (int)e;
+}
+
+SGC_API int sgc_clear_status(sgc_state* st) {
+    if (!st) return SGC_ERR_NULL;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    if (e == cudaSuccess) e = cudaMemset(&st->cnt->status, 0, 4);
+    return (int)e;
+}
+
+SGC_API int sgc_last_launches(sgc_state* st, int32_t* out) {
+    if (!st || !out) return SGC_ERR_NULL;
+    *out = st->last_launches;
+    return SGC_OK;
+}
+
+SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out, void* stream) {
+    if (!out) return SGC_ERR_NULL;
+    if (row0 < 0 || nrows < 0 || col0 < 0 || ncols < 0 || col0 + ncols > ((int64_t)1 << 32) ||
+        row0 + nrows > ((int64_t)1 << 32))
+        return SGC_ERR_DIM;
+    return (int)sgc::launch_z_block(seed, row0, nrows, col0, ncols, out, static_cast<cudaStream_t>(stream));
+}
+
+SGC_API const char* sgc_strerror(int code) {
+    switch (code) {
+        case SGC_OK: return "success";
+        case SGC_ERR_NULL: return "a required pointer is NULL";
+        case SGC_ERR_DIM: return "dimension out of range (need 1 <= s <= min(k, d), d < 2^32, k <= 65536, s <= 1024)";
+        case SGC_ERR_HYPER: return "hyper-parameter out of range (beta in [0,1), eps > 0, finite lr and alpha)";
+        case SGC_ERR_ALIGN: return "grad and weight must be 16-byte aligned";
+        case SGC_ERR_WHAT: return "unknown record selector";
+        case SGC_ERR_SIZE: return "destination buffer too small";
+        case SGC_ERR_GROUP: return "states of a group must be distinct and share d, k, s and seed";
+        case SGC_ERR_NOSTEP: return "no step has run yet";
+        default: break;
+    }
+    if (code > 0) return cudaGetErrorString((cudaError_t)code);
+    return "unknown error";
+}
+
+SGC_API int sgc_version(void) { return 100; }
+
+}  // extern "C"

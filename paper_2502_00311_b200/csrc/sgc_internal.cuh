@@ -1,0 +1,119 @@
+// Internal declarations of the SGC CUDA library (sm_100a).  Not part of the public C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sgc.h"
+
+namespace sgc {
+
+// ------------------------------------------------------------------------------------------------
+// Measurement matrix: A[j][i] = sigma_k * Z(seed, j, i), never stored (Section 3.3 fixes only the law:
+// i.i.d. zero-mean normal entries of standard deviation 1/sqrt(k)).
+//
+// Z(seed, row, col):
+//   ck = mix32(mix32(col + 0x9E3779B9*seed_lo) ^ seed_hi),  mk = mix32(ck ^ 0x5BD1E995) | 1
+//   h  = ck + row*mk;  h ^= h >> 16;  h *= 0x85EBCA6B;  h ^= h >> 15
+//   S  = sum of the four bytes of h;  x = S - 510;  w = x*x
+//   z  = x * fma(fma(w, C2, C1), w, C0)      (fp32, round to nearest)
+//   Z  = z with the low 16 bits cleared       (exactly a bfloat16)
+// The byte sum is an Irwin-Hall(4) variable; the odd polynomial maps its quantiles onto the normal's.
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kGolden = 0x9E3779B9u;
+constexpr uint32_t kMulEntry = 0x85EBCA6Bu;
+constexpr uint32_t kStrideSalt = 0x5BD1E995u;
+constexpr uint32_t kC0 = 0x3bd72bb5u, kC1 = 0x30aad71cu, kC2 = 0x28f3f07fu;
+
+__host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
+    x ^= x >> 16; x *= 0x7feb352du;
+    x ^= x >> 15; x *= 0x846ca68bu;
+    x ^= x >> 16;
+    return x;
+}
+
+struct ColKey { uint32_t ck, mk; };
+
+__host__ __device__ __forceinline__ ColKey column_key(uint32_t seed_lo, uint32_t seed_hi, uint32_t col) {
+    ColKey c;
+    c.ck = mix32(mix32(col + kGolden * seed_lo) ^ seed_hi);
+    c.mk = mix32(c.ck ^ kStrideSalt) | 1u;
+    return c;
+}
+
+// h0 = ck + row*mk (the caller advances it by mk per row)
+__device__ __forceinline__ float z_from_word(uint32_t h0) {
+    uint32_t h = h0;
+    h ^= h >> 16; h *= kMulEntry; h ^= h >> 15;
+    // bytes summed straight into the mantissa of 2^23: the float 8388608 + S
+    const uint32_t sb = __dp4a(h, 0x01010101u, 0x4B000000u);
+    const float x = __uint_as_float(sb) - 8389118.0f;          // S - 510, exact
+    const float w = __fmul_rn(x, x);                           // exact (|x| <= 510)
+    float q = __fmaf_rn(w, __uint_as_float(kC2), __uint_as_float(kC1));
+    q = __fmaf_rn(q, w, __uint_as_float(kC0));
+    const float z = __fmul_rn(x, q);
+    return __uint_as_float(__float_as_uint(z) & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ uint16_t z_bf16_bits(float z) { return (uint16_t)(__float_as_uint(z) >> 16); }
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+// ------------------------------------------------------------------------------------------------
+// limits
+// ------------------------------------------------------------------------------------------------
+constexpr int kMaxK = 65536;
+constexpr int kMaxS = 1024;
+constexpr int kSelCap = 32768;          // candidate slots of the top-s filter
+constexpr int kSelBins = 4096;          // 12-bit magnitude histogram of the sample
+constexpr int kCorrThreads = 512;       // threads per block of the correlation pass
+constexpr int kCorrCols = 2;            // columns per thread and tile
+constexpr int kCorrTop = 2;             // candidates kept per block and residual
+constexpr int kRescoreCap = 16;         // candidates rescored in fp64 per iteration and residual
+constexpr int kBookThreads = 1024;
+
+struct Cand { float score; uint32_t idx; };
+
+// device-resident counters of one state
+struct Counters {
+    unsigned int status;        // sticky SGC_STATUS_* bits
+    unsigned int sel_count;     // candidates appended by the filter pass
+    unsigned int sel_ticket;    // blocks of the sample pass that have finished
+    unsigned int sel_tau;       // threshold on the sign-cleared bit pattern
+    int done[2];                // completed OMP iterations per residual (M^, V^)
+    int stopped[2];             // 1 once a residual's OMP has stopped early
+    int n_upd, mismatch, negv, pad;
+};
+
+}  // namespace sgc
+
+// the state behind the opaque handle
+struct sgc_state {
+    int64_t d; int32_t k, s; uint64_t seed; float lr, beta1, beta2, eps, alpha; int64_t t;
+    int device; int sm_count;
+    cudaStream_t last_stream; bool has_stream;
+    int32_t last_launches; bool stepped;
+    int corr_grid, corr_smem;
+    // device memory (one allocation, carved)
+    void* base; size_t bytes;
+    float *M, *V; double *p, *q;
+    uint32_t* sel_idx; float* sel_val;
+    double *y64, *r64;          // [2][k]
+    float2* r32;                // [k] (M^ residual, V^ residual)
+    unsigned long long* sel_cand; unsigned int* sel_hist;
+    sgc::Cand* corr_cand;       // [2][corr_grid][kCorrTop]
+    uint16_t* zsel;             // [2][s][k] selected columns of Z as bfloat16 bits
+    uint32_t* lam;              // [2][s]
+    double *F, *acoef, *x, *gvec, *cvec, *rnorm;   // [2][s*s], [2][s] ...
+    uint32_t* upd_idx; double* upd_val;
+    sgc::Counters* cnt;
+};
+
+namespace sgc {
+// launchers (each returns the cudaError_t of its launches); defined in the .cu files
+cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches);
+cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launches);
+cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches);
+cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
+                           cudaStream_t stream);
+cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
+}  // namespace sgc

@@ -1,0 +1,260 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on seeded inputs.
+
+Bar: index sets (top-s support, OMP supports, updated positions) bit-exact; p, q, M, V within 1e-5 and the
+recovered update within 1e-4, both as max-abs error relative to the largest reference magnitude.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from golden_util import read_z_golden
+from paper_2502_00311_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_STATE = 1e-5
+TOL_UPDATE = 1e-4
+
+
+@pytest.fixture(scope="module")
+def sgc():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2502_00311_b200 import binding
+    binding.lib()
+    return binding
+
+
+def rel(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return np.abs(a - b).max() / max(np.abs(b).max(), 1e-300)
+
+
+def cuda(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+# ---- the A generator ----------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", [0, 1, 0x123456789ABCDEF])
+def test_z_generator_bit_exact(sgc, seed):
+    blocks, xor, total = read_z_golden(seed)
+    for (r0, c0), want in blocks.items():
+        got = sgc.z_block(seed, r0, 32, c0, 32).cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, want)
+    for (r0, nr, c0, nc) in [(0, 300, 0, 257), (65000, 536, 4294967000, 296), (7, 1, 123456789, 1)]:
+        got = sgc.z_block(seed, r0, nr, c0, nc).cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), oracle.z_block(seed, r0, nr, c0, nc).view(np.uint32))
+
+
+# ---- a1 top-s -------------------------------------------------------------------------------------------
+def run_select(sgc, g, s, k=None):
+    d = g.size
+    k = k or max(s, 8)
+    st = sgc.Sgc(d, k, s, 3, 1e-3, 0.9, 0.999, 1e-8)
+    w = cuda(np.zeros(d, dtype=np.float32))
+    st.step(cuda(g), w)
+    idx, val, status = st.get("sel_idx"), st.get("sel_val"), st.get("status")
+    st.close()
+    return idx, val, status
+
+
+@pytest.mark.parametrize("d,s", [(1, 1), (5, 5), (1023, 7), (4096, 16), (32768, 64), (32769, 64), (100003, 33),
+                                 (1 << 20, 256), (3_000_001, 1024)])
+def test_select_matches_oracle(sgc, d, s):
+    rng = np.random.default_rng(d + s)
+    g = (rng.standard_t(3.0, size=d) * 1e-3).astype(np.float32)
+    idx, val, status = run_select(sgc, g, s, k=max(s, 16))
+    widx, wval = oracle.sparsify(g, s)
+    assert np.array_equal(idx, widx) and np.array_equal(val, wval)
+    assert not status & sgc.STATUS_SELECT_FALLBACK
+
+
+def test_select_ties_and_degenerate_distributions(sgc):
+    # many equal magnitudes: the sampled threshold cannot separate them -> exact fallback, lowest indices win
+    d, s = 200_000, 20
+    g = np.full(d, 0.5, dtype=np.float32)
+    g[::3] *= -1
+    g[[17, 99_999, 150_000]] = [2.0, -3.0, 2.0]
+    idx, val, status = run_select(sgc, g, s)
+    widx, wval = oracle.sparsify(g, s)
+    assert np.array_equal(idx, widx) and np.array_equal(val, wval)
+    assert status & sgc.STATUS_SELECT_FALLBACK
+    # all zeros, signed zeros
+    g = np.zeros(70_000, dtype=np.float32)
+    g[1::2] = -0.0
+    idx, val, _ = run_select(sgc, g, 9)
+    assert idx.tolist() == list(range(9))
+    # Gaussian (light tails) and a constant-plus-spikes vector
+    rng = np.random.default_rng(0)
+    g = rng.standard_normal(2_000_000).astype(np.float32)
+    idx, val, status = run_select(sgc, g, 128, k=128)
+    widx, _ = oracle.sparsify(g, 128)
+    assert np.array_equal(idx, widx) and not status & sgc.STATUS_SELECT_FALLBACK
+
+
+def test_select_flags_non_finite_input(sgc):
+    g = np.random.default_rng(1).standard_normal(50_000).astype(np.float32)
+    g[1234] = np.nan
+    g[4321] = np.inf
+    _, _, status = run_select(sgc, g, 8)
+    assert status & sgc.STATUS_NONFINITE_INPUT
+
+
+# ---- whole step, config-1 shape and relatives -------------------------------------------------------------
+def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_support=False, compare_every=1):
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha)
+    ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha or 1.0)
+    supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0))
+    w0 = inputs.weights(d, 99)
+    w_gpu = cuda(w0.copy())
+    w_ref = w0.copy()
+    worst = dict(p=0.0, q=0.0, M=0.0, V=0.0, upd=0.0, x=0.0)
+    for step in range(1, steps + 1):
+        if redraw_support:
+            supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0) + 7919 * step)
+        g = inputs.gradient(d, kind, supp, sign, inputs.step_seed(cfg_id, 0, step))
+        w_before = w_ref.copy()
+        st.step(cuda(g), w_gpu)
+        ref.step(g, w_ref)
+        assert st.get("t") == step == ref.get("t")
+        assert np.array_equal(st.get("sel_idx"), ref.get("sel_idx"))
+        assert np.array_equal(st.get("sel_val"), ref.get("sel_val"))
+        for name in ("p", "q", "M", "V"):
+            worst[name] = max(worst[name], rel(st.get(name), ref.get(name)))
+        assert st.get("doneM") == ref.get("doneM") and st.get("doneV") == ref.get("doneV")
+        assert np.array_equal(st.get("lamM"), ref.get("lamM")), "OMP(M^) selection order differs at step %d" % step
+        assert np.array_equal(st.get("lamV"), ref.get("lamV")), "OMP(V^) selection order differs at step %d" % step
+        worst["x"] = max(worst["x"], rel(st.get("xM"), ref.get("xM")), rel(st.get("xV"), ref.get("xV")))
+        n = int(ref.get("n_upd"))
+        assert st.get("n_upd") == n and st.get("mismatch") == ref.get("mismatch") and st.get("negv") == ref.get("negv")
+        assert np.array_equal(st.get("upd_idx")[:n], ref.get("upd_idx")[:n])
+        if n:
+            worst["upd"] = max(worst["upd"], rel(st.get("upd_val")[:n], ref.get("upd_val")[:n]))
+        wg = w_gpu.cpu().numpy()
+        touched = np.zeros(d, dtype=bool)
+        touched[ref.get("upd_idx")[:n]] = True
+        assert np.array_equal(wg[~touched], w_before[~touched])            # nothing else is written
+        if n:
+            dw_g = wg[touched].astype(np.float64) - w_before[touched]
+            dw_r = w_ref[touched].astype(np.float64) - w_before[touched]
+            assert np.abs(dw_g - dw_r).max() <= TOL_UPDATE * np.abs(dw_r).max() + 1.2e-7 * np.abs(w_before[touched]).max()
+    for name in ("p", "q", "M", "V"):
+        assert worst[name] < TOL_STATE, (name, worst[name])
+    assert worst["x"] < TOL_UPDATE and worst["upd"] < TOL_UPDATE, worst
+    status = st.get("status")
+    st.close()
+    ref.close()
+    return worst, status
+
+
+def test_config1_ten_steps(sgc):
+    # 64x64 matrix, k=256, s=16, N(0, 0.1^2) noise + 16 planted U(1,2) entries, seed 0, 10 steps
+    worst, status = run_both(sgc, 4096, 256, 16, 0, "gauss", 10, cfg_id=1)
+    assert not status & (sgc.STATUS_CANDIDATE_OVERFLOW | sgc.STATUS_SELECT_FALLBACK | sgc.STATUS_NONFINITE_INPUT)
+
+
+@pytest.mark.parametrize("d,k,s", [(1000, 64, 1), (4099, 96, 12), (70_001, 333, 17), (1 << 17, 512, 64)])
+def test_awkward_shapes(sgc, d, k, s):
+    # d not a multiple of 4 or of the tile, k not a multiple of 32, s = 1 and s = k/8
+    run_both(sgc, d, k, s, 5, "student", 3, cfg_id=2)
+
+
+def test_alpha_and_redrawn_supports(sgc):
+    # alpha = 2 as in the paper's experiments; the planted support is redrawn every step so that M^ and V^
+    # stop being s-sparse and the recovery is inexact (supports of the two recoveries may differ)
+    run_both(sgc, 20_000, 256, 8, 11, "student", 6, cfg_id=2, alpha=2.0, redraw_support=True)
+
+
+def test_constant_sparse_gradient_closed_form(sgc):
+    # exactly s non-zeros held constant: N = alpha*sign(g) on the support, W_t = W_0 - t*lr*alpha*sign(g)
+    d, k, s, lr = 50_000, 512, 10, 1e-3
+    rng = np.random.default_rng(8)
+    supp = np.sort(rng.choice(d, size=s, replace=False))
+    g = np.zeros(d, dtype=np.float32)
+    g[supp] = (rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
+    w0 = rng.standard_normal(d).astype(np.float32)
+    st = sgc.Sgc(d, k, s, 2, lr, 0.9, 0.999, 1e-8)
+    w = cuda(w0.copy())
+    gd = cuda(g)
+    for t in range(1, 5):
+        st.step(gd, w)
+        assert sorted(st.get("lamM").tolist()) == supp.tolist() == sorted(st.get("lamV").tolist())
+    want = w0.astype(np.float64)
+    want[supp] -= 4 * lr * np.sign(g[supp])
+    np.testing.assert_allclose(w.cpu().numpy(), want, rtol=0, atol=3e-6)
+    st.close()
+
+
+def test_dependent_column_stops_like_the_oracle(sgc):
+    # k = 2: a third column is always dependent; both sides stop after two iterations
+    d, k, s = 64, 2, 2
+    g = np.random.default_rng(3).standard_normal(d).astype(np.float32)
+    st = sgc.Sgc(d, k, s, 3, 1e-3, 0.9, 0.999, 1e-8)
+    ref = oracle.Oracle(d, k, s, 3, 1e-3, 0.9, 0.999, 1e-8)
+    w = cuda(np.zeros(d, dtype=np.float32))
+    wr = np.zeros(d, dtype=np.float32)
+    st.step(cuda(g), w)
+    ref.step(g, wr)
+    assert st.get("doneM") == ref.get("doneM") and np.array_equal(st.get("lamM"), ref.get("lamM"))
+    st.close()
+
+
+def test_state_set_get_roundtrip_and_resume(sgc):
+    d, k, s = 30_000, 128, 6
+    hp = inputs.ADAM
+    supp, sign = inputs.planted_support(d, s, 5)
+    gs = [inputs.gradient(d, "student", supp, sign, 100 + i) for i in range(4)]
+    a = sgc.Sgc(d, k, s, 9, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    wa = cuda(inputs.weights(d, 1))
+    for g in gs[:2]:
+        a.step(cuda(g), wa)
+    b = sgc.Sgc(d, k, s, 9, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    b.set_state(a.get("M"), a.get("V"), int(a.get("t")))
+    wb = wa.clone()
+    for g in gs[2:]:
+        a.step(cuda(g), wa)
+        b.step(cuda(g), wb)
+    assert np.array_equal(a.get("M"), b.get("M")) and np.array_equal(wa.cpu().numpy(), wb.cpu().numpy())
+    a.close()
+    b.close()
+
+
+def test_group_equals_independent_steps(sgc):
+    d, k, s, n = 40_000, 256, 8, 3
+    hp = inputs.ADAM
+    solo = [sgc.Sgc(d, k, s, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(n)]
+    grp = [sgc.Sgc(d, k, s, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(n)]
+    ws = [cuda(inputs.weights(d, 10 + i)) for i in range(n)]
+    wg = [w.clone() for w in ws]
+    for step in range(2):
+        gr = []
+        for i in range(n):
+            supp, sign = inputs.planted_support(d, s, 50 + i)
+            gr.append(cuda(inputs.gradient(d, "student", supp, sign, 1000 * i + step)))
+        for i in range(n):
+            solo[i].step(gr[i], ws[i])
+        sgc.step_group(grp, gr, wg)
+        for i in range(n):
+            assert np.array_equal(solo[i].get("lamM"), grp[i].get("lamM"))
+            assert np.array_equal(ws[i].cpu().numpy(), wg[i].cpu().numpy())
+    with pytest.raises(sgc.SgcError):
+        other = sgc.Sgc(d, k, s, 5, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+        sgc.step_group([grp[0], other], gr[:2], wg[:2])
+    for st in solo + grp:
+        st.close()
+
+
+def test_step_rejects_misaligned_pointers(sgc):
+    import torch
+    st = sgc.Sgc(1000, 16, 2, 0, 1e-3, 0.9, 0.999, 1e-8)
+    buf = torch.zeros(1001, dtype=torch.float32, device="cuda")
+    good = torch.zeros(1000, dtype=torch.float32, device="cuda")
+    with pytest.raises(sgc.SgcError) as e:
+        st.step(buf[1:], good)
+    assert e.value.code == -4
+    with pytest.raises(sgc.SgcError):
+        st.get("p")          # no step has run yet
+    st.close()
