@@ -137,6 +137,15 @@ SGC_API int sgc_clear_status(sgc_state* st);
 /* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out);
 
+/* Per-kernel timing of the steps that follow (no counterpart in the paper: measurement support).
+ * While enabled, sgc_step brackets every kernel launch with CUDA events on the caller's stream;
+ * sgc_get_profile synchronises and returns the totals accumulated since sgc_set_profile(st, 1):
+ *   ms[0] top-s sample    ms[1] top-s filter (the pass over the gradient)   ms[2] top-s pick
+ *   ms[3] projection+Adam ms[4] correlation passes   ms[5] OMP bookkeeping   ms[6] combine+scatter
+ *   launches[i] = number of kernel launches behind ms[i].   Both are host arrays of 8 entries. */
+SGC_API int sgc_set_profile(sgc_state* st, int enable);
+SGC_API int sgc_get_profile(sgc_state* st, float* ms, int32_t* launches);
+
 /* Fills a device buffer with Z(seed, row0 + r, col0 + c), r < nrows, c < ncols, row-major
  * (the A definition above without the scale); for checking the generator.
  *   out   device pointer, nrows*ncols floats */

@@ -13,7 +13,7 @@ _LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
 _lib = None
 
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
-           "sgc_clear_status", "sgc_last_launches", "sgc_z_block", "sgc_strerror", "sgc_version"]
+           "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_z_block", "sgc_strerror", "sgc_version"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -66,6 +66,10 @@ def lib():
         L.sgc_clear_status.argtypes = [vp]
         L.sgc_last_launches.restype = C.c_int
         L.sgc_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
+        L.sgc_set_profile.restype = C.c_int
+        L.sgc_set_profile.argtypes = [vp, C.c_int]
+        L.sgc_get_profile.restype = C.c_int
+        L.sgc_get_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.sgc_z_block.restype = C.c_int
         L.sgc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, vp]
         L.sgc_strerror.restype = C.c_char_p
@@ -156,6 +160,17 @@ class Sgc:
         n = C.c_int32(0)
         _check(lib().sgc_last_launches(self._h, C.byref(n)), "sgc_last_launches")
         return n.value
+
+    def set_profile(self, enable):
+        _check(lib().sgc_set_profile(self._h, 1 if enable else 0), "sgc_set_profile")
+
+    def get_profile(self):
+        """Per-phase totals since set_profile(True): dict phase -> (ms, launches)."""
+        ms = (C.c_float * 8)()
+        n = (C.c_int32 * 8)()
+        _check(lib().sgc_get_profile(self._h, ms, n), "sgc_get_profile")
+        names = ("select_sample", "select_filter", "select_pick", "project_adam", "corr", "book", "scatter")
+        return {names[i]: (float(ms[i]), int(n[i])) for i in range(7)}
 
     def close(self):
         if getattr(self, "_h", None):

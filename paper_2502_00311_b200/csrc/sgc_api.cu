@@ -63,6 +63,9 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
     sgc_state* st = new (std::nothrow) sgc_state();
     if (!st) return (int)cudaErrorMemoryAllocation;
     memset(st, 0, sizeof(*st));
+    st->ev_pool = new (std::nothrow) std::vector<cudaEvent_t>();
+    st->ev_phase = new (std::nothrow) std::vector<int>();
+    if (!st->ev_pool || !st->ev_phase) { delete st->ev_pool; delete st->ev_phase; delete st; return (int)cudaErrorMemoryAllocation; }
     st->d = d; st->k = k; st->s = s; st->seed = seed; st->lr = lr; st->beta1 = beta1; st->beta2 = beta2; st->eps = eps;
     st->alpha = 1.0f; st->t = 0;
     cudaError_t e = cudaGetDevice(&st->device);
@@ -78,6 +81,7 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
     }
     if (e != cudaSuccess) {
         if (st->base) cudaFree(st->base);
+        delete st->ev_pool; delete st->ev_phase;
         delete st;
         return (int)e;
     }
@@ -121,6 +125,8 @@ SGC_API int sgc_destroy(sgc_state* st) {
     cudaError_t e = cudaSuccess;
     if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
     cudaError_t e2 = cudaFree(st->base);
+    for (cudaEvent_t ev : *st->ev_pool) cudaEventDestroy(ev);
+    delete st->ev_pool; delete st->ev_phase;
     delete st;
     return (int)(e != cudaSuccess ? e : e2);
 }
@@ -196,6 +202,38 @@ SGC_API int sgc_clear_status(sgc_state* st) {
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out) {
     if (!st || !out) return SGC_ERR_NULL;
     *out = st->last_launches;
+    return SGC_OK;
+}
+
+// folds the recorded event pairs into the per-phase totals (the stream must have drained)
+static void drain_profile(sgc_state* st) {
+    for (size_t i = 0; i + 1 < st->ev_used; i += 2) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, (*st->ev_pool)[i], (*st->ev_pool)[i + 1]) == cudaSuccess)
+            st->prof_ms[(*st->ev_phase)[i / 2]] += ms;
+    }
+    st->ev_used = 0;
+    st->ev_phase->clear();
+}
+
+SGC_API int sgc_set_profile(sgc_state* st, int enable) {
+    if (!st) return SGC_ERR_NULL;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    st->ev_used = 0;
+    st->ev_phase->clear();
+    for (int i = 0; i < sgc::kNumPhases; ++i) { st->prof_ms[i] = 0.0f; st->prof_launches[i] = 0; }
+    st->profile = enable != 0;
+    return (int)e;
+}
+
+SGC_API int sgc_get_profile(sgc_state* st, float* ms, int32_t* launches) {
+    if (!st || !ms || !launches) return SGC_ERR_NULL;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    if (e != cudaSuccess) return (int)e;
+    drain_profile(st);
+    for (int i = 0; i < sgc::kNumPhases; ++i) { ms[i] = st->prof_ms[i]; launches[i] = st->prof_launches[i]; }
     return SGC_OK;
 }
 

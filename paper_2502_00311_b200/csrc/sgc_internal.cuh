@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "sgc.h"
 
 namespace sgc {
@@ -93,6 +95,11 @@ struct sgc_state {
     cudaStream_t last_stream; bool has_stream;
     int32_t last_launches; bool stepped;
     int corr_grid, corr_smem;
+    // optional per-kernel timing (sgc_set_profile)
+    bool profile;
+    std::vector<cudaEvent_t>* ev_pool; size_t ev_used;
+    std::vector<int>* ev_phase;          // phase of each (start, stop) event pair
+    float prof_ms[8]; int32_t prof_launches[8];
     // device memory (one allocation, carved)
     void* base; size_t bytes;
     float *M, *V; double *p, *q;
@@ -109,6 +116,30 @@ struct sgc_state {
 };
 
 namespace sgc {
+enum Phase { kPhaseSample = 0, kPhaseFilter = 1, kPhasePick = 2, kPhaseProject = 3, kPhaseCorr = 4, kPhaseBook = 5,
+             kPhaseScatter = 6, kNumPhases = 8 };
+
+// Brackets the launches issued during its lifetime with a pair of events when profiling is on.
+struct PhaseTimer {
+    sgc_state* st; cudaStream_t stream; bool on;
+    PhaseTimer(sgc_state* s, cudaStream_t cs, int phase, int n_launches) : st(s), stream(cs), on(s->profile) {
+        if (!on) return;
+        while (st->ev_pool->size() < st->ev_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+            st->ev_pool->push_back(e);
+        }
+        st->ev_phase->push_back(phase);
+        st->prof_launches[phase] += n_launches;
+        cudaEventRecord((*st->ev_pool)[st->ev_used], stream);
+    }
+    ~PhaseTimer() {
+        if (!on) return;
+        cudaEventRecord((*st->ev_pool)[st->ev_used + 1], stream);
+        st->ev_used += 2;
+    }
+};
+
 // launchers (each returns the cudaError_t of its launches); defined in the .cu files
 cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches);
 cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launches);

@@ -66,6 +66,7 @@ cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launche
     const double sigma = (double)(float)(1.0 / sqrt((double)st->k));
     const int grid = (st->k + kProjThreads - 1) / kProjThreads;
     const size_t smem = (size_t)st->s * (sizeof(ColKey) + sizeof(float));
+    PhaseTimer timer(st, stream, kPhaseProject, 1);
     k_project_adam<<<grid, kProjThreads, smem, stream>>>((uint32_t)(st->seed & 0xFFFFFFFFu), (uint32_t)(st->seed >> 32),
                                                          st->k, st->s, st->sel_idx, st->sel_val, st->M, st->V, st->p,
                                                          st->q, st->y64, st->r64, st->r32, st->cnt, sigma, b1, b2, c1, c2);

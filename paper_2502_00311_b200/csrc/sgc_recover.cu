@@ -381,11 +381,18 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
     a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
     a.cnt = st->cnt;
     for (int it = 0; it < st->s; ++it) {
-        k_corr<kCorrCols><<<st->corr_grid, kCorrThreads, st->corr_smem, stream>>>(
-            seed_lo, seed_hi, (unsigned long long)st->d, st->k, st->s, st->r32, st->lam, st->cnt, st->corr_cand, tiles);
-        k_book<<<2, kBookThreads, 0, stream>>>(a, it);
+        {
+            PhaseTimer timer(st, stream, kPhaseCorr, 1);
+            k_corr<kCorrCols><<<st->corr_grid, kCorrThreads, st->corr_smem, stream>>>(
+                seed_lo, seed_hi, (unsigned long long)st->d, st->k, st->s, st->r32, st->lam, st->cnt, st->corr_cand, tiles);
+        }
+        {
+            PhaseTimer timer(st, stream, kPhaseBook, 1);
+            k_book<<<2, kBookThreads, 0, stream>>>(a, it);
+        }
         *launches += 2;
     }
+    PhaseTimer timer(st, stream, kPhaseScatter, 1);
     k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weight, st->upd_idx, st->upd_val,
                                               (double)st->alpha, (double)st->eps, (double)st->lr);
     *launches += 1;

@@ -248,15 +248,24 @@ cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream,
     if (target < 32ull) target = 32ull;
     int sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
     if (sample_grid < 1) sample_grid = 1;
-    k_sample<<<direct ? 1 : sample_grid, kSampleThreads, 0, stream>>>(grad, d, (unsigned int)n_chunks, (unsigned int)target,
-                                                                      st->sel_hist, st->cnt, direct);
+    {
+        PhaseTimer timer(st, stream, kPhaseSample, 1);
+        k_sample<<<direct ? 1 : sample_grid, kSampleThreads, 0, stream>>>(grad, d, (unsigned int)n_chunks, (unsigned int)target,
+                                                                          st->sel_hist, st->cnt, direct);
+    }
     unsigned long long n4 = d >> 2;
     unsigned long long blocks = (n4 + 512ull * 4ull - 1) / (512ull * 4ull);
     const unsigned long long max_blocks = (unsigned long long)st->sm_count * 4ull;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
-    k_filter<<<(unsigned int)blocks, 512, 0, stream>>>(grad, d, st->sel_cand, st->cnt);
-    k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)st->s, st->sel_cand, st->cnt, st->sel_idx, st->sel_val);
+    {
+        PhaseTimer timer(st, stream, kPhaseFilter, 1);
+        k_filter<<<(unsigned int)blocks, 512, 0, stream>>>(grad, d, st->sel_cand, st->cnt);
+    }
+    {
+        PhaseTimer timer(st, stream, kPhasePick, 1);
+        k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)st->s, st->sel_cand, st->cnt, st->sel_idx, st->sel_val);
+    }
     *launches += 3;
     return cudaGetLastError();
 }
