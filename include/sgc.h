@@ -137,6 +137,26 @@ SGC_API int sgc_clear_status(sgc_state* st);
 /* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out);
 
+/* Top-s selection (step a1 alone) for callers that cannot allocate device memory.  The paper has no
+ * counterpart: this is the same selection that sgc_step performs first, offered on its own with its
+ * scratch (278 784 bytes: threshold histogram, candidate list, counters) held in a static device array
+ * inside the library instead of in a state object.  Meant for hosts where a cudaMalloc is off the table at
+ * call time, e.g. a framework that has already claimed all device memory for its own pool, or a thread
+ * that cannot afford cudaMalloc's device-wide synchronisation.  The call makes no cudaMalloc/cudaFree and
+ * uses no allocating routine.
+ *   grad        device pointer, d floats, 16-byte aligned, read only
+ *   d, s        1 <= s <= min(d, 1024), d < 2^32; anything larger is rejected with SGC_ERR_DIM
+ *   out_idx     device pointer, s uint32: positions of the s largest |g| (ties -> lower index), ascending
+ *   out_val     device pointer, s floats: the gradient values at those positions
+ *   out_status  device pointer to one uint32 receiving SGC_STATUS_* bits of this call, or NULL
+ *   stream      a cudaStream_t; all work is enqueued there, the call does not synchronise
+ * The first call on each device looks up the device address of the static array (cudaGetSymbolAddress)
+ * and should therefore come before any stream capture.  Every call on a device shares that array and
+ * finds the previous call's contents in it: what must start at zero is cleared on `stream` first.  Calls
+ * that overlap on the GPU race on the array; serialise them (one stream, or events between streams). */
+SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t s, uint32_t* out_idx, float* out_val,
+                                uint32_t* out_status, void* stream);
+
 /* Per-kernel timing of the steps that follow (no counterpart in the paper: measurement support).
  * While enabled, sgc_step brackets every kernel launch with CUDA events on the caller's stream;
  * sgc_get_profile synchronises and returns the totals accumulated since sgc_set_profile(st, 1):

@@ -13,7 +13,7 @@ _LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
 _lib = None
 
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
-           "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_z_block", "sgc_strerror", "sgc_version"]
+           "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block", "sgc_strerror", "sgc_version"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -70,6 +70,8 @@ def lib():
         L.sgc_set_profile.argtypes = [vp, C.c_int]
         L.sgc_get_profile.restype = C.c_int
         L.sgc_get_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        L.sgc_sparsify_static.restype = C.c_int
+        L.sgc_sparsify_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp, vp, vp]
         L.sgc_z_block.restype = C.c_int
         L.sgc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, vp]
         L.sgc_strerror.restype = C.c_char_p
@@ -117,6 +119,24 @@ def z_block(seed, row0, nrows, col0, ncols, stream=None):
     _check(lib().sgc_z_block(C.c_uint64(seed), row0, nrows, col0, ncols, C.c_void_p(out.data_ptr()),
                              _stream_ptr(stream)), "sgc_z_block")
     return out
+
+
+def sparsify_static(grad, s, out_idx, out_val, out_status=None, stream=None):
+    """sgc_sparsify_static: top-s selection into caller-provided CUDA tensors, without any device allocation.
+
+    For hosts that cannot call cudaMalloc when they need the selection (all device memory already handed to a
+    framework's pool, or a thread that must not trigger cudaMalloc's device-wide synchronisation).  out_idx:
+    int32/uint32-sized CUDA tensor of s elements, out_val: float32 CUDA tensor of s elements, out_status:
+    optional CUDA tensor holding one 32-bit word.  Calls on one device share a static scratch array inside the
+    library and must not overlap on the GPU.
+    """
+    d = grad.numel()
+    if out_idx.numel() < s or out_idx.element_size() != 4 or not out_idx.is_cuda or not out_idx.is_contiguous():
+        raise TypeError("out_idx must be a contiguous CUDA tensor of at least s 32-bit integers")
+    st_ptr = C.c_void_p(out_status.data_ptr()) if out_status is not None else C.c_void_p(0)
+    _check(lib().sgc_sparsify_static(_dev_ptr(grad, d, "grad"), d, int(s), C.c_void_p(out_idx.data_ptr()),
+                                     _dev_ptr(out_val, s, "out_val"), st_ptr, _stream_ptr(stream)),
+           "sgc_sparsify_static")
 
 
 class Sgc:

@@ -10,6 +10,8 @@
 // If the candidate list ends up with fewer than s or more than its capacity (degenerate value
 // distributions, e.g. all magnitudes equal), k_pick instead runs the same exact radix select over the
 // whole gradient (slow, still correct) and reports SGC_STATUS_SELECT_FALLBACK.
+#include <mutex>
+
 #include "sgc_internal.cuh"
 
 namespace sgc {
@@ -271,3 +273,101 @@ cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream,
 }
 
 }  // namespace sgc
+
+// ------------------------------------------------------------------------------------------------
+// sgc_sparsify_static: the top-s selection (a1) for callers that must not allocate device memory.
+//
+// Some hosts of this library cannot call cudaMalloc at the moment they need a selection: a training loop
+// whose framework has already claimed all device memory for its own caching allocator (a cudaMalloc from
+// a library then fails or fragments the pool), or a latency-critical thread for which cudaMalloc's implicit
+// device-wide synchronisation would stall every other stream.  For them the scratch that the selection
+// needs (threshold histogram, candidate list, counters: kStaticScratchBytes = 278 784 bytes) lives in a
+// file-scope __device__ array that every GPU loading this library holds until the process exits.
+//
+// The array's name is only a host-side handle; kernels need its device address, which the first call on
+// each device obtains with cudaGetSymbolAddress (that first call should therefore happen before any stream
+// capture).  The call itself allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
+// All calls on one device share the array, and it keeps the previous call's contents: the parts that must
+// start at zero are cleared on the caller's stream at the start of every call.  Two calls that overlap on
+// the GPU (different streams, or different host threads) race on the array and give undefined results.
+// ------------------------------------------------------------------------------------------------
+namespace sgc {
+namespace {
+
+constexpr size_t kStaticCntOff = 0;                                              // Counters (padded to 256)
+constexpr size_t kStaticHistOff = 256;                                           // u32[kSelBins]
+constexpr size_t kStaticCandOff = kStaticHistOff + sizeof(unsigned int) * kSelBins;   // u64[kSelCap]
+constexpr size_t kStaticScratchBytes = kStaticCandOff + sizeof(unsigned long long) * kSelCap;
+static_assert(sizeof(Counters) <= 256, "counter block must fit its slot");
+static_assert(kStaticScratchBytes == 278784, "documented size of the static scratch");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticSetup { bool ready; unsigned char* ptr; int sm_count; };
+StaticSetup g_static_setup[kMaxDevices];            // zero-initialised; written once per device
+std::mutex g_static_mutex;
+
+__global__ void k_copy_status(const Counters* __restrict__ cnt, uint32_t* __restrict__ out) { *out = cnt->status; }
+
+}  // namespace
+}  // namespace sgc
+
+extern "C" SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t s, uint32_t* out_idx, float* out_val,
+                                           uint32_t* out_status, void* stream) {
+    using namespace sgc;
+    if (!grad || !out_idx || !out_val) return SGC_ERR_NULL;
+    if (d < 1 || s < 1 || (int64_t)s > d || d >= ((int64_t)1 << 32) || s > kMaxS) return SGC_ERR_DIM;
+    if ((uintptr_t)grad & 15u) return SGC_ERR_ALIGN;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= kMaxDevices) return SGC_ERR_DIM;
+    StaticSetup setup;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_setup[dev].ready) {           // once per device, with that device current
+            void* p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_static_scratch);
+            if (e != cudaSuccess) return (int)e;
+            int sms = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return (int)e;
+            g_static_setup[dev].ptr = static_cast<unsigned char*>(p);
+            g_static_setup[dev].sm_count = sms;
+            g_static_setup[dev].ready = true;
+        }
+        setup = g_static_setup[dev];
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    Counters* cnt = reinterpret_cast<Counters*>(setup.ptr + kStaticCntOff);
+    unsigned int* hist = reinterpret_cast<unsigned int*>(setup.ptr + kStaticHistOff);
+    unsigned long long* cand = reinterpret_cast<unsigned long long*>(setup.ptr + kStaticCandOff);
+    // counters and histogram must start at zero; the candidate list is overwritten before it is read
+    e = cudaMemsetAsync(setup.ptr, 0, kStaticCandOff, cs);
+    if (e != cudaSuccess) return (int)e;
+    const unsigned long long du = (unsigned long long)d;
+    const int direct = du <= (unsigned long long)kSelCap;
+    unsigned long long n_chunks = du / 16384ull;
+    if (n_chunks < 1024ull) n_chunks = 1024ull;
+    if (n_chunks > 65536ull) n_chunks = 65536ull;
+    unsigned long long n_sample = n_chunks * kSampleChunk;
+    if (n_sample > du) n_sample = du;
+    unsigned long long want = 8ull * (unsigned long long)s;
+    if (want < 2048ull) want = 2048ull;
+    unsigned long long target = (want * n_sample + du - 1) / du;
+    if (target < 32ull) target = 32ull;
+    int sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
+    if (sample_grid < 1) sample_grid = 1;
+    k_sample<<<direct ? 1 : sample_grid, kSampleThreads, 0, cs>>>(grad, du, (unsigned int)n_chunks, (unsigned int)target,
+                                                                  hist, cnt, direct);
+    unsigned long long n4 = du >> 2;
+    unsigned long long blocks = (n4 + 512ull * 4ull - 1) / (512ull * 4ull);
+    const unsigned long long max_blocks = (unsigned long long)setup.sm_count * 4ull;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks < 1) blocks = 1;
+    k_filter<<<(unsigned int)blocks, 512, 0, cs>>>(grad, du, cand, cnt);
+    k_pick<<<1, kPickThreads, 0, cs>>>(grad, du, (unsigned int)s, cand, cnt, out_idx, out_val);
+    if (out_status) k_copy_status<<<1, 1, 0, cs>>>(cnt, out_status);
+    return (int)cudaGetLastError();
+}
