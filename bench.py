@@ -31,7 +31,8 @@ METRIC = "sgc_step_ms_per_4096x4096_matrix_k2048_s64"
 WORKLOADS = {
     "c2_4096x4096": dict(d=4096 * 4096, k=2048, s=64, seed=1, kind="student", cfg_id=2),
     "c1_64x64": dict(d=64 * 64, k=256, s=16, seed=0, kind="gauss", cfg_id=1),
-    "small_2M_k2048_s8": dict(d=1 << 21, k=2048, s=8, seed=1, kind="student", cfg_id=2),      # profiler-sized case
+    "small_2M_k2048_s8": dict(d=1 << 21, k=2048, s=8, seed=1, kind="student", cfg_id=2),      # profiler-sized cases
+    "small_2M_k2048_s64": dict(d=1 << 21, k=2048, s=64, seed=1, kind="student", cfg_id=2),
     "c5_4096x11008_k1024_s16": dict(d=4096 * 11008, k=1024, s=16, seed=1, kind="student", cfg_id=5),
 }
 FP32_LANES_PER_SM = 128
@@ -42,8 +43,9 @@ def peaks():
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return dict(hbm_gbs=float(p["hbm_gbs"]), source="measured", sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)))
-    return dict(hbm_gbs=6650.0, source="fallback", sm_max_mhz=1965.0)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]), source="measured",
+                    sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)))
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback", sm_max_mhz=1965.0)
 
 
 class ClockSampler:
@@ -163,6 +165,7 @@ def run_ours(args, wl):
     dev_grads = [g.cuda() for g in host_grads]
     weight = torch.from_numpy(inputs.weights(d, 99 + rank)).cuda()
     st = binding.Sgc(d, k, s, wl["seed"], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    st.set_mode(args.mode)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -187,10 +190,19 @@ def run_ours(args, wl):
     e1.record(stream)
     barrier()
     total_ms = e0.elapsed_time(e1)
-    prof = st.get_profile()
-    st.set_profile(False)
     clocks = sampler.stop()
     status = int(st.get("status"))
+    st.set_profile(False)
+    # per-kernel times and the number of screening passes that did work, from a second, instrumented run of the
+    # same steps (event pairs around every launch and a read-back of the round counter perturb the step time)
+    st.set_profile(True)
+    rounds = []
+    for i in range(args.steps):
+        st.step(dev_grads[(args.warmup + i) % ring], weight, stream)
+        rounds.append(int(st.get("rounds")))
+    prof = st.get_profile()
+    st.set_profile(False)
+    lockstep = int(st.get("fallback"))
 
     # ---- end to end: pinned host gradient -> device, step, update record -> host -----------------------
     stage = torch.empty(d, dtype=torch.float32, device="cuda")
@@ -218,11 +230,28 @@ def run_ours(args, wl):
 
     if rank == 0:
         pk = peaks()
-        corr_ms, corr_n = prof["corr"]
-        corr_avg_s = corr_ms / max(corr_n, 1) * 1e-3
-        flops_per_launch = 2.0 * k * d * 2                      # one fused multiply-add per generated entry and residual
-        alu_peak = 148 * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
-        achieved = flops_per_launch / corr_avg_s / 1e12
+        n_pass = 2 * min(128, (min(s, 128) + 15) // 16 * 16)     # residuals per screening pass (both recoveries)
+        pass_ms, _ = prof["pass"]
+        working = max(sum(rounds), 1)
+        if sum(rounds) > 0:
+            # dominant kernel: the tensor-core screening pass, C = A^T R with A generated on the fly
+            pass_avg_s = pass_ms / working * 1e-3
+            achieved = 2.0 * k * d * n_pass / pass_avg_s / 1e12
+            roof = {"kernel": "k_pass", "bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / pk["bf16_tflops"], "traffic": None, "peak_source": pk["source"],
+                    "note": "2*k*d*N flops per pass (N = %d residuals, bf16 x bf16 -> fp32 on tcgen05); the operand A is "
+                            "regenerated by the CUDA cores (k*d entries per pass), which is what limits the pass" % n_pass,
+                    "avg_launch_ms": pass_avg_s * 1e3, "launches": sum(rounds),
+                    "generated_entries_per_s": k * d / pass_avg_s}
+        else:
+            omp_ms, omp_n = prof["omp"]
+            it_s = omp_ms / max(args.steps * s, 1) * 1e-3
+            alu_peak = 148 * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+            achieved = 2.0 * k * d * 2 / it_s / 1e12
+            roof = {"kernel": "k_omp (lock-step)", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                    "frac": achieved / alu_peak, "traffic": None,
+                    "note": "useful fp32 FMA flops 2*k*d*2 per OMP iteration; peak = 148 SM * 128 lanes * 2 * sm_max_mhz",
+                    "avg_launch_ms": it_s * 1e3, "launches": omp_n}
         filt_ms, filt_n = prof["select_filter"]
         filt_gbs = 4.0 * d / (filt_ms / max(filt_n, 1) * 1e-3) / 1e9
         line = {
@@ -231,12 +260,9 @@ def run_ours(args, wl):
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "d": d, "k": k, "s": s, "seed_A": wl["seed"],
                        "l2": "%d rotating gradients of %.0f MiB (> 126 MB L2)" % (ring, d * 4 / 2 ** 20),
-                       "replicas": world, "status_word": status},
-            "roofline": {"kernel": "k_corr", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
-                         "frac": achieved / alu_peak, "traffic": None,
-                         "note": "useful fp32 FMA flops 2*k*d*2 per launch; peak = 148 SM * 128 lanes * 2 * sm_max_mhz "
-                                 "(derived); generating A costs ~13 more lane-ops per entry, so this fraction is capped "
-                                 "near 2/15", "avg_launch_ms": corr_avg_s * 1e3, "launches": corr_n},
+                       "replicas": world, "status_word": status, "recovery": "lock-step" if lockstep else "speculative",
+                       "screening_passes_per_step": rounds},
+            "roofline": roof,
             "roofline_select": {"kernel": "k_filter", "bound": "hbm", "achieved": filt_gbs, "peak": pk["hbm_gbs"],
                                 "unit": "GB/s", "frac": filt_gbs / pk["hbm_gbs"], "peak_source": pk["source"],
                                 "avg_launch_ms": filt_ms / max(filt_n, 1)},
@@ -267,6 +293,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_4096x4096", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", type=int, default=0, choices=[0, 1, 2], help="recovery: 0 auto, 1 lock-step, 2 speculative")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = WORKLOADS[args.workload]

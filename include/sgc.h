@@ -88,7 +88,17 @@ enum {
     SGC_GET_DONE_M = 17,    /* int32      completed OMP iterations for M^                       */
     SGC_GET_DONE_V = 18,    /* int32      completed OMP iterations for V^                       */
     SGC_GET_RNORM_M = 19,   /* double[s]  residual norm after each OMP(M^) iteration            */
-    SGC_GET_RNORM_V = 20    /* double[s]  same for OMP(V^)                                      */
+    SGC_GET_RNORM_V = 20,   /* double[s]  same for OMP(V^)                                      */
+    SGC_GET_ROUNDS = 21,    /* int32      screening passes over all d columns that the last step needed (speculative recovery) */
+    SGC_GET_FALLBACK = 22,  /* int32      1 when the last step finished (or ran entirely) in lock-step  */
+    SGC_GET_N_CAND = 23     /* int32      length of the candidate list kept for the next step           */
+};
+
+/* How the recovery (a4) finds the picks of Algorithm 3; the picks themselves do not depend on it. */
+enum {
+    SGC_MODE_AUTO = 0,        /* speculative when k is a multiple of 64 and d >= 65536, lock-step otherwise */
+    SGC_MODE_LOCKSTEP = 1,    /* one pass over all d columns per OMP iteration                             */
+    SGC_MODE_SPECULATIVE = 2  /* OMP on a candidate list, confirmed by batched tensor-core screening passes */
 };
 
 /* Problem statement of Section 3 (Eq. 3) with the method of Algorithm 2.
@@ -123,6 +133,13 @@ SGC_API int sgc_destroy(sgc_state* st);
 
 /* alpha of Eq. (8) ("a scaling factor"); must be finite. */
 SGC_API int sgc_set_alpha(sgc_state* st, float alpha);
+
+/* Chooses the recovery strategy (SGC_MODE_*).  Both strategies return the picks of Algorithm 3 (Appendix B):
+ * the speculative one runs OMP on a short candidate list and then proves, with one tensor-core pass over all
+ * d columns against the residuals of all iterations at once, that no other column would have been picked; a
+ * refuted pick is replaced by the true argmax and the round repeats from there.
+ * SGC_ERR_DIM when SGC_MODE_SPECULATIVE is requested and k is not a multiple of 64. */
+SGC_API int sgc_set_mode(sgc_state* st, int32_t mode);
 
 /* Synchronises with the state's last step and copies one record to host memory (selectors above).
  *   dst    host pointer; bytes = its capacity, must cover the record */
@@ -161,7 +178,8 @@ SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t s, uint32_
  * While enabled, sgc_step brackets every kernel launch with CUDA events on the caller's stream;
  * sgc_get_profile synchronises and returns the totals accumulated since sgc_set_profile(st, 1):
  *   ms[0] top-s sample    ms[1] top-s filter (the pass over the gradient)   ms[2] top-s pick
- *   ms[3] projection+Adam ms[4] correlation passes   ms[5] OMP bookkeeping   ms[6] combine+scatter
+ *   ms[3] projection+Adam ms[4] OMP kernels (candidate-list and lock-step)   ms[5] resolve + bookkeeping
+ *   ms[6] combine+scatter ms[7] tensor-core screening passes
  *   launches[i] = number of kernel launches behind ms[i].   Both are host arrays of 8 entries. */
 SGC_API int sgc_set_profile(sgc_state* st, int enable);
 SGC_API int sgc_get_profile(sgc_state* st, float* ms, int32_t* launches);
@@ -170,6 +188,21 @@ SGC_API int sgc_get_profile(sgc_state* st, float* ms, int32_t* launches);
  * (the A definition above without the scale); for checking the generator.
  *   out   device pointer, nrows*ncols floats */
 SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out, void* stream);
+
+/* The screening pass of the recovery on its own ("Projection" of Algorithm 3 for n residuals at once):
+ * reports every pair (column i, residual j) with |<Z_i, R_j>| / ||Z_i|| >= tau[j], where Z_i is column i of
+ * the unscaled measurement matrix of (seed, k) and R_j row j of rt.  Runs on the tensor cores.
+ *   d, k        1 <= d < 2^32; k a multiple of 64, 64 <= k <= 65536
+ *   n           number of residuals, a multiple of 32, 32 <= n <= 256
+ *   rt          device pointer, n x k bfloat16 bit patterns, row-major, 16-byte aligned, read only
+ *   tau         device pointer, n floats (+infinity disables a residual)
+ *   rep_count   device pointer, n uint32: number of reports per residual (may exceed rep_cap)
+ *   rep         device pointer, n x rep_cap pairs (uint32 column, float score bits); the first
+ *               min(rep_count[j], rep_cap) pairs of row j are valid, in no particular order
+ *   error_flag  device pointer to one int32, set to 1 if the kernel gave up on an internal wait (results invalid)
+ * Everything is enqueued on stream; the call does not synchronise. */
+SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uint16_t* rt, const float* tau, uint32_t* rep_count,
+                       uint32_t* rep, int32_t rep_cap, int32_t* error_flag, void* stream);
 
 /* Human-readable text for a return code of this library (static storage). */
 SGC_API const char* sgc_strerror(int code);

@@ -13,7 +13,8 @@ _LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
 _lib = None
 
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
-           "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block", "sgc_strerror", "sgc_version"]
+           "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
+           "sgc_set_mode", "sgc_screen", "sgc_strerror", "sgc_version"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -22,7 +23,10 @@ RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, 
                upd_idx=(11, np.uint32, "s"), upd_val=(12, np.float64, "s"), n_upd=(13, np.int32, None),
                status=(14, np.uint32, None), mismatch=(15, np.int32, None), negv=(16, np.int32, None),
                doneM=(17, np.int32, None), doneV=(18, np.int32, None), rnormM=(19, np.float64, "s"),
-               rnormV=(20, np.float64, "s"))
+               rnormV=(20, np.float64, "s"), rounds=(21, np.int32, None), fallback=(22, np.int32, None),
+               n_cand=(23, np.int32, None))
+
+MODE_AUTO, MODE_LOCKSTEP, MODE_SPECULATIVE = 0, 1, 2
 
 STATUS_NONFINITE_INPUT = 1
 STATUS_DEPENDENT_COLUMN = 2
@@ -74,6 +78,10 @@ def lib():
         L.sgc_sparsify_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp, vp, vp]
         L.sgc_z_block.restype = C.c_int
         L.sgc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, vp]
+        L.sgc_set_mode.restype = C.c_int
+        L.sgc_set_mode.argtypes = [vp, C.c_int32]
+        L.sgc_screen.restype = C.c_int
+        L.sgc_screen.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32, vp, vp, vp, vp, C.c_int32, vp, vp]
         L.sgc_strerror.restype = C.c_char_p
         L.sgc_strerror.argtypes = [C.c_int]
         L.sgc_version.restype = C.c_int
@@ -121,6 +129,23 @@ def z_block(seed, row0, nrows, col0, ncols, stream=None):
     return out
 
 
+def screen(seed, d, k, rt, tau, rep_cap, stream=None):
+    """sgc_screen: tensor-core screening pass.  rt: CUDA int16/uint16-sized tensor [n, k] of bfloat16 bit patterns
+    (or a torch.bfloat16 tensor), tau: float32 CUDA tensor [n].  Returns (rep_count [n] int32, rep [n, rep_cap, 2] int32
+    holding (column, score bits), error_flag [1] int32) as CUDA tensors; nothing is synchronised."""
+    import torch
+    n = rt.shape[0]
+    if rt.element_size() != 2 or not rt.is_cuda or not rt.is_contiguous() or rt.shape[1] != k:
+        raise TypeError("rt must be a contiguous CUDA tensor [n, k] of 16-bit elements")
+    rep_count = torch.empty(n, dtype=torch.int32, device="cuda")
+    rep = torch.empty((n, rep_cap, 2), dtype=torch.int32, device="cuda")
+    err = torch.empty(1, dtype=torch.int32, device="cuda")
+    _check(lib().sgc_screen(C.c_uint64(seed), int(d), int(k), int(n), C.c_void_p(rt.data_ptr()), _dev_ptr(tau, n, "tau"),
+                            C.c_void_p(rep_count.data_ptr()), C.c_void_p(rep.data_ptr()), int(rep_cap),
+                            C.c_void_p(err.data_ptr()), _stream_ptr(stream)), "sgc_screen")
+    return rep_count, rep, err
+
+
 def sparsify_static(grad, s, out_idx, out_val, out_status=None, stream=None):
     """sgc_sparsify_static: top-s selection into caller-provided CUDA tensors, without any device allocation.
 
@@ -150,6 +175,9 @@ class Sgc:
         self._h = h
         if alpha is not None:
             self.set_alpha(alpha)
+
+    def set_mode(self, mode):
+        _check(lib().sgc_set_mode(self._h, int(mode)), "sgc_set_mode")
 
     def set_alpha(self, alpha):
         _check(lib().sgc_set_alpha(self._h, alpha), "sgc_set_alpha")
@@ -189,8 +217,8 @@ class Sgc:
         ms = (C.c_float * 8)()
         n = (C.c_int32 * 8)()
         _check(lib().sgc_get_profile(self._h, ms, n), "sgc_get_profile")
-        names = ("select_sample", "select_filter", "select_pick", "project_adam", "corr", "book", "scatter")
-        return {names[i]: (float(ms[i]), int(n[i])) for i in range(7)}
+        names = ("select_sample", "select_filter", "select_pick", "project_adam", "omp", "resolve", "scatter", "pass")
+        return {names[i]: (float(ms[i]), int(n[i])) for i in range(8)}
 
     def close(self):
         if getattr(self, "_h", None):

@@ -41,6 +41,18 @@ size_t layout(sgc_state* st, unsigned char* base) {
     st->upd_idx = carve<uint32_t>(base, off, s);
     st->upd_val = carve<double>(base, off, s);
     st->cnt = carve<sgc::Counters>(base, off, 1);
+    st->ctl = carve<sgc::SpecCtl>(base, off, 1);
+    if (st->spec_ok) {
+        const size_t n = (size_t)st->pass_n;
+        st->rt = carve<uint16_t>(base, off, n * k);
+        st->tau = carve<float>(base, off, n);
+        st->rep_count = carve<unsigned int>(base, off, n);
+        st->rep = carve<uint2>(base, off, n * sgc::kRepCap);
+        st->pick_score = carve<double>(base, off, 2 * s);
+        st->cand_list = carve<uint32_t>(base, off, sgc::kCandCap);
+        st->cand_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
+        st->rtmp = carve<double>(base, off, k);
+    }
     return off;
 }
 
@@ -77,8 +89,9 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
     }
     if (e == cudaSuccess) {
         layout(st, static_cast<unsigned char*>(st->base));
-        e = cudaMemset(st->base, 0, st->bytes);        // M_0 = V_0 = 0, counters, histogram
+        e = cudaMemset(st->base, 0, st->bytes);        // M_0 = V_0 = 0, counters, histogram, empty candidate list
     }
+    if (e == cudaSuccess) e = sgc::finish_recover_setup(st);
     if (e != cudaSuccess) {
         if (st->base) cudaFree(st->base);
         delete st->ev_pool; delete st->ev_phase;
@@ -138,6 +151,14 @@ SGC_API int sgc_set_alpha(sgc_state* st, float alpha) {
     return SGC_OK;
 }
 
+SGC_API int sgc_set_mode(sgc_state* st, int32_t mode) {
+    if (!st) return SGC_ERR_NULL;
+    if (mode < SGC_MODE_AUTO || mode > SGC_MODE_SPECULATIVE) return SGC_ERR_WHAT;
+    if (mode == SGC_MODE_SPECULATIVE && !st->spec_ok) return SGC_ERR_DIM;
+    st->mode = mode;
+    return SGC_OK;
+}
+
 SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
     if (!st || !dst) return SGC_ERR_NULL;
     const size_t k = (size_t)st->k, s = (size_t)st->s;
@@ -170,6 +191,9 @@ SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
         case SGC_GET_DONE_V: src = &st->cnt->done[1]; n = 4; break;
         case SGC_GET_RNORM_M: src = st->rnorm; n = 8 * s; break;
         case SGC_GET_RNORM_V: src = st->rnorm + s; n = 8 * s; break;
+        case SGC_GET_ROUNDS: src = &st->ctl->rounds; n = 4; break;
+        case SGC_GET_FALLBACK: src = &st->ctl->fallback; n = 4; break;
+        case SGC_GET_N_CAND: src = &st->ctl->n_cand; n = 4; break;
         default: return SGC_ERR_WHAT;
     }
     if (needs_step && !st->stepped) return SGC_ERR_NOSTEP;
@@ -245,11 +269,34 @@ SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0
     return (int)sgc::launch_z_block(seed, row0, nrows, col0, ncols, out, static_cast<cudaStream_t>(stream));
 }
 
+SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uint16_t* rt, const float* tau, uint32_t* rep_count,
+                       uint32_t* rep, int32_t rep_cap, int32_t* error_flag, void* stream) {
+    if (!rt || !tau || !rep_count || !rep || !error_flag) return SGC_ERR_NULL;
+    if (d < 1 || d >= ((int64_t)1 << 32) || k < 64 || k > sgc::kMaxK || k % 64 != 0 || n < 32 || n > sgc::kPassMaxN ||
+        n % 32 != 0 || rep_cap < 1)
+        return SGC_ERR_DIM;
+    if (((uintptr_t)rt & 15u) || ((uintptr_t)rep & 7u)) return SGC_ERR_ALIGN;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = sgc::pass_configure(n);
+    unsigned char map[sgc::kTensorMapBytes];
+    if (e == cudaSuccess) e = sgc::pass_encode_map(map, rt, n, k);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(rep_count, 0, sizeof(uint32_t) * (size_t)n, cs);
+    if (e == cudaSuccess) e = cudaMemsetAsync(error_flag, 0, sizeof(int32_t), cs);
+    if (e == cudaSuccess)
+        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, rep_count, reinterpret_cast<uint2*>(rep), rep_cap, nullptr,
+                             error_flag, sms, cs);
+    return (int)e;
+}
+
 SGC_API const char* sgc_strerror(int code) {
     switch (code) {
         case SGC_OK: return "success";
         case SGC_ERR_NULL: return "a required pointer is NULL";
-        case SGC_ERR_DIM: return "dimension out of range (need 1 <= s <= min(k, d), d < 2^32, k <= 65536, s <= 1024)";
+        case SGC_ERR_DIM: return "dimension out of range (need 1 <= s <= min(k, d), d < 2^32, k <= 65536, s <= 1024; "
+                                 "the speculative recovery and sgc_screen need k to be a multiple of 64)";
         case SGC_ERR_HYPER: return "hyper-parameter out of range (beta in [0,1), eps > 0, finite lr and alpha)";
         case SGC_ERR_ALIGN: return "grad and weight must be 16-byte aligned";
         case SGC_ERR_WHAT: return "unknown record selector";
@@ -262,6 +309,6 @@ SGC_API const char* sgc_strerror(int code) {
     return "unknown error";
 }
 
-SGC_API int sgc_version(void) { return 100; }
+SGC_API int sgc_version(void) { return 200; }
 
 }  // extern "C"

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <vector>
 
@@ -72,8 +73,35 @@ constexpr int kCorrCols = 2;            // columns per thread and tile
 constexpr int kCorrTop = 2;             // candidates kept per block and residual
 constexpr int kRescoreCap = 16;         // candidates rescored in fp64 per iteration and residual
 constexpr int kBookThreads = 1024;
+constexpr int kOmpThreads = 1024;       // threads per block of the cooperative OMP kernel
+constexpr int kCandCap = 8192;          // candidate columns kept for the restricted (speculative) OMP
+constexpr int kCandKeep = 4096;         // the list is rebuilt from the supports once it grows beyond this
+constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
+constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
+constexpr int kMaxRounds = 8;           // speculate / screen / resolve rounds enqueued per step
+constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
+constexpr double kScreenMargin = 2.2e-3;  // bound on |score from bfloat16 residual - exact score| / ||r|| (2^-9 + slack)
+constexpr uint32_t kNoColumn = 0xFFFFFFFFu;
 
 struct Cand { float score; uint32_t idx; };
+
+// device-resident control block of the speculative recovery (one per state)
+struct SpecCtl {
+    int round_active;       // 1 while another speculate / screen / resolve round is needed
+    int fallback;           // 1: the remaining picks are made in lock-step over all columns
+    int v[2];               // verified picks per residual (M^, V^)
+    uint32_t forced[2];     // column that must become pick v[m] (the verified global winner), or kNoColumn
+    int base[2];            // first speculative pick of the current round
+    int hi[2];              // one past the last speculative pick of the current round
+    int extra[2];           // 1: the residual after pick hi-1 is screened without a pick (harvest + forced winner)
+    int dep[2];             // 1: pick hi-1 turned out linearly dependent on the support
+    int finished[2];        // recovery of this residual complete
+    int n_cand;             // length of the candidate list
+    int rounds;             // screening passes that did work in the last step
+    int pass_error;         // a wait inside the screening pass expired
+    int stop[2];            // scratch of the cooperative kernel: speculation of residual m has ended
+    double ynorm[2];        // ||y|| per residual
+};
 
 // device-resident counters of one state
 struct Counters {
@@ -95,6 +123,11 @@ struct sgc_state {
     cudaStream_t last_stream; bool has_stream;
     int32_t last_launches; bool stepped;
     int corr_grid, corr_smem;
+    int mode;                   // 0 auto, 1 lock-step only, 2 speculative whenever k allows it
+    bool spec_ok;               // speculative recovery usable for this (d, k)
+    int pass_n;                 // residuals per screening pass (multiple of 32, <= 256); pass_n / 2 per residual stream
+    double z_harvest, z_floor;  // thresholds of the screening pass in units of ||r|| / sqrt(k)
+    unsigned char tmap[128];    // CUtensorMap of the residual matrix R^T
     // optional per-kernel timing (sgc_set_profile)
     bool profile;
     std::vector<cudaEvent_t>* ev_pool; size_t ev_used;
@@ -113,11 +146,21 @@ struct sgc_state {
     double *F, *acoef, *x, *gvec, *cvec, *rnorm;   // [2][s*s], [2][s] ...
     uint32_t* upd_idx; double* upd_val;
     sgc::Counters* cnt;
+    // speculative recovery
+    sgc::SpecCtl* ctl;
+    uint16_t* rt;               // R^T [pass_n][k] bfloat16 bits: the residuals screened by one pass
+    float* tau;                 // [pass_n] thresholds
+    unsigned int* rep_count;    // [pass_n]
+    uint2* rep;                 // [pass_n][kRepCap] (column, score bits)
+    double* pick_score;         // [2][s] exact score |<Z_i, r>| / ||Z_i|| of every speculative pick
+    uint32_t* cand_list;        // [kCandCap]
+    unsigned int* cand_bits;    // bitmap over [0, d): membership in cand_list
+    double* rtmp;               // [k] scratch residual of the resolve kernel
 };
 
 namespace sgc {
 enum Phase { kPhaseSample = 0, kPhaseFilter = 1, kPhasePick = 2, kPhaseProject = 3, kPhaseCorr = 4, kPhaseBook = 5,
-             kPhaseScatter = 6, kNumPhases = 8 };
+             kPhaseScatter = 6, kPhasePass = 7, kNumPhases = 8 };
 
 // Brackets the launches issued during its lifetime with a pair of events when profiling is on.
 struct PhaseTimer {
@@ -147,4 +190,12 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
 cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
                            cudaStream_t stream);
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
+cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T
+
+// screening pass (sgc_pass.cu)
+int pass_stages(int n);
+cudaError_t pass_configure(int n);
+cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
+cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, unsigned int* rep_count,
+                        uint2* rep, int rep_cap, const int* gate, int* error, int sm_count, cudaStream_t stream);
 }  // namespace sgc

@@ -1,0 +1,391 @@
+// Screening pass of the recovery (a4): the "Projection" line of Algorithm 3, p = A^T r, for a whole batch of
+// residual vectors at once, as one dense contraction  C = A^T R  on the tcgen05 tensor cores.
+//
+//   A (k x d) is regenerated tile by tile by the CUDA cores straight into shared memory as bfloat16 (Z is
+//   exactly representable there), in the K-major 128-byte-swizzled layout the UMMA descriptors expect;
+//   R^T (N x k, bfloat16, one residual per row) arrives chunk by chunk through TMA;
+//   accumulators live in tensor memory (fp32, 128 lanes = 128 columns of A, N columns each);
+//   the epilogue reads them back with tcgen05.ld, divides by the column norm ||Z_i|| (accumulated by the
+//   generator threads as a by-product) and appends every (column, residual) pair whose score
+//   |<Z_i, R_n>| / ||Z_i|| reaches the residual's threshold tau_n to that residual's report list.
+//
+// Nothing of size d is written: the output is the short report lists.  The pass serves two purposes of the
+// speculative OMP (see sgc_recover.cu): it verifies that no column outside the candidate set beats a
+// speculated pick, and it harvests new candidates.
+//
+// One persistent CTA per SM; warp roles: 0 = TMA producer, 1 = MMA issuer (owns the tensor-memory
+// allocation), 2-5 = epilogue (one per 32-lane quadrant of tensor memory), 6-21 = generators.
+// Every wait on an mbarrier is bounded (two seconds); on expiry the CTA records an error, leaves all loops,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "sgc_internal.cuh"
+
+namespace sgc {
+namespace {
+
+constexpr int kGenWarps = 16;                                // 512 generator threads: two per column of a sweep
+constexpr int kFirstGenWarp = 6;                             // warps 2..5 are the epilogue
+constexpr int kPassThreads = 32 * (kFirstGenWarp + kGenWarps);   // 704
+constexpr int kTileCols = 128;                               // UMMA M: columns of A per accumulator tile
+constexpr int kSuperCols = 2 * kTileCols;                    // columns of A per sweep over k
+constexpr int kChunkRows = 64;                               // rows of A per pipeline stage (128 B of bf16)
+constexpr int kTileBytes = kTileCols * kChunkRows * 2;       // 16384
+constexpr int kNormRing = 8;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct PassArgs {
+    uint32_t seed_lo, seed_hi;
+    unsigned long long d;
+    int k, n;                    // n: residuals per pass (multiple of 32, <= 256)
+    int stages, bufs;            // pipeline depth; accumulator buffers in tensor memory (2 when n <= 128)
+    unsigned int num_super;      // ceil(d / 256)
+    const float* tau;            // [n] thresholds (+inf = unused residual)
+    unsigned int* rep_count;     // [n]
+    uint2* rep;                  // [n][rep_cap]  (column, score bits)
+    int rep_cap;
+    const int* gate;             // optional: the kernel returns at once when *gate == 0
+    int* error;                  // set to 1 when a wait expired
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// bounded wait: false when the limit expired or another thread of the CTA already gave up
+__device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const unsigned long long t = global_ns();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    uint64_t desc = (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    desc |= (uint64_t)1 << 16;                 // leading byte offset (unused with swizzled K-major): 16 B
+    desc |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
+    desc |= (uint64_t)1 << 46;                 // descriptor version of sm_100
+    desc |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return desc;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// ---- the kernel -----------------------------------------------------------------------------------------
+// dynamic shared memory (after alignment to 1024 bytes):
+//   stages x { A tile 0 (16 KB) | A tile 1 (16 KB) | R^T chunk (n x 128 B) }
+//   norms  float[kNormRing][256][2]      partial ||Z_i||^2 of the two generator threads of each column
+//   tau    float[256]
+//   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
+__global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
+    if (a.gate != nullptr && *a.gate == 0) return;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const int stage_bytes = 2 * kTileBytes + a.n * 128;
+    const uint32_t norms_off = (uint32_t)a.stages * stage_bytes;
+    float* norms = reinterpret_cast<float*>(gen_base + norms_off);
+    float* tau_s = norms + kNormRing * kSuperCols * 2;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tau_s + 256);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * a.stages;
+    const uint32_t bar_accf = bar_empty + 8u * a.stages, bar_acce = bar_accf + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kc_count = a.k / kChunkRows;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < a.stages; ++s) {
+            mbar_init(bar_full + 8u * s, kGenWarps + 1);
+            mbar_init(bar_empty + 8u * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_accf + 8u * b, 1);
+            mbar_init(bar_acce + 8u * b, 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    for (int i = threadIdx.x; i < 256; i += kPassThreads) tau_s[i] = i < a.n ? a.tau[i] : __int_as_float(0x7f800000);
+    if (warp == 1) {           // tensor memory: all 512 columns (the only CTA on this SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int acc_cols = 2 * a.n;              // tensor-memory columns of one accumulator buffer (two tiles)
+
+    if (warp == 0) {
+        // ---------------- TMA producer: one chunk of R^T per stage -----------------------------------------
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x) {
+                for (int kc = 0; kc < kc_count; ++kc, ++it) {
+                    const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
+                    if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u);
+                    tma_load_2d(base + st * stage_bytes + 2 * kTileBytes, &tmap, kc * kChunkRows, 0, bar_full + 8u * st);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(a.n);
+            uint32_t it = 0, sweep_i = 0;
+            bool ok = true;
+            for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
+                const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
+                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                for (int kc = 0; kc < kc_count; ++kc, ++it) {
+                    const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
+                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + st * stage_bytes;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+#pragma unroll
+                        for (int kk = 0; kk < kChunkRows / 16; ++kk) {
+                            umma_bf16(tmem_base + buf * acc_cols + t * a.n, umma_desc(sa + t * kTileBytes + kk * 32),
+                                      umma_desc(sa + 2 * kTileBytes + kk * 32), idesc, (kc | kk) != 0 ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(bar_empty + 8u * st);        // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(bar_accf + 8u * buf);    // accumulators of this sweep complete
+            }
+        }
+    } else if (warp < kFirstGenWarp) {
+        // ---------------- epilogue: scores against thresholds ----------------------------------------------
+        const int quad = warp & 3;
+        uint32_t sweep_i = 0;
+        bool ok = true;
+        for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
+            const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag))) { ok = false; break; }
+            tc_fence_after();
+            const float* nr = norms + (size_t)(sweep_i % kNormRing) * kSuperCols * 2;
+#pragma unroll 1
+            for (int t = 0; t < 2; ++t) {
+                const int col_local = t * kTileCols + quad * 32 + lane;
+                const unsigned long long col = (unsigned long long)sweep * kSuperCols + col_local;
+                const float n2 = nr[col_local * 2] + nr[col_local * 2 + 1];
+                const float inv = (col < a.d && n2 > 0.0f) ? 1.0f / sqrtf(n2) : 0.0f;
+#pragma unroll 1
+                for (int c0 = 0; c0 < a.n; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * acc_cols + t * a.n + c0, v);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float sc = fabsf(__uint_as_float(v[i])) * inv;
+                        if (sc >= tau_s[c0 + i] && inv > 0.0f) {
+                            const unsigned int slot = atomicAdd(&a.rep_count[c0 + i], 1u);
+                            if (slot < (unsigned int)a.rep_cap)
+                                a.rep[(size_t)(c0 + i) * a.rep_cap + slot] = make_uint2((uint32_t)col, __float_as_uint(sc));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+        }
+    } else {
+        // ---------------- generators: Z tiles as bfloat16, swizzled K-major --------------------------------
+        const int g = threadIdx.x - kFirstGenWarp * 32;
+        const int col_local = g & (kSuperCols - 1), half = g >> 8;
+        const int tile = col_local >> 7, m = col_local & (kTileCols - 1);
+        const uint32_t row_off = (uint32_t)tile * kTileBytes + (uint32_t)m * 128u;
+        const uint32_t sw = (uint32_t)(m & 7);
+        uint32_t it = 0, sweep_i = 0;
+        bool ok = true;
+        for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
+            const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)((unsigned long long)sweep * kSuperCols + col_local));
+            float norm = 0.0f;
+            for (int kc = 0; kc < kc_count; ++kc, ++it) {
+                const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag))) { ok = false; break; }
+                uint32_t h = key.ck + (uint32_t)(kc * kChunkRows + half * 32) * key.mk;
+                const uint32_t dst = base + st * stage_bytes + row_off;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float z0 = z_from_word(h); h += key.mk;
+                        const float z1 = z_from_word(h); h += key.mk;
+                        norm = __fmaf_rn(z0, z0, norm);
+                        norm = __fmaf_rn(z1, z1, norm);
+                        w[e] = __byte_perm(__float_as_uint(z0), __float_as_uint(z1), 0x7632);
+                    }
+                    st_shared_v4(dst + ((((uint32_t)(half * 4 + c)) ^ sw) << 4), w[0], w[1], w[2], w[3]);
+                }
+                if (kc == kc_count - 1) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_full + 8u * st);
+            }
+        }
+    }
+    // ---------------- tail: everyone meets, tensor memory is returned ---------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0) atomicExch(a.error, 1);
+        // give copies and MMAs still in flight time to land before shared and tensor memory are released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// ---- host side --------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+std::mutex g_encode_mutex;
+EncodeTiledFn g_encode = nullptr;
+
+cudaError_t get_encoder(EncodeTiledFn* out) {
+    std::lock_guard<std::mutex> lock(g_encode_mutex);
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *out = g_encode;
+    return cudaSuccess;
+}
+
+size_t pass_smem_bytes(int n, int stages) {
+    return 1024 + (size_t)stages * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 256) +
+           8 * (2 * (size_t)stages + 4) + 16;
+}
+
+}  // namespace
+
+int pass_stages(int n) { return n <= 128 ? 4 : 3; }
+
+cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
+    EncodeTiledFn enc = nullptr;
+    cudaError_t e = get_encoder(&enc);
+    if (e != cudaSuccess) return e;
+    const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)n};
+    const cuuint64_t gstride[1] = {(cuuint64_t)k * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kChunkRows, (cuuint32_t)n};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(static_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(rt), gdim,
+                           gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t pass_configure(int n) {
+    static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map storage");
+    return cudaFuncSetAttribute(k_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+}
+
+cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, unsigned int* rep_count,
+                        uint2* rep, int rep_cap, const int* gate, int* error, int sm_count, cudaStream_t stream) {
+    PassArgs a;
+    a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
+    a.d = d; a.k = k; a.n = n;
+    a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;
+    a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
+    a.tau = tau; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
+    unsigned int grid = (unsigned int)sm_count;
+    if (grid > a.num_super) grid = a.num_super;
+    CUtensorMap map;
+    memcpy(&map, tmap, sizeof(map));
+    k_pass<<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    return cudaGetLastError();
+}
+
+}  // namespace sgc

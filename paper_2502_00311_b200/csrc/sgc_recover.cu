@@ -1,21 +1,53 @@
 // a4 + a5: x^M = OMP_A(M^), x^V = OMP_A(V^) (Eq. 7; Appendix B Algorithm 3), then
 // N = alpha x^M / (sqrt(x^V) + eps) and W <- W - lr N (Eq. 8, Eq. 3; Algorithm 2 line 6).
 //
-// Both recoveries advance in lock-step, one iteration per pair of launches:
-//   k_corr   the "Projection" + "Select" lines of Algorithm 3 without the d x d Gram matrix (Appendix B allows
-//            the memory-efficient form): every column of A is regenerated tile by tile and correlated with
-//            BOTH residuals, scores <A_i, r>^2 / ||A_i||^2 are reduced to the best few per block (fp32 screen);
-//   k_book   one block per residual: rescoring of the screened candidates in fp64 (the argmax decision),
-//            then the inverse-Cholesky recurrences of Algorithm 3 (c = F^T g, gamma, new column of F,
-//            a_j, x = F a) in fp64 and the residual r = y - A_Lambda x.
-// k_scatter applies Eq. (8) on the common support and updates W.
+// Algorithm 3 needs, for every pick, the argmax of |<A_i, r>| / ||A_i|| over all d columns ("Projection" and
+// "Select"), and A is regenerated rather than stored, so one such argmax costs k*d generated entries.  Two ways
+// of getting the picks are implemented; both produce exactly the picks of Algorithm 3.
+//
+// Lock-step (k_omp, mode 1): one pass over all columns per pick, both residuals (M^ and V^) against every
+//   generated entry; fp32 screen, fp64 decision among the near-maximal candidates, then the inverse-Cholesky
+//   recurrences of Algorithm 3 (c = F^T g, gamma, new column of F, a_j, x = F a) in fp64 and r = y - A_Lambda x.
+//
+// Speculative (rounds of k_omp mode 0, the tensor-core screening pass, k_resolve): OMP first runs on a short
+//   candidate list only (the supports of the previous step plus harvested columns), which costs next to
+//   nothing, and records the residual before every pick.  ONE pass over all d columns then correlates A with
+//   all those residuals at once (sgc_pass.cu) and reports every column whose score comes within the rounding
+//   margin of the speculated pick's.  k_resolve walks the picks in order: a pick without a challenger, or one
+//   that wins the fp64 rescoring against its challengers, is the true argmax; at the first pick that loses,
+//   the global winner (known from the same pass) is forced, the columns reported for that residual join the
+//   candidate list and the next round continues from there.  Every round fixes at least one more pick; what is
+//   still open after kMaxRounds rounds, or after any overflow, is finished in lock-step.
+//
+// Both modes run inside one cooperative kernel: all blocks correlate (phase A), grid barrier, blocks 0 and 1
+// keep the books of M^ and V^ (phase B), grid barrier.  k_scatter applies Eq. (8) on the common support.
+#include <cooperative_groups.h>
+
 #include "sgc_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace sgc {
 namespace {
 
+struct OmpArgs {
+    uint32_t seed_lo, seed_hi;
+    unsigned long long d;
+    int k, s;
+    unsigned int num_tiles;            // lock-step tiles of kOmpThreads * kCorrCols columns
+    double sigma;
+    int half_n;                        // residuals per stream in one screening pass
+    double z_harvest, z_floor;         // screening thresholds in units of ||r|| / sqrt(k)
+    Cand* corr_cand;                   // [2][grid][kCorrTop]
+    const double* y64; double* r64; float* r32;      // r32 viewed as float[2k] (interleaved pairs)
+    uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
+    Counters* cnt; SpecCtl* ctl;
+    uint16_t* rt; float* tau; unsigned int* rep_count; double* pick_score;
+    const uint32_t* cand_list;
+};
+
 // ------------------------------------------------------------------------------------------------
-// correlation pass
+// small helpers
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ bool better(float sa, uint32_t ia, float sb, uint32_t ib) {
     return (sa > sb) || (sa == sb && ia < ib);
@@ -23,8 +55,9 @@ __device__ __forceinline__ bool better(float sa, uint32_t ia, float sb, uint32_t
 
 struct Top2 {
     float s1, s2; uint32_t i1, i2;
-    __device__ __forceinline__ void init() { s1 = s2 = -1.0f; i1 = i2 = 0xFFFFFFFFu; }
+    __device__ __forceinline__ void init() { s1 = s2 = -1.0f; i1 = i2 = kNoColumn; }
     __device__ __forceinline__ void push(float s, uint32_t i) {
+        if (i == i1 || i == i2) return;
         if (better(s, i, s1, i1)) { s2 = s1; i2 = i1; s1 = s; i1 = i; }
         else if (better(s, i, s2, i2)) { s2 = s; i2 = i; }
     }
@@ -34,41 +67,148 @@ __device__ __forceinline__ void warp_merge(Top2& t) {
     for (int o = 16; o > 0; o >>= 1) {
         const float a1 = __shfl_xor_sync(0xffffffffu, t.s1, o), a2 = __shfl_xor_sync(0xffffffffu, t.s2, o);
         const uint32_t j1 = __shfl_xor_sync(0xffffffffu, t.i1, o), j2 = __shfl_xor_sync(0xffffffffu, t.i2, o);
-        t.push(a1, j1);
-        t.push(a2, j2);
+        if (j1 != kNoColumn) t.push(a1, j1);
+        if (j2 != kNoColumn) t.push(a2, j2);
     }
 }
 
-template <int C>
-__global__ void __launch_bounds__(kCorrThreads, 2)
-k_corr(uint32_t seed_lo, uint32_t seed_hi, unsigned long long d, int k, int s, const float2* __restrict__ r32,
-       const uint32_t* __restrict__ lam, const Counters* __restrict__ cnt, Cand* __restrict__ out,
-       unsigned int num_tiles) {
-    extern __shared__ float2 sr[];                       // residual pair per row
-    __shared__ uint32_t mask_idx[2][kMaxS];
-    __shared__ int mask_n[2];
-    __shared__ Top2 wtop[2][kCorrThreads / 32];
-    for (int j = threadIdx.x; j < k; j += kCorrThreads) sr[j] = r32[j];
-    const int done0 = cnt->done[0], done1 = cnt->done[1];
+__device__ __forceinline__ double warp_sum(double v) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// deterministic block sum (kOmpThreads threads); every thread receives the result.  red: 32 doubles.
+__device__ double block_sum(double v, double* red) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = (lane < kOmpThreads / 32) ? red[lane] : 0.0;
+    t = warp_sum(t);
+    return t;
+}
+
+__device__ __forceinline__ uint16_t bf16_rn_bits(float f) {          // round to nearest even (finite input)
+    const uint32_t b = __float_as_uint(f);
+    return (uint16_t)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+}
+
+// shared memory of the bookkeeping code (blocks 0 and 1 of k_omp, the only block of k_resolve)
+struct BookSmem {
+    double red[32];
+    float fred[32];
+    double gvec[kMaxS];               // Gram column g
+    double cvec[kMaxS];               // c = F^T g
+    double xs[kMaxS];                 // current coefficients
+    double best_dot, best_n2, best_score;
+    double cur_rnorm;                 // ||r|| of the residual the next pick is made from
+    uint32_t best_idx;
+    uint32_t cand_idx[kRescoreCap];
+    int n_cand;
+    int hi, extra, dep;               // speculation record of this block's stream
+    unsigned int smax_bits;
+};
+
+// exact score of one column against a residual: dot = <Z_i, r>, n2 = ||Z_i||^2 (fp64), for every thread
+__device__ void rescore_column(const OmpArgs& a, BookSmem& sh, uint32_t idx, const double* r, double* dot_out, double* n2_out) {
+    const ColKey key = column_key(a.seed_lo, a.seed_hi, idx);
+    double dot = 0.0, n2 = 0.0;
+    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) {
+        const double z = (double)z_from_word(key.ck + (uint32_t)row * key.mk);
+        dot += z * r[row];
+        n2 += z * z;
+    }
+    *dot_out = block_sum(dot, sh.red);
+    *n2_out = block_sum(n2, sh.red);
+}
+
+// fp64 argmax of |<A_i, r>| / ||A_i|| among sh.cand_idx[0..nc), lowest index on ties -> sh.best_*
+__device__ void rescore_candidates(const OmpArgs& a, BookSmem& sh, int nc, const double* r) {
+    if (threadIdx.x == 0) { sh.best_score = -1.0; sh.best_idx = kNoColumn; sh.best_dot = 0.0; sh.best_n2 = 1.0; }
+    __syncthreads();
+    for (int c = 0; c < nc; ++c) {
+        const uint32_t idx = sh.cand_idx[c];
+        double dot, n2;
+        rescore_column(a, sh, idx, r, &dot, &n2);
+        if (threadIdx.x == 0) {
+            const double sc = n2 > 0.0 ? dot * dot / n2 : 0.0;
+            if (sc > sh.best_score || (sc == sh.best_score && idx < sh.best_idx)) {
+                sh.best_score = sc; sh.best_idx = idx; sh.best_dot = dot; sh.best_n2 = n2;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// x = F a and r = y - A_Lambda x for the first v picks (F, a and the stored columns are prefixes of their
+// final values, so any earlier state can be rebuilt); r goes to r_out, x to sh.xs (and x_out when given).
+// Returns ||r||.
+__device__ double rebuild_prefix(const OmpArgs& a, BookSmem& sh, int m, int v, double* r_out, float* r32_out, double* x_out) {
+    const int k = a.k, s = a.s;
+    const double* y = a.y64 + (size_t)m * k;
+    const uint16_t* zs = a.zsel + (size_t)m * s * k;
+    const double* F = a.F + (size_t)m * s * s;
+    const double* ac = a.acoef + (size_t)m * s;
+    __syncthreads();
+    if ((int)threadIdx.x < v) {
+        const int i = threadIdx.x;
+        double acc = 0.0;
+        for (int l = i; l < v; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
+        sh.xs[i] = acc;
+        if (x_out) x_out[i] = acc;
+    }
+    __syncthreads();
+    double rn2 = 0.0;
+    for (int row = threadIdx.x; row < k; row += kOmpThreads) {
+        double acc = 0.0;
+        for (int l = 0; l < v; ++l) acc += sh.xs[l] * (double)bf16_bits_to_float(zs[(size_t)l * k + row]);
+        const double rv = y[row] - a.sigma * acc;
+        r_out[row] = rv;
+        if (r32_out) r32_out[2 * row + m] = (float)rv;
+        rn2 += rv * rv;
+    }
+    rn2 = block_sum(rn2, sh.red);
+    return sqrt(rn2);
+}
+
+__device__ void write_rt_row(const OmpArgs& a, int m, int c, const double* r) {
+    uint16_t* dst = a.rt + ((size_t)m * a.half_n + c) * a.k;
+    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) dst[row] = bf16_rn_bits((float)r[row]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// phase A, lock-step: every column of A against both residuals (thread = kCorrCols columns x all rows)
+// ------------------------------------------------------------------------------------------------
+__device__ void corr_all_columns(const OmpArgs& a, float2* sr, uint32_t (*mask_idx)[kMaxS], int* mask_n, Top2 (*wtop)[32],
+                                 const int* picks) {
+    const int k = a.k, s = a.s;
+    const float2* r32 = reinterpret_cast<const float2*>(a.r32);
+    __syncthreads();
+    for (int j = threadIdx.x; j < k; j += kOmpThreads) sr[j] = r32[j];
     Top2 best[2];
     best[0].init(); best[1].init();
-    constexpr unsigned int kTileCols = kCorrThreads * C;
-    for (unsigned int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+    constexpr unsigned int kTileCols = kOmpThreads * kCorrCols;
+    for (unsigned int tile = blockIdx.x; tile < a.num_tiles; tile += gridDim.x) {
         const unsigned long long col_base = (unsigned long long)tile * kTileCols;
         __syncthreads();
         if (threadIdx.x < 2) mask_n[threadIdx.x] = 0;
         __syncthreads();
         // already selected columns that fall into this tile are excluded from the argmax
-        for (int e = threadIdx.x; e < done0 + done1; e += kCorrThreads) {
-            const int m = e < done0 ? 0 : 1;
-            const uint32_t l = lam[m * s + (m ? e - done0 : e)];
+        for (int e = threadIdx.x; e < picks[0] + picks[1]; e += kOmpThreads) {
+            const int m = e < picks[0] ? 0 : 1;
+            const uint32_t l = a.lam[m * s + (m ? e - picks[0] : e)];
             if (l >= col_base && l < col_base + kTileCols) mask_idx[m][atomicAdd(&mask_n[m], 1)] = l;
         }
-        uint32_t h[C], mk[C];
-        float am[C], av[C], an[C];
+        uint32_t h[kCorrCols], mk[kCorrCols];
+        float am[kCorrCols], av[kCorrCols], an[kCorrCols];
 #pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const ColKey key = column_key(seed_lo, seed_hi, (uint32_t)(col_base + c * kCorrThreads + threadIdx.x));
+        for (int c = 0; c < kCorrCols; ++c) {
+            const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)(col_base + c * kOmpThreads + threadIdx.x));
             h[c] = key.ck; mk[c] = key.mk;
             am[c] = av[c] = an[c] = 0.0f;
         }
@@ -77,7 +217,7 @@ k_corr(uint32_t seed_lo, uint32_t seed_hi, unsigned long long d, int k, int s, c
         for (int row = 0; row < k; ++row) {
             const float2 rr = sr[row];
 #pragma unroll
-            for (int c = 0; c < C; ++c) {
+            for (int c = 0; c < kCorrCols; ++c) {
                 const float z = z_from_word(h[c]);
                 h[c] += mk[c];
                 am[c] = __fmaf_rn(z, rr.x, am[c]);
@@ -86,30 +226,28 @@ k_corr(uint32_t seed_lo, uint32_t seed_hi, unsigned long long d, int k, int s, c
             }
         }
 #pragma unroll
-        for (int c = 0; c < C; ++c) {
-            const unsigned long long col = col_base + c * kCorrThreads + threadIdx.x;
-            if (col >= d) continue;
+        for (int c = 0; c < kCorrCols; ++c) {
+            const unsigned long long col = col_base + c * kOmpThreads + threadIdx.x;
+            if (col >= a.d) continue;
             const float inv = an[c] > 0.0f ? 1.0f / an[c] : 0.0f;
             float sm = am[c] * am[c] * inv, sv = av[c] * av[c] * inv;
             for (int e = 0; e < mask_n[0]; ++e) if (mask_idx[0][e] == (uint32_t)col) sm = -1.0f;
             for (int e = 0; e < mask_n[1]; ++e) if (mask_idx[1][e] == (uint32_t)col) sv = -1.0f;
-            best[0].push(sm, (uint32_t)col);
-            best[1].push(sv, (uint32_t)col);
+            if (sm >= 0.0f) best[0].push(sm, (uint32_t)col);
+            if (sv >= 0.0f) best[1].push(sv, (uint32_t)col);
         }
     }
-    // block reduction of the two running top-2 lists
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     warp_merge(best[0]);
     warp_merge(best[1]);
+    __syncthreads();
     if (lane == 0) { wtop[0][warp] = best[0]; wtop[1][warp] = best[1]; }
     __syncthreads();
     if (warp < 2) {
-        Top2 t;
-        t.init();
-        if (lane < kCorrThreads / 32) t = wtop[warp][lane];
+        Top2 t = wtop[warp][lane];
         warp_merge(t);
         if (lane == 0) {
-            Cand* o = out + ((size_t)warp * gridDim.x + blockIdx.x) * kCorrTop;
+            Cand* o = a.corr_cand + ((size_t)warp * gridDim.x + blockIdx.x) * kCorrTop;
             o[0].score = t.s1; o[0].idx = t.i1;
             o[1].score = t.s2; o[1].idx = t.i2;
         }
@@ -117,113 +255,127 @@ k_corr(uint32_t seed_lo, uint32_t seed_hi, unsigned long long d, int k, int s, c
 }
 
 // ------------------------------------------------------------------------------------------------
-// bookkeeping: fp64 argmax among the screened candidates + Algorithm 3 recurrences
+// phase A, restricted: the candidate list against both residuals (warp = one column, lanes over rows)
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ double warp_sum(double v) {
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// deterministic block sum; every thread receives the result.  red: 32 doubles of shared memory.
-__device__ double block_sum(double v, double* red) {
+__device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], const int* picks) {
+    const int k = a.k, s = a.s;
+    const float2* r32 = reinterpret_cast<const float2*>(a.r32);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    v = warp_sum(v);
+    Top2 best[2];
+    best[0].init(); best[1].init();
+    const int stride = gridDim.x * (kOmpThreads / 32);
+    for (int e = warp * gridDim.x + blockIdx.x; e < n_cand; e += stride) {        // neighbours go to different blocks
+        const uint32_t col = a.cand_list[e];
+        bool t0 = false, t1 = false;
+        for (int q = lane; q < picks[0]; q += 32) t0 |= (a.lam[q] == col);
+        for (int q = lane; q < picks[1]; q += 32) t1 |= (a.lam[s + q] == col);
+        t0 = __any_sync(0xffffffffu, t0);
+        t1 = __any_sync(0xffffffffu, t1);
+        const ColKey key = column_key(a.seed_lo, a.seed_hi, col);
+        float dm = 0.0f, dv = 0.0f, n2 = 0.0f;
+        uint32_t h = key.ck + (uint32_t)lane * key.mk;
+        const uint32_t step = 32u * key.mk;
+        for (int row = lane; row < k; row += 32) {
+            const float z = z_from_word(h);
+            h += step;
+            const float2 rr = r32[row];
+            dm = __fmaf_rn(z, rr.x, dm);
+            dv = __fmaf_rn(z, rr.y, dv);
+            n2 = __fmaf_rn(z, z, n2);
+        }
+        dm = warp_sum(dm); dv = warp_sum(dv); n2 = warp_sum(n2);
+        const float inv = n2 > 0.0f ? 1.0f / n2 : 0.0f;
+        if (!t0) best[0].push(dm * dm * inv, col);
+        if (!t1) best[1].push(dv * dv * inv, col);
+    }
     __syncthreads();
-    if (lane == 0) red[warp] = v;
+    if (lane == 0) { wtop[0][warp] = best[0]; wtop[1][warp] = best[1]; }
     __syncthreads();
-    double t = (lane < kBookThreads / 32) ? red[lane] : 0.0;
-    t = warp_sum(t);
-    return t;
+    if (warp < 2) {
+        Top2 t = wtop[warp][lane];
+        warp_merge(t);
+        if (lane == 0) {
+            Cand* o = a.corr_cand + ((size_t)warp * gridDim.x + blockIdx.x) * kCorrTop;
+            o[0].score = t.s1; o[0].idx = t.i1;
+            o[1].score = t.s2; o[1].idx = t.i2;
+        }
+    }
 }
 
-struct BookArgs {
-    uint32_t seed_lo, seed_hi;
-    int k, s, corr_grid;
-    double sigma;
-    const Cand* corr_cand;
-    const double* y64; double* r64; float* r32;       // r32 viewed as float[2k] (interleaved pairs)
-    uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
-    Counters* cnt;
-};
-
-__global__ void __launch_bounds__(kBookThreads, 1)
-k_book(BookArgs a, int iter) {
-    const int m = blockIdx.x;                    // 0: M^, 1: V^
-    if (a.cnt->stopped[m]) return;
-    __shared__ double red[32];
-    __shared__ float fred[32];
-    __shared__ uint32_t cand_idx[kRescoreCap];
-    __shared__ int n_cand;
-    __shared__ double gvec[kMaxS];               // Gram column g, then reused
-    __shared__ double cvec[kMaxS];               // c = F^T g
-    __shared__ double xs[kMaxS];                 // current coefficients
-    __shared__ double best_dot, best_n2, best_score;
-    __shared__ uint32_t best_idx;
-    const int k = a.k, s = a.s, j = iter;
+// ------------------------------------------------------------------------------------------------
+// phase B: one pick of Algorithm 3 for residual m (whole block).  The pick is `forced` when given, otherwise
+// the fp64 argmax among the screened candidates of phase A.
+// Returns 0 = booked, 1 = no candidate left, 2 = the picked column is linearly dependent on the support.
+// spec_c >= 0: the pick is speculative and screened as residual spec_c of stream m (score and threshold are
+// recorded); spec_next >= 0: the new residual becomes row spec_next of the screened batch.
+// ------------------------------------------------------------------------------------------------
+__device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t forced, int spec_c, int spec_next,
+                         bool final_pick) {
+    const int k = a.k, s = a.s;
     const double* y = a.y64 + (size_t)m * k;
     double* r = a.r64 + (size_t)m * k;
     uint16_t* zs = a.zsel + (size_t)m * s * k;
     double* F = a.F + (size_t)m * s * s;
     double* xg = a.x + (size_t)m * s;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    // ---- 1. screened candidates: everything within 2e-3 (relative, squared scores) of the best fp32 score
-    const Cand* cc = a.corr_cand + (size_t)m * a.corr_grid * kCorrTop;
-    const int n_entries = a.corr_grid * kCorrTop;
-    float mx = -1.0f;
-    for (int e = threadIdx.x; e < n_entries; e += kBookThreads) mx = fmaxf(mx, cc[e].score);
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (threadIdx.x == 0) { n_cand = 0; best_score = -1.0; best_idx = 0xFFFFFFFFu; best_dot = 0.0; best_n2 = 1.0; }
+    int nc;
     __syncthreads();
-    if (lane == 0) fred[warp] = mx;
-    __syncthreads();
-    mx = fred[lane];
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    const float thr = mx - 2e-3f * fabsf(mx);
-    for (int e = threadIdx.x; e < n_entries; e += kBookThreads) {
-        const Cand c = cc[e];
-        if (c.idx != 0xFFFFFFFFu && c.score >= 0.0f && c.score >= thr) {
-            const int slot = atomicAdd(&n_cand, 1);
-            if (slot < kRescoreCap) cand_idx[slot] = c.idx;
+    if (forced != kNoColumn) {
+        if (threadIdx.x == 0) sh.cand_idx[0] = forced;
+        nc = 1;
+        __syncthreads();
+    } else {
+        // ---- 1. screened candidates: everything within 2e-3 (relative, squared scores) of the best fp32 score
+        const Cand* cc = a.corr_cand + (size_t)m * gridDim.x * kCorrTop;
+        const int n_entries = gridDim.x * kCorrTop;
+        float mx = -1.0f;
+        for (int e = threadIdx.x; e < n_entries; e += kOmpThreads) {
+            const Cand c = cc[e];
+            if (c.idx != kNoColumn) mx = fmaxf(mx, c.score);
         }
-    }
-    __syncthreads();
-    int nc = n_cand;
-    if (nc > kRescoreCap) {
-        if (threadIdx.x == 0) atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
-        nc = kRescoreCap;
-    }
-    if (nc == 0) {          // nothing left to select (cannot happen while fewer than d columns are taken)
-        if (threadIdx.x == 0) { a.cnt->stopped[m] = 1; atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN); }
-        return;
-    }
-    // ---- 2. fp64 rescoring: the argmax of |<A_i, r>| / ||A_i|| among the candidates, lowest index on ties
-    for (int c = 0; c < nc; ++c) {
-        const uint32_t idx = cand_idx[c];
-        const ColKey key = column_key(a.seed_lo, a.seed_hi, idx);
-        double dot = 0.0, n2 = 0.0;
-        for (int row = threadIdx.x; row < k; row += kBookThreads) {
-            const double z = (double)z_from_word(key.ck + (uint32_t)row * key.mk);
-            dot += z * r[row];
-            n2 += z * z;
-        }
-        dot = block_sum(dot, red);
-        n2 = block_sum(n2, red);
-        if (threadIdx.x == 0) {
-            const double sc = n2 > 0.0 ? dot * dot / n2 : 0.0;
-            if (sc > best_score || (sc == best_score && idx < best_idx)) {
-                best_score = sc; best_idx = idx; best_dot = dot; best_n2 = n2;
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if (threadIdx.x == 0) sh.n_cand = 0;
+        if (lane == 0) sh.fred[warp] = mx;
+        __syncthreads();
+        mx = sh.fred[lane];
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float thr = mx - 2e-3f * fabsf(mx);
+        for (int e = threadIdx.x; e < n_entries; e += kOmpThreads) {
+            const Cand c = cc[e];
+            if (c.idx != kNoColumn && c.score >= 0.0f && c.score >= thr) {
+                const int slot = atomicAdd(&sh.n_cand, 1);
+                if (slot < kRescoreCap) sh.cand_idx[slot] = c.idx;
             }
         }
         __syncthreads();
+        nc = sh.n_cand;
+        if (nc > kRescoreCap) {
+            if (threadIdx.x == 0) atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
+            nc = kRescoreCap;
+        }
+        if (nc == 0) return 1;
     }
-    const uint32_t lam_new = best_idx;
-    const double dot_r = best_dot, n2_new = best_n2;
+    // ---- 2. fp64 rescoring: the argmax of |<A_i, r>| / ||A_i|| among the candidates, lowest index on ties
+    rescore_candidates(a, sh, nc, r);
+    const uint32_t lam_new = sh.best_idx;
+    const double dot_r = sh.best_dot, n2_new = sh.best_n2;
+    if (spec_c >= 0) {
+        // what the screening pass must be able to refute: any column scoring above this pick, up to the margin
+        if (threadIdx.x == 0) {
+            const double ps = sqrt(sh.best_score), rn = sh.cur_rnorm, unit = rn / sqrt((double)k);
+            a.pick_score[(size_t)m * s + j] = ps;
+            double t = ps - kScreenMargin * rn;
+            if (t > a.z_harvest * unit) t = a.z_harvest * unit;
+            if (t < a.z_floor * unit) t = a.z_floor * unit;
+            a.tau[m * a.half_n + spec_c] = (float)t;
+            a.lam[(size_t)m * s + j] = lam_new;
+        }
+    }
     // ---- 3. store the new column (bfloat16 bits, exact) ------------------------------------------------
     {
         const ColKey key = column_key(a.seed_lo, a.seed_hi, lam_new);
         uint16_t* znew = zs + (size_t)j * k;
-        for (int row = threadIdx.x; row < k; row += kBookThreads)
+        for (int row = threadIdx.x; row < k; row += kOmpThreads)
             znew[row] = z_bf16_bits(z_from_word(key.ck + (uint32_t)row * key.mk));
     }
     __syncthreads();
@@ -231,71 +383,374 @@ k_book(BookArgs a, int iter) {
     const double sig2 = a.sigma * a.sigma;
     {
         const uint16_t* znew = zs + (size_t)j * k;
-        for (int l = warp; l < j; l += kBookThreads / 32) {
+        for (int l = warp; l < j; l += kOmpThreads / 32) {
             const uint16_t* zl = zs + (size_t)l * k;
             double acc = 0.0;
             for (int row = lane; row < k; row += 32)
                 acc += (double)(bf16_bits_to_float(zl[row]) * bf16_bits_to_float(znew[row]));   // product exact in fp32
             acc = warp_sum(acc);
-            if (lane == 0) gvec[l] = sig2 * acc;
+            if (lane == 0) sh.gvec[l] = sig2 * acc;
         }
     }
     __syncthreads();
     // ---- 5. c = F^T g ;  F is upper triangular, F(l,i) stored at F[l*s + i] ----------------------------
     double csq = 0.0;
-    if (threadIdx.x < j) {
+    if ((int)threadIdx.x < j) {
         const int i = threadIdx.x;
         double acc = 0.0;
-        for (int l = 0; l <= i; ++l) acc += F[(size_t)l * s + i] * gvec[l];
-        cvec[i] = acc;
+        for (int l = 0; l <= i; ++l) acc += F[(size_t)l * s + i] * sh.gvec[l];
+        sh.cvec[i] = acc;
         csq = acc * acc;
     }
-    csq = block_sum(csq, red);
+    csq = block_sum(csq, sh.red);
     // ---- 6. gamma = 1/sqrt(g_ll - c^T c); a dependent column stops this recovery --------------------------
     const double gnn = sig2 * n2_new;
     const double piv = gnn - csq;
-    if (!(piv > 1e-10 * gnn)) {
-        if (threadIdx.x == 0) { a.cnt->stopped[m] = 1; atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN); }
-        return;
-    }
+    if (!(piv > 1e-10 * gnn)) return 2;
     const double gamma = 1.0 / sqrt(piv);
     // ---- 7. new column of F: [-gamma F c ; gamma] ------------------------------------------------------
     __syncthreads();
-    if (threadIdx.x < j) {
+    if ((int)threadIdx.x < j) {
         const int i = threadIdx.x;
         double acc = 0.0;
-        for (int l = i; l < j; ++l) acc += F[(size_t)i * s + l] * cvec[l];
+        for (int l = i; l < j; ++l) acc += F[(size_t)i * s + l] * sh.cvec[l];
         F[(size_t)i * s + j] = -gamma * acc;
-    } else if (threadIdx.x == j) {
+    } else if ((int)threadIdx.x == j) {
         F[(size_t)j * s + j] = gamma;
     }
     // ---- 8. a_j = gamma <a_new, r> ;  x = F a  grows by a_j * F(:, j) -------------------------------------
     const double aj = gamma * a.sigma * dot_r;
     __syncthreads();
-    if (threadIdx.x <= j) {
+    if ((int)threadIdx.x <= j) {
         const int i = threadIdx.x;
         const double xo = (i < j) ? xg[i] : 0.0;
         const double xn = xo + aj * F[(size_t)i * s + j];
         xg[i] = xn;
-        xs[i] = xn;
+        sh.xs[i] = xn;
     }
     if (threadIdx.x == 0) { a.acoef[(size_t)m * s + j] = aj; a.lam[(size_t)m * s + j] = lam_new; }
     __syncthreads();
     // ---- 9. r = y - A_Lambda x ---------------------------------------------------------------------------
     double rn2 = 0.0;
-    for (int row = threadIdx.x; row < k; row += kBookThreads) {
+    uint16_t* rt_row = spec_next >= 0 ? a.rt + ((size_t)m * a.half_n + spec_next) * k : nullptr;
+    for (int row = threadIdx.x; row < k; row += kOmpThreads) {
         double acc = 0.0;
-        for (int l = 0; l <= j; ++l) acc += xs[l] * (double)bf16_bits_to_float(zs[(size_t)l * k + row]);
+        for (int l = 0; l <= j; ++l) acc += sh.xs[l] * (double)bf16_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r[row] = rv;
         a.r32[2 * row + m] = (float)rv;
+        if (rt_row) rt_row[row] = bf16_rn_bits((float)rv);
         rn2 += rv * rv;
     }
-    rn2 = block_sum(rn2, red);
+    rn2 = block_sum(rn2, sh.red);
     if (threadIdx.x == 0) {
         a.rnorm[(size_t)m * s + j] = sqrt(rn2);
-        a.cnt->done[m] = j + 1;
+        sh.cur_rnorm = sqrt(rn2);
+        if (final_pick) { a.cnt->done[m] = j + 1; a.ctl->v[m] = j + 1; }
     }
+    __syncthreads();
+    return 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+// the cooperative OMP kernel.  mode 0: speculate on the candidate list; mode 1: lock-step over all columns.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
+    cg::grid_group grid = cg::this_grid();
+    extern __shared__ float2 sr[];                       // residual pair per row (lock-step only)
+    __shared__ BookSmem sh;
+    __shared__ uint32_t mask_idx[2][kMaxS];
+    __shared__ int mask_n[2];
+    __shared__ Top2 wtop[2][32];
+    volatile SpecCtl* ctl = a.ctl;
+    // ---- gate: identical in every block, because nothing below changes the control block before the first barrier
+    const int fin[2] = {ctl->finished[0], ctl->finished[1]};
+    if (mode == 0) { if (!ctl->round_active || ctl->fallback) return; }
+    else { if (fin[0] && fin[1]) return; }
+    const int v0[2] = {ctl->v[0], ctl->v[1]};
+    const uint32_t forced0[2] = {ctl->forced[0], ctl->forced[1]};
+    const int n_cand = ctl->n_cand;
+    const int base[2] = {v0[0] + (forced0[0] != kNoColumn ? 1 : 0), v0[1] + (forced0[1] != kNoColumn ? 1 : 0)};
+    grid.sync();
+    const int mb = blockIdx.x;                           // blocks 0 and 1 keep the books of M^ and V^
+    if (mb < 2) {
+        if (!fin[mb]) {
+            // state after the verified picks (a failed speculation left later values behind)
+            const double rn = rebuild_prefix(a, sh, mb, v0[mb], a.r64 + (size_t)mb * a.k, a.r32, a.x + (size_t)mb * a.s);
+            if (threadIdx.x == 0) {
+                sh.cur_rnorm = rn;
+                if (v0[mb] == 0) a.ctl->ynorm[mb] = rn;
+                sh.hi = base[mb]; sh.extra = 0; sh.dep = 0;
+                a.ctl->stop[mb] = 0;
+            }
+            if (mode == 0 && forced0[mb] == kNoColumn) write_rt_row(a, mb, 0, a.r64 + (size_t)mb * a.k);
+        } else if (threadIdx.x == 0) {
+            a.ctl->stop[mb] = 1;
+        }
+        if (mode == 0) {
+            for (int c = threadIdx.x; c < a.half_n; c += kOmpThreads) {
+                a.rep_count[mb * a.half_n + c] = 0u;
+                a.tau[mb * a.half_n + c] = __int_as_float(0x7f800000);
+            }
+        }
+    }
+    grid.sync();
+    for (int i = 0;; ++i) {
+        int jm[2], picks[2];
+        bool act[2], need_corr = false;
+        for (int m = 0; m < 2; ++m) {
+            jm[m] = v0[m] + i;
+            act[m] = !fin[m] && jm[m] < a.s && !ctl->stop[m];
+            if (mode == 0 && jm[m] - base[m] >= a.half_n) act[m] = false;
+            picks[m] = jm[m] < a.s ? jm[m] : a.s;
+            if (act[m] && !(i == 0 && forced0[m] != kNoColumn)) need_corr = true;
+        }
+        if (!act[0] && !act[1]) break;
+        if (need_corr) {
+            if (mode == 0) corr_candidates(a, n_cand, wtop, picks);
+            else corr_all_columns(a, sr, mask_idx, mask_n, wtop, picks);
+        }
+        grid.sync();
+        if (mb < 2 && act[mb]) {
+            const int m = mb, j = jm[m];
+            const uint32_t forced = (i == 0) ? forced0[m] : kNoColumn;
+            const bool speculative = (mode == 0) && forced == kNoColumn;
+            const int c = j - base[m];                            // -1 for a forced pick
+            const int next = (mode == 0 && c + 1 < a.half_n && j + 1 < a.s) ? c + 1 : -1;
+            const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative);
+            if (threadIdx.x == 0) {
+                if (rc == 0) {
+                    sh.hi = j + 1;
+                } else if (speculative) {
+                    // no candidate left: the current residual is screened without a pick; dependent column: the
+                    // pick is screened, and the recovery stops there if the pick is confirmed
+                    if (rc == 1) {
+                        sh.extra = 1;
+                        a.tau[m * a.half_n + c] = (float)(a.z_harvest * sh.cur_rnorm / sqrt((double)a.k));
+                    } else { sh.dep = 1; sh.hi = j + 1; }
+                    a.ctl->stop[m] = 1;
+                } else {
+                    // a confirmed pick cannot be made: this recovery ends with j picks
+                    a.cnt->stopped[m] = 1;
+                    atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN);
+                    a.cnt->done[m] = j;
+                    a.ctl->v[m] = j;
+                    a.ctl->finished[m] = 1;
+                    a.ctl->stop[m] = 1;
+                    sh.hi = base[m] > j ? j : sh.hi;
+                }
+            }
+        }
+        grid.sync();
+    }
+    if (mb < 2 && threadIdx.x == 0 && !fin[mb]) {
+        if (mode == 0) {
+            a.ctl->base[mb] = base[mb];
+            a.ctl->hi[mb] = sh.hi < base[mb] ? base[mb] : sh.hi;
+            a.ctl->extra[mb] = sh.extra;
+            a.ctl->dep[mb] = sh.dep;
+        } else if (!a.ctl->finished[mb]) {
+            a.cnt->done[mb] = a.ctl->v[mb];
+            a.ctl->finished[mb] = 1;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// resolve: confirm or refute the speculated picks with the reports of the screening pass
+// ------------------------------------------------------------------------------------------------
+struct ResolveArgs {
+    OmpArgs o;
+    const uint2* rep; int rep_cap;
+    unsigned int* cand_bits; uint32_t* cand_list; double* rtmp;
+};
+
+__device__ __forceinline__ bool in_support(const uint32_t* lam, int n, uint32_t col) {
+    for (int q = 0; q < n; ++q) if (lam[q] == col) return true;
+    return false;
+}
+
+// Collects into sh.cand_idx[start..] the reported columns of one residual that are not in the first n_sup picks,
+// differ from `skip`, and score within `window` of the best such report, provided that best reaches `floor_sc`.
+// Returns the number of candidates (start included), or -1 on overflow.
+__device__ int collect_challengers(BookSmem& sh, const uint2* rep, unsigned int count, const uint32_t* lam, int n_sup,
+                                   uint32_t skip, float floor_sc, float window, int start) {
+    __syncthreads();
+    if (threadIdx.x == 0) { sh.smax_bits = 0u; sh.n_cand = start; }
+    __syncthreads();
+    for (unsigned int e = threadIdx.x; e < count; e += kOmpThreads) {
+        const uint2 rp = rep[e];
+        const float sc = __uint_as_float(rp.y);
+        if (sc >= floor_sc && rp.x != skip && !in_support(lam, n_sup, rp.x)) atomicMax(&sh.smax_bits, rp.y);   // scores are >= 0
+    }
+    __syncthreads();
+    const unsigned int smax_bits = sh.smax_bits;
+    if (smax_bits == 0u) return start;
+    const float lo = __uint_as_float(smax_bits) - window;
+    for (unsigned int e = threadIdx.x; e < count; e += kOmpThreads) {
+        const uint2 rp = rep[e];
+        const float sc = __uint_as_float(rp.y);
+        if (sc >= floor_sc && sc >= lo && rp.x != skip && !in_support(lam, n_sup, rp.x)) {
+            const int slot = atomicAdd(&sh.n_cand, 1);
+            if (slot < kRescoreCap) sh.cand_idx[slot] = rp.x;
+        }
+    }
+    __syncthreads();
+    const int n = sh.n_cand;
+    return n > kRescoreCap ? -1 : n;
+}
+
+// the reported columns of one residual join the candidate list (the forced winner first)
+__device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, unsigned int count, uint32_t first) {
+    volatile SpecCtl* ctl = ra.o.ctl;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        sh.n_cand = ctl->n_cand;
+        if (first != kNoColumn && sh.n_cand < kCandCap) {
+            const unsigned int bit = 1u << (first & 31u);
+            if (!(atomicOr(&ra.cand_bits[first >> 5], bit) & bit)) ra.cand_list[sh.n_cand++] = first;
+        }
+    }
+    __syncthreads();
+    for (unsigned int e = threadIdx.x; e < count; e += kOmpThreads) {
+        const uint32_t col = rep[e].x;
+        const unsigned int bit = 1u << (col & 31u);
+        if (atomicOr(&ra.cand_bits[col >> 5], bit) & bit) continue;
+        const int slot = atomicAdd(&sh.n_cand, 1);
+        if (slot < kCandCap) ra.cand_list[slot] = col;
+        else atomicAnd(&ra.cand_bits[col >> 5], ~bit);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ctl->n_cand = sh.n_cand < kCandCap ? sh.n_cand : kCandCap;
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
+    const OmpArgs& a = ra.o;
+    __shared__ BookSmem sh;
+    __shared__ int give_up;
+    volatile SpecCtl* ctl = a.ctl;
+    if (!ctl->round_active) return;
+    if (ctl->fallback || ctl->pass_error) {
+        if (threadIdx.x == 0) { ctl->fallback = 1; ctl->round_active = 0; }
+        return;
+    }
+    if (threadIdx.x == 0) { give_up = 0; ctl->rounds = ctl->rounds + 1; }
+    __syncthreads();
+    const int s = a.s;
+    for (int m = 0; m < 2; ++m) {
+        if (ctl->finished[m]) continue;
+        const int base = ctl->base[m], hi = ctl->hi[m], extra = ctl->extra[m], dep = ctl->dep[m];
+        const uint32_t* lam = a.lam + (size_t)m * s;
+        int v = base;
+        uint32_t forced = kNoColumn;
+        bool failed = false, bad = false;
+        for (int j = base; j < hi && !failed && !bad; ++j) {
+            const int n = m * a.half_n + (j - base);
+            const unsigned int count = a.rep_count[n];
+            if (count > (unsigned int)ra.rep_cap) { bad = true; break; }
+            const uint32_t pick = lam[j];
+            const double ps = a.pick_score[(size_t)m * s + j];
+            const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
+            const float margin = (float)(kScreenMargin * rn);
+            if (threadIdx.x == 0) sh.cand_idx[0] = pick;
+            const int nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, j, pick, (float)ps - margin,
+                                               2.0f * margin, 1);
+            if (nc < 0) { bad = true; break; }
+            if (nc == 1) { v = j + 1; continue; }                 // nobody comes close: the pick is the argmax
+            rebuild_prefix(a, sh, m, j, ra.rtmp, nullptr, nullptr);
+            rescore_candidates(a, sh, nc, ra.rtmp);
+            if (sh.best_idx == pick) { v = j + 1; continue; }
+            forced = sh.best_idx; v = j; failed = true;
+            harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
+        }
+        if (!failed && !bad) {
+            if (dep) {
+                // the dependent pick was the true argmax: Algorithm 3 cannot extend the support, this recovery ends
+                v = hi - 1;
+                if (threadIdx.x == 0) {
+                    a.cnt->stopped[m] = 1; a.cnt->done[m] = v; ctl->finished[m] = 1;
+                    atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN);
+                }
+            } else if (hi >= s) {
+                v = s;
+                if (threadIdx.x == 0) { a.cnt->done[m] = s; ctl->finished[m] = 1; }
+            } else if (extra) {
+                // residual screened without a pick: its best reported column is the next pick
+                const int n = m * a.half_n + (hi - base);
+                const unsigned int count = a.rep_count[n];
+                const double rn = hi == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + hi - 1];
+                const float margin = (float)(kScreenMargin * rn);
+                int nc = -1;
+                if (count >= 1u && count <= (unsigned int)ra.rep_cap)
+                    nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, hi, kNoColumn, 0.0f, 2.0f * margin, 0);
+                if (nc <= 0) bad = true;
+                else {
+                    rebuild_prefix(a, sh, m, hi, ra.rtmp, nullptr, nullptr);
+                    rescore_candidates(a, sh, nc, ra.rtmp);
+                    forced = sh.best_idx; v = hi;
+                    harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
+                }
+            } else {
+                v = hi;                                           // the pass had no room for more residuals
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ctl->v[m] = v;
+            ctl->forced[m] = forced;
+            if (bad) give_up = 1;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (give_up) {
+            ctl->fallback = 1; ctl->round_active = 0;
+            atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
+        } else if (ctl->finished[0] && ctl->finished[1]) {
+            ctl->round_active = 0;
+        }
+    }
+}
+
+// start of the recovery of one step
+__global__ void k_spec_init(SpecCtl* ctl, int speculate) {
+    if (threadIdx.x == 0) {
+        ctl->round_active = speculate; ctl->fallback = speculate ? 0 : 1;
+        ctl->v[0] = ctl->v[1] = 0;
+        ctl->forced[0] = ctl->forced[1] = kNoColumn;
+        ctl->finished[0] = ctl->finished[1] = 0;
+        ctl->stop[0] = ctl->stop[1] = 0;
+        ctl->rounds = 0; ctl->pass_error = 0;
+    }
+}
+
+// end of the step: the supports found stay (or become) candidates of the next step
+__global__ void __launch_bounds__(kOmpThreads, 1)
+k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uint32_t* cand_list, unsigned int* cand_bits) {
+    __shared__ int n_s;
+    int n = ctl->n_cand;
+    if (n > kCandKeep) {
+        for (int e = threadIdx.x; e < n; e += kOmpThreads) {
+            const uint32_t col = cand_list[e];
+            atomicAnd(&cand_bits[col >> 5], ~(1u << (col & 31u)));
+        }
+        n = 0;
+    }
+    if (threadIdx.x == 0) n_s = n;
+    __syncthreads();
+    for (int e = threadIdx.x; e < 2 * s; e += kOmpThreads) {
+        const int m = e / s, j = e % s;
+        if (j >= cnt->done[m]) continue;
+        const uint32_t col = lam[e];
+        const unsigned int bit = 1u << (col & 31u);
+        if (atomicOr(&cand_bits[col >> 5], bit) & bit) continue;
+        const int slot = atomicAdd(&n_s, 1);
+        if (slot < kCandCap) cand_list[slot] = col;
+        else atomicAnd(&cand_bits[col >> 5], ~bit);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ctl->n_cand = n_s < kCandCap ? n_s : kCandCap;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -351,51 +806,128 @@ k_scatter(int s, uint32_t* lam, double* x, Counters* __restrict__ cnt, float* __
     }
 }
 
+// z with d * P(|N(0,1)| > z) = target (bisection on erfc)
+double normal_tail_threshold(double d, double target) {
+    double p = target / d;
+    if (p > 0.5) p = 0.5;
+    double lo = 0.0, hi = 12.0;
+    for (int i = 0; i < 80; ++i) {
+        const double mid = 0.5 * (lo + hi);
+        if (erfc(mid / sqrt(2.0)) > p) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+OmpArgs make_args(const sgc_state* st) {
+    OmpArgs a;
+    a.seed_lo = (uint32_t)(st->seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(st->seed >> 32);
+    a.d = (unsigned long long)st->d; a.k = st->k; a.s = st->s;
+    const unsigned long long tile_cols = (unsigned long long)kOmpThreads * kCorrCols;
+    a.num_tiles = (unsigned int)(((unsigned long long)st->d + tile_cols - 1) / tile_cols);
+    a.sigma = (double)(float)(1.0 / sqrt((double)st->k));
+    a.half_n = st->pass_n / 2;
+    a.z_harvest = st->z_harvest; a.z_floor = st->z_floor;
+    a.corr_cand = st->corr_cand; a.y64 = st->y64; a.r64 = st->r64; a.r32 = reinterpret_cast<float*>(st->r32);
+    a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
+    a.cnt = st->cnt; a.ctl = st->ctl;
+    a.rt = st->rt; a.tau = st->tau; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
+    a.cand_list = st->cand_list;
+    return a;
+}
+
+cudaError_t launch_omp(sgc_state* st, const OmpArgs& a, int mode, cudaStream_t stream) {
+    OmpArgs args = a;
+    int m = mode;
+    void* params[2] = {&args, &m};
+    return cudaLaunchCooperativeKernel((const void*)k_omp, dim3((unsigned int)st->corr_grid), dim3(kOmpThreads), params,
+                                       (size_t)st->corr_smem, stream);
+}
+
 }  // namespace
 
 cudaError_t configure_recover(sgc_state* st) {
     const size_t smem = (size_t)st->k * sizeof(float2);
-    cudaError_t e = cudaFuncSetAttribute(k_corr<kCorrCols>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_corr<kCorrCols>, kCorrThreads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_omp, kOmpThreads, smem);
     if (e != cudaSuccess) return e;
     if (occ < 1) return cudaErrorInvalidConfiguration;
-    const unsigned long long tile_cols = (unsigned long long)kCorrThreads * kCorrCols;
-    const unsigned long long tiles = ((unsigned long long)st->d + tile_cols - 1) / tile_cols;
-    unsigned long long grid = (unsigned long long)st->sm_count * occ;
-    if (grid > tiles) grid = tiles;
-    st->corr_grid = (int)grid;
+    int coop = 0;
+    e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, st->device);
+    if (e != cudaSuccess) return e;
+    if (!coop) return cudaErrorNotSupported;
+    st->corr_grid = st->sm_count * occ;                  // every block resident: required by the grid barrier
+    if (st->corr_grid < 2) return cudaErrorInvalidConfiguration;
     st->corr_smem = (int)smem;
+    // speculative recovery: needs whole 64-row chunks of A for the tensor-core pass
+    st->spec_ok = (st->k % 64 == 0);
+    int half = st->s < 128 ? st->s : 128;
+    half = (half + 15) / 16 * 16;
+    st->pass_n = 2 * half;
+    st->z_harvest = normal_tail_threshold((double)st->d, 256.0);
+    st->z_floor = normal_tail_threshold((double)st->d, 1024.0);
+    if (st->spec_ok) {
+        e = pass_configure(st->pass_n);
+        if (e != cudaSuccess) return e;
+    }
     return cudaSuccess;
 }
 
+cudaError_t finish_recover_setup(sgc_state* st) {
+    if (!st->spec_ok) return cudaSuccess;
+    return pass_encode_map(st->tmap, st->rt, st->pass_n, st->k);
+}
+
 cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches) {
-    const uint32_t seed_lo = (uint32_t)(st->seed & 0xFFFFFFFFu), seed_hi = (uint32_t)(st->seed >> 32);
-    const unsigned long long tile_cols = (unsigned long long)kCorrThreads * kCorrCols;
-    const unsigned int tiles = (unsigned int)(((unsigned long long)st->d + tile_cols - 1) / tile_cols);
-    BookArgs a;
-    a.seed_lo = seed_lo; a.seed_hi = seed_hi; a.k = st->k; a.s = st->s; a.corr_grid = st->corr_grid;
-    a.sigma = (double)(float)(1.0 / sqrt((double)st->k));
-    a.corr_cand = st->corr_cand; a.y64 = st->y64; a.r64 = st->r64; a.r32 = reinterpret_cast<float*>(st->r32);
-    a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
-    a.cnt = st->cnt;
-    for (int it = 0; it < st->s; ++it) {
-        {
-            PhaseTimer timer(st, stream, kPhaseCorr, 1);
-            k_corr<kCorrCols><<<st->corr_grid, kCorrThreads, st->corr_smem, stream>>>(
-                seed_lo, seed_hi, (unsigned long long)st->d, st->k, st->s, st->r32, st->lam, st->cnt, st->corr_cand, tiles);
-        }
-        {
-            PhaseTimer timer(st, stream, kPhaseBook, 1);
-            k_book<<<2, kBookThreads, 0, stream>>>(a, it);
-        }
-        *launches += 2;
+    const OmpArgs a = make_args(st);
+    const bool speculate = st->spec_ok && (st->mode == 2 || (st->mode == 0 && st->d >= (1ll << 16)));
+    cudaError_t e = cudaSuccess;
+    {
+        PhaseTimer timer(st, stream, kPhaseBook, 1);
+        k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0);
+        *launches += 1;
     }
-    PhaseTimer timer(st, stream, kPhaseScatter, 1);
-    k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weight, st->upd_idx, st->upd_val,
-                                              (double)st->alpha, (double)st->eps, (double)st->lr);
-    *launches += 1;
+    if (speculate) {
+        ResolveArgs ra;
+        ra.o = a; ra.rep = st->rep; ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list;
+        ra.rtmp = st->rtmp;
+        for (int round = 0; round < kMaxRounds && e == cudaSuccess; ++round) {
+            {
+                PhaseTimer timer(st, stream, kPhaseCorr, 1);
+                e = launch_omp(st, a, 0, stream);
+            }
+            if (e != cudaSuccess) break;
+            {
+                PhaseTimer timer(st, stream, kPhasePass, 1);
+                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->rep_count, st->rep, kRepCap,
+                                &st->ctl->round_active, &st->ctl->pass_error, st->sm_count, stream);
+            }
+            if (e != cudaSuccess) break;
+            {
+                PhaseTimer timer(st, stream, kPhaseBook, 1);
+                k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
+            }
+            *launches += 3;
+        }
+        if (e != cudaSuccess) return e;
+    }
+    {
+        PhaseTimer timer(st, stream, kPhaseCorr, 1);
+        e = launch_omp(st, a, 1, stream);
+        *launches += 1;
+    }
+    if (e != cudaSuccess) return e;
+    {
+        PhaseTimer timer(st, stream, kPhaseScatter, 1);
+        k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weight, st->upd_idx, st->upd_val,
+                                                  (double)st->alpha, (double)st->eps, (double)st->lr);
+        *launches += 1;
+        if (speculate) {
+            k_cand_update<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->cnt, st->lam, st->s, st->cand_list, st->cand_bits);
+            *launches += 1;
+        }
+    }
     return cudaGetLastError();
 }
 

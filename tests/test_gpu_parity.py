@@ -103,9 +103,12 @@ def test_select_flags_non_finite_input(sgc):
 
 
 # ---- whole step, config-1 shape and relatives -------------------------------------------------------------
-def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_support=False, compare_every=1):
+def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_support=False, compare_every=1, mode=None,
+             stats=None):
     hp = inputs.ADAM
     st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha)
+    if mode is not None:
+        st.set_mode(mode)
     ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha or 1.0)
     supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0))
     w0 = inputs.weights(d, 99)
@@ -120,6 +123,8 @@ def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_suppo
         st.step(cuda(g), w_gpu)
         ref.step(g, w_ref)
         assert st.get("t") == step == ref.get("t")
+        if stats is not None:
+            stats.append((int(st.get("rounds")), int(st.get("fallback")), int(st.get("n_cand"))))
         assert np.array_equal(st.get("sel_idx"), ref.get("sel_idx"))
         assert np.array_equal(st.get("sel_val"), ref.get("sel_val"))
         for name in ("p", "q", "M", "V"):
@@ -160,6 +165,49 @@ def test_config1_ten_steps(sgc):
 def test_awkward_shapes(sgc, d, k, s):
     # d not a multiple of 4 or of the tile, k not a multiple of 32, s = 1 and s = k/8
     run_both(sgc, d, k, s, 5, "student", 3, cfg_id=2)
+
+
+# ---- speculative recovery (candidate-list OMP confirmed by tensor-core screening passes) ---------------------
+@pytest.mark.parametrize("d,k,s,kind", [(4096, 256, 16, "gauss"), (1 << 17, 512, 64, "student"), (70_001, 320, 17, "student"),
+                                        (200_000, 128, 5, "student"), (50_000, 2048, 130, "student")])
+def test_speculative_recovery_matches_the_oracle(sgc, d, k, s, kind):
+    # same bar as the lock-step path: supports in selection order bit-exact, values within tolerance; the planted
+    # support is fixed, so after the first step the candidate list holds it and one screening pass per step suffices
+    stats = []
+    worst, status = run_both(sgc, d, k, s, 5, kind, 4, cfg_id=2, mode=2, stats=stats)
+    assert not status & sgc.STATUS_CANDIDATE_OVERFLOW
+    assert all(fb == 0 for _, fb, _ in stats), stats
+    assert all(r >= 1 for r, _, _ in stats), stats
+
+
+def test_speculative_recovery_with_redrawn_supports_and_alpha(sgc):
+    # every step is a cold start for the candidate list, and the recovery is inexact (picks among noise columns)
+    stats = []
+    run_both(sgc, 150_000, 256, 8, 11, "student", 5, cfg_id=2, alpha=2.0, redraw_support=True, mode=2, stats=stats)
+    assert all(fb == 0 for _, fb, _ in stats), stats
+
+
+def test_speculative_and_lockstep_agree_bit_for_bit_on_supports(sgc):
+    d, k, s = 300_000, 2048, 24          # k large enough for exact recovery: the picks are the planted support
+    hp = inputs.ADAM
+    supp, sign = inputs.planted_support(d, s, 77)
+    a = sgc.Sgc(d, k, s, 6, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    b = sgc.Sgc(d, k, s, 6, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    a.set_mode(sgc.MODE_LOCKSTEP)
+    b.set_mode(sgc.MODE_SPECULATIVE)
+    wa, wb = cuda(inputs.weights(d, 3)), cuda(inputs.weights(d, 3))
+    for step in range(1, 6):
+        g = cuda(inputs.gradient(d, "student", supp, sign, 900 + step))
+        a.step(g, wa)
+        b.step(g, wb)
+        assert a.get("fallback") == 1 and b.get("fallback") == 0
+        for name in ("lamM", "lamV", "upd_idx"):
+            assert np.array_equal(a.get(name), b.get(name)), (name, step)
+        assert rel(b.get("xM"), a.get("xM")) < 1e-9 and rel(b.get("xV"), a.get("xV")) < 1e-9
+        assert rel(wb.cpu().numpy(), wa.cpu().numpy()) < 1e-7
+    assert b.get("rounds") == 1          # warm candidate list: one confirming pass per step
+    a.close()
+    b.close()
 
 
 def test_alpha_and_redrawn_supports(sgc):
