@@ -194,12 +194,14 @@ SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0
  * the unscaled measurement matrix of (seed, k) and R_j row j of rt.  Runs on the tensor cores.
  *   d, k        1 <= d < 2^32; k a multiple of 64, 64 <= k <= 65536
  *   n           number of residuals, a multiple of 32, 32 <= n <= 256
- *   rt          device pointer, n x k bfloat16 bit patterns, row-major, 16-byte aligned, read only
+ *   rt          device pointer, n x k binary16 (IEEE half) bit patterns, row-major, 16-byte aligned, read only
  *   tau         device pointer, n floats (+infinity disables a residual)
  *   rep_count   device pointer, n uint32: number of reports per residual (may exceed rep_cap)
  *   rep         device pointer, n x rep_cap pairs (uint32 column, float score bits); the first
  *               min(rep_count[j], rep_cap) pairs of row j are valid, in no particular order
  *   error_flag  device pointer to one int32, set to 1 if the kernel gave up on an internal wait (results invalid)
+ * Scores carry a relative error of up to 1e-3 (the norm ||Z_i|| is accumulated in short binary16 partial sums), so a
+ * pair whose exact score lies within that distance of its threshold may or may not be reported.
  * Everything is enqueued on stream; the call does not synchronise. */
 SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uint16_t* rt, const float* tau, uint32_t* rep_count,
                        uint32_t* rep, int32_t rep_cap, int32_t* error_flag, void* stream);

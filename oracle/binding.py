@@ -40,6 +40,16 @@ def lib():
             L.orc_sigma.argtypes = [C.c_int32]
             L.orc_z_block.restype = None
             L.orc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, f32p]
+            L.orc_half_round.restype = C.c_uint16
+            L.orc_half_round.argtypes = [C.c_double]
+            L.orc_half_value.restype = C.c_double
+            L.orc_half_value.argtypes = [C.c_uint16]
+            L.orc_half_fma.restype = C.c_uint16
+            L.orc_half_fma.argtypes = [C.c_uint16, C.c_uint16, C.c_uint16]
+            L.orc_half_mul.restype = C.c_uint16
+            L.orc_half_mul.argtypes = [C.c_uint16, C.c_uint16]
+            L.orc_z_of_byte_sum.restype = C.c_uint16
+            L.orc_z_of_byte_sum.argtypes = [C.c_int32]
             L.orc_sparsify.restype = C.c_int32
             L.orc_sparsify.argtypes = [f32p, C.c_int64, C.c_int32, u32p, f32p]
             L.orc_project.restype = None

@@ -19,7 +19,7 @@
 //   * Bias correction (Algorithm 2 lines 4-5) produces temporaries; M and V are stored uncorrected.
 //   * A has i.i.d. entries of standard deviation 1/sqrt(k) (Section 3.3).  Here
 //     A[j][i] = sigma_k * Z(seed, j, i) with sigma_k = fl32(1/sqrt(k)) and Z a counter-based
-//     approximately standard-normal value defined below; A is never stored.
+//     approximately standard-normal value (a binary16 number) defined below; A is never stored.
 //   * Ties in |g| and in the OMP argmax go to the lower index; selected columns are not re-selected.
 //   * Exactly s OMP iterations unless the new column is numerically dependent on the support.
 //   * Eq. (8) is applied on the intersection of the two supports where x^V > 0; elsewhere N = 0.
@@ -45,24 +45,27 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------
-// Z(seed, row, col): the measurement-matrix entry before scaling.
+// Z(seed, row, col): the measurement-matrix entry before scaling.  The paper fixes only the law of
+// A (i.i.d. zero-mean normal entries of standard deviation 1/sqrt(k), Section 3.3); this is the
+// concrete, counter-based realisation of it.  Every value of Z is exactly a binary16 (half) number.
 //
 //  1. column keys  ck = mix32( mix32(col + 0x9E3779B9 * seed_lo) ^ seed_hi )     (offset)
-//                  mk = mix32( ck ^ 0x5BD1E995 ) | 1                               (odd row stride)
-//  2. entry word   h  = ck + row * mk ; h ^= h>>16 ; h *= 0x85EBCA6B ; h ^= h>>15
-//  3. byte sum     S  = b0 + b1 + b2 + b3 of h           (0..1020, Irwin-Hall of order 4)
-//  4. centred      x  = S - 510                           (exact small integer in fp32)
-//  5. quantile map z  = x * ( C0 + w*(C1 + w*C2) ), w = x*x, evaluated in fp32 with two fused
-//                        multiply-adds (Horner) and one rounded multiply
-//  6. truncate z to its upper 16 bits (a bfloat16 value held in an fp32)
+//                  mk = mix32( ck ^ 0x5BD1E995 ) | 1                               (odd stride)
+//  2. pair word    one 32-bit word serves the two rows 2p and 2p+1 of a column:
+//                  h = ck + p * mk ; h ^= h>>16 ; h *= 0x85EBCA6B ; h ^= h>>15
+//  3. byte sums    S = b0 + b1 of h for the even row, b2 + b3 for the odd row   (0..510, triangular law)
+//  4. centred      x = (S - 255) / 256                      (exact in binary16)
+//  5. quantile map w = x*x ; q = fma(fma(w, C2, C1), w, C0) ; Z = x*q , every operation rounded to
+//                  binary16 (round to nearest even, subnormals kept) -- the arithmetic of the GPU's
+//                  packed half-precision instructions, restated here through exact double products
 //
-// Both column keys pass through a full-avalanche finaliser once per column; the per-entry mixing
-// (step 2) is deliberately short because it runs k*d times per correlation pass on the GPU.  The
-// per-column odd stride mk makes two columns share their entry sequence only if both 32-bit keys
+// The odd polynomial maps the quantiles of the triangular law onto those of the standard normal;
+// C0..C2 were chosen once (variance 1.0000, kurtosis 2.999, Kolmogorov distance 3.5e-3 to the
+// normal over the 511 lattice points, |Z| <= 3.37, Z monotone in S) and are frozen as bit patterns.
+// Both column keys pass through a full-avalanche finaliser once per column; the per-word mixing
+// (step 2) is deliberately short because it runs k*d/2 times per correlation pass on the GPU.  The
+// per-column odd stride mk makes two columns share their word sequence only if both 32-bit keys
 // are related, which does not happen among d < 2^32 columns in expectation.
-// The odd polynomial of step 5 maps the quantiles of the byte-sum distribution onto those of the
-// standard normal; C0..C2 were fitted once (weighted least squares over the 1021 lattice points,
-// then rescaled so that E[Z^2] = 1 after truncation) and are frozen as bit patterns.
 // mix32 is the public-domain "lowbias32" integer finaliser.
 // ------------------------------------------------------------------------------------------
 inline uint32_t mix32(uint32_t x) {
@@ -75,26 +78,66 @@ inline uint32_t mix32(uint32_t x) {
 inline float bits_to_float(uint32_t b) { float f; std::memcpy(&f, &b, 4); return f; }
 inline uint32_t float_to_bits(float f) { uint32_t b; std::memcpy(&b, &f, 4); return b; }
 
+// ---- binary16 arithmetic, restated with doubles -----------------------------------------------
+// value of a binary16 bit pattern (finite patterns only)
+inline double half_value(uint16_t b) {
+    const int sign = b >> 15, e = (b >> 10) & 31, m = b & 1023;
+    const double mag = e == 0 ? std::ldexp((double)m, -24) : std::ldexp((double)(1024 + m), e - 25);
+    return sign ? -mag : mag;
+}
+// nearest binary16 (ties to even) of a double of magnitude below 65520; subnormals are kept
+inline uint16_t half_round(double v) {
+    const uint16_t sign = std::signbit(v) ? 0x8000 : 0;
+    const double a = std::fabs(v);
+    if (a == 0.0) return sign;
+    int e;
+    std::frexp(a, &e);                                  // a = f * 2^e, f in [0.5, 1)
+    int q = e - 11;                                     // spacing 2^q of binary16 numbers near a (11-bit significand)
+    if (q < -24) q = -24;                               // subnormal range: spacing 2^-24
+    const double scaled = std::ldexp(a, -q);            // exact
+    double r = std::nearbyint(scaled);                  // default rounding mode: to nearest, ties to even
+    // r in [0, 2048]; r == 2048 means the significand overflowed into the next binade
+    int64_t n = (int64_t)r;
+    if (n == 0) return sign;
+    int exp_field;
+    if (n >= 2048) { n >>= 1; q += 1; }
+    if (n >= 1024) exp_field = q + 25; else exp_field = 0;        // normal: value = n * 2^q with 1024 <= n < 2048
+    return (uint16_t)(sign | (exp_field << 10) | (n & 1023));
+}
+// products of two binary16 numbers are exact in double; the sum with a third is exact unless the product lies
+// more than 30 binary orders below it, where it cannot move the rounded result onto or off a tie
+inline uint16_t half_mul(uint16_t a, uint16_t b) { return half_round(half_value(a) * half_value(b)); }
+inline uint16_t half_fma(uint16_t a, uint16_t b, uint16_t c) { return half_round(half_value(a) * half_value(b) + half_value(c)); }
+
 inline uint32_t column_key(uint64_t seed, uint32_t col) {
     const uint32_t seed_lo = (uint32_t)(seed & 0xFFFFFFFFu);
     const uint32_t seed_hi = (uint32_t)(seed >> 32);
     return mix32(mix32(col + 0x9E3779B9U * seed_lo) ^ seed_hi);
 }
 
+// step 5 for one lattice point S in [0, 510]
+inline uint16_t z_of_byte_sum(int S) {
+    const uint16_t C0 = 0x40c2, C1 = 0xbad9, C2 = 0x3f89;
+    const uint16_t x = half_round((double)(S - 255) / 256.0);          // exact
+    const uint16_t w = half_mul(x, x);
+    uint16_t q = half_fma(w, C2, C1);
+    q = half_fma(q, w, C0);
+    return half_mul(x, q);
+}
+
+// Z takes one of 511 values; they are computed once from the definition above and looked up afterwards
+struct ZTable {
+    float z[511];
+    ZTable() { for (int S = 0; S <= 510; ++S) z[S] = (float)half_value(z_of_byte_sum(S)); }
+};
+inline const ZTable& z_table() { static const ZTable t; return t; }
+
 inline float z_from_key(uint32_t ck, uint32_t row) {
     const uint32_t mk = mix32(ck ^ 0x5BD1E995U) | 1U;
-    uint32_t h = ck + row * mk;
+    uint32_t h = ck + (row >> 1) * mk;
     h ^= h >> 16; h *= 0x85EBCA6BU; h ^= h >> 15;
-    const int S = (int)(h & 0xFF) + (int)((h >> 8) & 0xFF) + (int)((h >> 16) & 0xFF) + (int)(h >> 24);
-    const float x = (float)(S - 510);
-    const float w = x * x;                               // exact: |x| <= 510
-    const float C0 = bits_to_float(0x3bd72bb5U);
-    const float C1 = bits_to_float(0x30aad71cU);
-    const float C2 = bits_to_float(0x28f3f07fU);
-    float q = std::fmaf(w, C2, C1);
-    q = std::fmaf(q, w, C0);
-    const float z = x * q;
-    return bits_to_float(float_to_bits(z) & 0xFFFF0000U);
+    const int S = (row & 1U) ? (int)((h >> 16) & 0xFF) + (int)(h >> 24) : (int)(h & 0xFF) + (int)((h >> 8) & 0xFF);
+    return z_table().z[S];
 }
 
 inline float sigma_of_k(int32_t k) { return (float)(1.0 / std::sqrt((double)k)); }
@@ -153,6 +196,13 @@ extern "C" {
 float orc_sigma(int32_t k) { return sigma_of_k(k); }
 
 // out[r * ncols + c] = Z(seed, row0 + r, col0 + c)
+// the binary16 arithmetic of the generator, exported so that the tests can pin it
+uint16_t orc_half_round(double v) { return half_round(v); }
+double orc_half_value(uint16_t b) { return half_value(b); }
+uint16_t orc_half_fma(uint16_t a, uint16_t b, uint16_t c) { return half_fma(a, b, c); }
+uint16_t orc_half_mul(uint16_t a, uint16_t b) { return half_mul(a, b); }
+uint16_t orc_z_of_byte_sum(int32_t S) { return z_of_byte_sum(S); }
+
 void orc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out) {
     for (int64_t c = 0; c < ncols; ++c) {
         const uint32_t ck = column_key(seed, (uint32_t)(col0 + c));

@@ -130,8 +130,8 @@ def z_block(seed, row0, nrows, col0, ncols, stream=None):
 
 
 def screen(seed, d, k, rt, tau, rep_cap, stream=None):
-    """sgc_screen: tensor-core screening pass.  rt: CUDA int16/uint16-sized tensor [n, k] of bfloat16 bit patterns
-    (or a torch.bfloat16 tensor), tau: float32 CUDA tensor [n].  Returns (rep_count [n] int32, rep [n, rep_cap, 2] int32
+    """sgc_screen: tensor-core screening pass.  rt: CUDA int16/uint16-sized tensor [n, k] of binary16 bit patterns
+    (or a torch.float16 tensor), tau: float32 CUDA tensor [n].  Returns (rep_count [n] int32, rep [n, rep_cap, 2] int32
     holding (column, score bits), error_flag [1] int32) as CUDA tensors; nothing is synchronised."""
     import torch
     n = rt.shape[0]

@@ -46,6 +46,7 @@ size_t layout(sgc_state* st, unsigned char* base) {
         const size_t n = (size_t)st->pass_n;
         st->rt = carve<uint16_t>(base, off, n * k);
         st->tau = carve<float>(base, off, n);
+        st->inv_scale = carve<float>(base, off, n);
         st->rep_count = carve<unsigned int>(base, off, n);
         st->rep = carve<uint2>(base, off, n * sgc::kRepCap);
         st->pick_score = carve<double>(base, off, 2 * s);
@@ -286,8 +287,8 @@ SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uin
     if (e == cudaSuccess) e = cudaMemsetAsync(rep_count, 0, sizeof(uint32_t) * (size_t)n, cs);
     if (e == cudaSuccess) e = cudaMemsetAsync(error_flag, 0, sizeof(int32_t), cs);
     if (e == cudaSuccess)
-        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, rep_count, reinterpret_cast<uint2*>(rep), rep_cap, nullptr,
-                             error_flag, sms, cs);
+        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
+                             nullptr, error_flag, sms, cs);
     return (int)e;
 }
 

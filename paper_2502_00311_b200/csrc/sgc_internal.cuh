@@ -13,20 +13,22 @@ namespace sgc {
 
 // ------------------------------------------------------------------------------------------------
 // Measurement matrix: A[j][i] = sigma_k * Z(seed, j, i), never stored (Section 3.3 fixes only the law:
-// i.i.d. zero-mean normal entries of standard deviation 1/sqrt(k)).
+// i.i.d. zero-mean normal entries of standard deviation 1/sqrt(k)).  Every Z is exactly a binary16 number.
 //
-// Z(seed, row, col):
+// Z(seed, row, col); one 32-bit word yields the two rows 2p and 2p+1 of a column:
 //   ck = mix32(mix32(col + 0x9E3779B9*seed_lo) ^ seed_hi),  mk = mix32(ck ^ 0x5BD1E995) | 1
-//   h  = ck + row*mk;  h ^= h >> 16;  h *= 0x85EBCA6B;  h ^= h >> 15
-//   S  = sum of the four bytes of h;  x = S - 510;  w = x*x
-//   z  = x * fma(fma(w, C2, C1), w, C0)      (fp32, round to nearest)
-//   Z  = z with the low 16 bits cleared       (exactly a bfloat16)
-// The byte sum is an Irwin-Hall(4) variable; the odd polynomial maps its quantiles onto the normal's.
+//   h  = ck + p*mk;  h ^= h >> 16;  h *= 0x85EBCA6B;  h ^= h >> 15
+//   S  = b0 + b1 (even row) or b2 + b3 (odd row), bytes of h;   x = (S - 255)/256
+//   w  = x*x;  q = fma(fma(w, C2, C1), w, C0);  Z = x*q        (binary16, round to nearest even)
+// A byte pair sum is triangular on 511 lattice points; the odd polynomial maps its quantiles onto the normal's.
+// Both rows are evaluated at once with packed half-precision instructions (f16x2).
 // ------------------------------------------------------------------------------------------------
 constexpr uint32_t kGolden = 0x9E3779B9u;
 constexpr uint32_t kMulEntry = 0x85EBCA6Bu;
 constexpr uint32_t kStrideSalt = 0x5BD1E995u;
-constexpr uint32_t kC0 = 0x3bd72bb5u, kC1 = 0x30aad71cu, kC2 = 0x28f3f07fu;
+constexpr uint32_t kC0x2 = 0x40c240c2u, kC1x2 = 0xbad9bad9u, kC2x2 = 0x3f893f89u;   // C0, C1, C2 in both halves
+constexpr uint32_t kInv256x2 = 0x1c001c00u;          // 2^-8
+constexpr uint32_t kCentrex2 = 0xc4ffc4ffu;          // -(1024 + 255)/256
 
 __host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du;
@@ -44,22 +46,50 @@ __host__ __device__ __forceinline__ ColKey column_key(uint32_t seed_lo, uint32_t
     return c;
 }
 
-// h0 = ck + row*mk (the caller advances it by mk per row)
-__device__ __forceinline__ float z_from_word(uint32_t h0) {
-    uint32_t h = h0;
-    h ^= h >> 16; h *= kMulEntry; h ^= h >> 15;
-    // bytes summed straight into the mantissa of 2^23: the float 8388608 + S
-    const uint32_t sb = __dp4a(h, 0x01010101u, 0x4B000000u);
-    const float x = __uint_as_float(sb) - 8389118.0f;          // S - 510, exact
-    const float w = __fmul_rn(x, x);                           // exact (|x| <= 510)
-    float q = __fmaf_rn(w, __uint_as_float(kC2), __uint_as_float(kC1));
-    q = __fmaf_rn(q, w, __uint_as_float(kC0));
-    const float z = __fmul_rn(x, q);
-    return __uint_as_float(__float_as_uint(z) & 0xFFFF0000u);
+__device__ __forceinline__ uint32_t hfma2(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
 
-__device__ __forceinline__ uint16_t z_bf16_bits(float z) { return (uint16_t)(__float_as_uint(z) >> 16); }
-__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+// h0 = ck + p*mk (the caller advances it by mk per row pair).  Returns Z of rows 2p (low half) and 2p+1 (high
+// half) as two binary16 bit patterns.
+__device__ __forceinline__ uint32_t z_pair_from_word(uint32_t h0) {
+    uint32_t h = h0;
+    h ^= h >> 16; h *= kMulEntry; h ^= h >> 15;
+    // byte pair sums straight into the significand of the half 1024: the halves 1024 + S (exact, S <= 510)
+    const uint32_t e0 = __dp4a(h, 0x00000101u, 0x6400u);
+    const uint32_t e1 = __dp4a(h, 0x01010000u, 0x6400u);
+    const uint32_t s2 = __byte_perm(e0, e1, 0x5410);
+    const uint32_t x = hfma2(s2, kInv256x2, kCentrex2);        // (S - 255)/256, exact
+    const uint32_t w = hmul2(x, x);
+    uint32_t q = hfma2(w, kC2x2, kC1x2);
+    q = hfma2(q, w, kC0x2);
+    return hmul2(x, q);
+}
+
+__device__ __forceinline__ float half_bits_to_float(uint32_t b) {
+    float f;
+    asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.f32.f16 %0, t;\n\t}" : "=f"(f) : "r"(b));
+    return f;
+}
+__device__ __forceinline__ float2 half2_bits_to_float2(uint32_t b) {
+    float2 f;
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tcvt.f32.f16 %0, lo;\n\tcvt.f32.f16 %1, hi;\n\t}"
+        : "=f"(f.x), "=f"(f.y) : "r"(b));
+    return f;
+}
+// Z(row) of the column with key (ck, mk), as binary16 bits / as a float
+__device__ __forceinline__ uint32_t z_bits_at(const ColKey& key, uint32_t row) {
+    const uint32_t z2 = z_pair_from_word(key.ck + (row >> 1) * key.mk);
+    return (row & 1u) ? (z2 >> 16) : (z2 & 0xFFFFu);
+}
+__device__ __forceinline__ float z_at(const ColKey& key, uint32_t row) { return half_bits_to_float(z_bits_at(key, row)); }
 
 // ------------------------------------------------------------------------------------------------
 // limits
@@ -80,7 +110,11 @@ constexpr int kRepCap = 2048;           // report slots per residual of one scre
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
 constexpr int kMaxRounds = 8;           // speculate / screen / resolve rounds enqueued per step
 constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
-constexpr double kScreenMargin = 2.2e-3;  // bound on |score from bfloat16 residual - exact score| / ||r|| (2^-9 + slack)
+// |score computed by the screening pass - exact score| <= kScreenMargin * ||r|| + kScreenNormMargin * score:
+// the residual is rounded to binary16 (relative error 2^-11 per element, hence at most 2^-11 ||r|| by
+// Cauchy-Schwarz), and the pass accumulates the column norm in short binary16 partial sums (error ~1e-4 relative)
+constexpr double kScreenMargin = 5.5e-4;
+constexpr double kScreenNormMargin = 1.0e-3;
 constexpr uint32_t kNoColumn = 0xFFFFFFFFu;
 
 struct Cand { float score; uint32_t idx; };
@@ -141,15 +175,16 @@ struct sgc_state {
     float2* r32;                // [k] (M^ residual, V^ residual)
     unsigned long long* sel_cand; unsigned int* sel_hist;
     sgc::Cand* corr_cand;       // [2][corr_grid][kCorrTop]
-    uint16_t* zsel;             // [2][s][k] selected columns of Z as bfloat16 bits
+    uint16_t* zsel;             // [2][s][k] selected columns of Z as binary16 bits
     uint32_t* lam;              // [2][s]
     double *F, *acoef, *x, *gvec, *cvec, *rnorm;   // [2][s*s], [2][s] ...
     uint32_t* upd_idx; double* upd_val;
     sgc::Counters* cnt;
     // speculative recovery
     sgc::SpecCtl* ctl;
-    uint16_t* rt;               // R^T [pass_n][k] bfloat16 bits: the residuals screened by one pass
-    float* tau;                 // [pass_n] thresholds
+    uint16_t* rt;               // R^T [pass_n][k] binary16 bits: the residuals screened by one pass, each row scaled
+    float* tau;                 // [pass_n] thresholds (in the scaled units of the row)
+    float* inv_scale;           // [pass_n] 1 / (power-of-two scale of the row)
     unsigned int* rep_count;    // [pass_n]
     uint2* rep;                 // [pass_n][kRepCap] (column, score bits)
     double* pick_score;         // [2][s] exact score |<Z_i, r>| / ||Z_i|| of every speculative pick
@@ -196,6 +231,7 @@ cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: 
 int pass_stages(int n);
 cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
-cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, unsigned int* rep_count,
-                        uint2* rep, int rep_cap, const int* gate, int* error, int sm_count, cudaStream_t stream);
+cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
+                        unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error, int sm_count,
+                        cudaStream_t stream);
 }  // namespace sgc

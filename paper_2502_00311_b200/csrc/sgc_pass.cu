@@ -1,9 +1,10 @@
 // Screening pass of the recovery (a4): the "Projection" line of Algorithm 3, p = A^T r, for a whole batch of
 // residual vectors at once, as one dense contraction  C = A^T R  on the tcgen05 tensor cores.
 //
-//   A (k x d) is regenerated tile by tile by the CUDA cores straight into shared memory as bfloat16 (Z is
-//   exactly representable there), in the K-major 128-byte-swizzled layout the UMMA descriptors expect;
-//   R^T (N x k, bfloat16, one residual per row) arrives chunk by chunk through TMA;
+//   A (k x d) is regenerated tile by tile by the CUDA cores straight into shared memory as binary16 (every Z
+//   is a binary16 number; the generator's packed f16x2 arithmetic emits two rows per instruction), in the
+//   K-major 128-byte-swizzled layout the UMMA descriptors expect;
+//   R^T (N x k, binary16, one residual per row, each row scaled by a power of two) arrives chunk by chunk through TMA;
 //   accumulators live in tensor memory (fp32, 128 lanes = 128 columns of A, N columns each);
 //   the epilogue reads them back with tcgen05.ld, divides by the column norm ||Z_i|| (accumulated by the
 //   generator threads as a by-product) and appends every (column, residual) pair whose score
@@ -31,7 +32,7 @@ constexpr int kFirstGenWarp = 6;                             // warps 2..5 are t
 constexpr int kPassThreads = 32 * (kFirstGenWarp + kGenWarps);   // 704
 constexpr int kTileCols = 128;                               // UMMA M: columns of A per accumulator tile
 constexpr int kSuperCols = 2 * kTileCols;                    // columns of A per sweep over k
-constexpr int kChunkRows = 64;                               // rows of A per pipeline stage (128 B of bf16)
+constexpr int kChunkRows = 64;                               // rows of A per pipeline stage (128 B of binary16)
 constexpr int kTileBytes = kTileCols * kChunkRows * 2;       // 16384
 constexpr int kNormRing = 8;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -42,7 +43,8 @@ struct PassArgs {
     int k, n;                    // n: residuals per pass (multiple of 32, <= 256)
     int stages, bufs;            // pipeline depth; accumulator buffers in tensor memory (2 when n <= 128)
     unsigned int num_super;      // ceil(d / 256)
-    const float* tau;            // [n] thresholds (+inf = unused residual)
+    const float* tau;            // [n] thresholds (+inf = unused residual), in the units of the (scaled) rows of R^T
+    const float* inv_scale;      // [n] factor that turns a score back into the caller's units, or nullptr for 1
     unsigned int* rep_count;     // [n]
     uint2* rep;                  // [n][rep_cap]  (column, score bits)
     int rep_cap;
@@ -78,10 +80,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// bounded wait: false when the limit expired or another thread of the CTA already gave up
-__device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// bounded wait: false when the limit expired or another thread of the CTA already gave up.  sleep_ns > 0 backs
+// off between polls so that a waiting warp leaves the issue slots to the generator warps.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns) {
     unsigned long long t0 = 0;
     for (uint32_t i = 0;; ++i) {
+        if (sleep_ns) __nanosleep(sleep_ns);
         if (mbar_try(bar, parity)) return true;
         if ((i & 63u) == 63u) {
             if (*abort_flag) return false;
@@ -90,6 +94,10 @@ __device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_fla
             else if (t - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, sleep_ns);
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -111,11 +119,11 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     desc |= (uint64_t)2 << 61;                 // SWIZZLE_128B
     return desc;
 }
-// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+// instruction descriptor: f16 x f16 -> fp32 (operand formats 0), both operands K-major, M = 128, N = n
 __device__ __forceinline__ uint32_t umma_idesc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
@@ -126,15 +134,12 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -195,14 +200,14 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer: one chunk of R^T per stage -----------------------------------------
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t st = 0, ph = 0;
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x) {
-                for (int kc = 0; kc < kc_count; ++kc, ++it) {
-                    const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
-                    if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag)) { ok = false; break; }
+                for (int kc = 0; kc < kc_count; ++kc) {
+                    if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 256)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u);
                     tma_load_2d(base + st * stage_bytes + 2 * kTileBytes, &tmap, kc * kChunkRows, 0, bar_full + 8u * st);
+                    if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
                 }
             }
         }
@@ -210,26 +215,26 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         // ---------------- MMA issuer ----------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(a.n);
-            uint32_t it = 0, sweep_i = 0;
+            uint32_t st = 0, ph = 0, sweep_i = 0;
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
                 const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
-                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 64)) { ok = false; break; }
                 tc_fence_after();
-                for (int kc = 0; kc < kc_count; ++kc, ++it) {
-                    const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
-                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag)) { ok = false; break; }
+                for (int kc = 0; kc < kc_count; ++kc) {
+                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 32)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = base + st * stage_bytes;
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
 #pragma unroll
                         for (int kk = 0; kk < kChunkRows / 16; ++kk) {
-                            umma_bf16(tmem_base + buf * acc_cols + t * a.n, umma_desc(sa + t * kTileBytes + kk * 32),
+                            umma_f16(tmem_base + buf * acc_cols + t * a.n, umma_desc(sa + t * kTileBytes + kk * 32),
                                       umma_desc(sa + 2 * kTileBytes + kk * 32), idesc, (kc | kk) != 0 ? 1u : 0u);
                         }
                     }
                     umma_commit(bar_empty + 8u * st);        // frees the stage once these MMAs have read it
+                    if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(bar_accf + 8u * buf);    // accumulators of this sweep complete
             }
@@ -241,7 +246,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         bool ok = true;
         for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
             const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag))) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag, 512))) { ok = false; break; }
             tc_fence_after();
             const float* nr = norms + (size_t)(sweep_i % kNormRing) * kSuperCols * 2;
 #pragma unroll 1
@@ -251,16 +256,18 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                 const float n2 = nr[col_local * 2] + nr[col_local * 2 + 1];
                 const float inv = (col < a.d && n2 > 0.0f) ? 1.0f / sqrtf(n2) : 0.0f;
 #pragma unroll 1
-                for (int c0 = 0; c0 < a.n; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * acc_cols + t * a.n + c0, v);
+                for (int c0 = 0; c0 < a.n; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * acc_cols + t * a.n + c0, v);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
+                    for (int i = 0; i < 16; ++i) {
                         const float sc = fabsf(__uint_as_float(v[i])) * inv;
                         if (sc >= tau_s[c0 + i] && inv > 0.0f) {
                             const unsigned int slot = atomicAdd(&a.rep_count[c0 + i], 1u);
-                            if (slot < (unsigned int)a.rep_cap)
-                                a.rep[(size_t)(c0 + i) * a.rep_cap + slot] = make_uint2((uint32_t)col, __float_as_uint(sc));
+                            if (slot < (unsigned int)a.rep_cap) {
+                                const float out = a.inv_scale ? sc * a.inv_scale[c0 + i] : sc;
+                                a.rep[(size_t)(c0 + i) * a.rep_cap + slot] = make_uint2((uint32_t)col, __float_as_uint(out));
+                            }
                         }
                     }
                 }
@@ -270,39 +277,46 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
         }
     } else {
-        // ---------------- generators: Z tiles as bfloat16, swizzled K-major --------------------------------
+        // ---------------- generators: Z tiles as binary16, swizzled K-major ---------------------------------
         const int g = threadIdx.x - kFirstGenWarp * 32;
         const int col_local = g & (kSuperCols - 1), half = g >> 8;
         const int tile = col_local >> 7, m = col_local & (kTileCols - 1);
         const uint32_t row_off = (uint32_t)tile * kTileBytes + (uint32_t)m * 128u;
         const uint32_t sw = (uint32_t)(m & 7);
-        uint32_t it = 0, sweep_i = 0;
+        uint32_t off[4];                                     // swizzled positions of this thread's four 16-byte chunks
+#pragma unroll
+        for (int c = 0; c < 4; ++c) off[c] = row_off + ((((uint32_t)(half * 4 + c)) ^ sw) << 4);
+        uint32_t st = 0, ph = 0, sweep_i = 0;
         bool ok = true;
         for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
             const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)((unsigned long long)sweep * kSuperCols + col_local));
             float norm = 0.0f;
-            for (int kc = 0; kc < kc_count; ++kc, ++it) {
-                const uint32_t st = it % a.stages, ph = (it / a.stages) & 1u;
-                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag))) { ok = false; break; }
-                uint32_t h = key.ck + (uint32_t)(kc * kChunkRows + half * 32) * key.mk;
-                const uint32_t dst = base + st * stage_bytes + row_off;
+            uint32_t h = key.ck + (uint32_t)(half * 16) * key.mk;   // one word per row pair
+            const uint32_t skip = 16u * key.mk;                  // the other generator thread of this column owns the next 32 rows
+            for (int kc = 0; kc < kc_count; ++kc) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 0))) { ok = false; break; }
+                const uint32_t dst = base + st * stage_bytes;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t w[4];
+                for (int c = 0; c < 4; c += 2) {
+                    uint32_t w[8];
+                    uint32_t n2 = 0u;                            // ||.||^2 of 16 entries as two binary16 partial sums
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float z0 = z_from_word(h); h += key.mk;
-                        const float z1 = z_from_word(h); h += key.mk;
-                        norm = __fmaf_rn(z0, z0, norm);
-                        norm = __fmaf_rn(z1, z1, norm);
-                        w[e] = __byte_perm(__float_as_uint(z0), __float_as_uint(z1), 0x7632);
+                    for (int e = 0; e < 8; ++e) {
+                        w[e] = z_pair_from_word(h);
+                        h += key.mk;
+                        n2 = hfma2(w[e], w[e], n2);
                     }
-                    st_shared_v4(dst + ((((uint32_t)(half * 4 + c)) ^ sw) << 4), w[0], w[1], w[2], w[3]);
+                    st_shared_v4(dst + off[c], w[0], w[1], w[2], w[3]);
+                    st_shared_v4(dst + off[c + 1], w[4], w[5], w[6], w[7]);
+                    const float2 part = half2_bits_to_float2(n2);
+                    norm += part.x + part.y;
                 }
+                h += skip;
                 if (kc == kc_count - 1) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full + 8u * st);
+                if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
             }
         }
     }
@@ -361,7 +375,7 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
     const cuuint64_t gstride[1] = {(cuuint64_t)k * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kChunkRows, (cuuint32_t)n};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(static_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(rt), gdim,
+    const CUresult r = enc(static_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(rt), gdim,
                            gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -372,14 +386,15 @@ cudaError_t pass_configure(int n) {
     return cudaFuncSetAttribute(k_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
 }
 
-cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, unsigned int* rep_count,
-                        uint2* rep, int rep_cap, const int* gate, int* error, int sm_count, cudaStream_t stream) {
+cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
+                        unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error, int sm_count,
+                        cudaStream_t stream) {
     PassArgs a;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
     a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;
     a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
-    a.tau = tau; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
+    a.tau = tau; a.inv_scale = inv_scale; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
     unsigned int grid = (unsigned int)sm_count;
     if (grid > a.num_super) grid = a.num_super;
     CUtensorMap map;

@@ -31,7 +31,7 @@ k_project_adam(uint32_t seed_lo, uint32_t seed_hi, int k, int s, const uint32_t*
     if (row >= k) return;
     double accp = 0.0, accq = 0.0;
     for (int i = 0; i < s; ++i) {
-        const double a = sigma * (double)z_from_word(keys[i].ck + (uint32_t)row * keys[i].mk);
+        const double a = sigma * (double)z_at(keys[i], (uint32_t)row);
         const double g = (double)vals[i];
         accp = accp + a * g;
         accq = accq + a * (g * g);
@@ -54,7 +54,7 @@ __global__ void k_z_block(uint32_t seed_lo, uint32_t seed_hi, long long row0, lo
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
         const long long r = e / ncols, c = e % ncols;
         const ColKey key = column_key(seed_lo, seed_hi, (uint32_t)(col0 + c));
-        out[e] = z_from_word(key.ck + (uint32_t)(row0 + r) * key.mk);
+        out[e] = z_at(key, (uint32_t)(row0 + r));
     }
 }
 

@@ -22,6 +22,7 @@
 // Both modes run inside one cooperative kernel: all blocks correlate (phase A), grid barrier, blocks 0 and 1
 // keep the books of M^ and V^ (phase B), grid barrier.  k_scatter applies Eq. (8) on the common support.
 #include <cooperative_groups.h>
+#include <cuda_fp16.h>
 
 #include "sgc_internal.cuh"
 
@@ -42,7 +43,7 @@ struct OmpArgs {
     const double* y64; double* r64; float* r32;      // r32 viewed as float[2k] (interleaved pairs)
     uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
     Counters* cnt; SpecCtl* ctl;
-    uint16_t* rt; float* tau; unsigned int* rep_count; double* pick_score;
+    uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; double* pick_score;
     const uint32_t* cand_list;
 };
 
@@ -93,9 +94,18 @@ __device__ double block_sum(double v, double* red) {
     return t;
 }
 
-__device__ __forceinline__ uint16_t bf16_rn_bits(float f) {          // round to nearest even (finite input)
-    const uint32_t b = __float_as_uint(f);
-    return (uint16_t)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+__device__ __forceinline__ uint16_t half_rn_bits(double v) { return __half_as_ushort(__double2half(v)); }   // nearest even
+
+// bound on |score seen by the screening pass - exact score| for a residual of norm rn and a score near ps
+__device__ __forceinline__ double screen_margin(double rn, double ps) { return kScreenMargin * rn + kScreenNormMargin * ps; }
+
+// power-of-two scale that brings a residual of norm rn into [2^12, 2^13): no binary16 overflow, and entries
+// down to 2^-26 of the norm stay normal numbers
+__device__ __forceinline__ double residual_scale(double rn) {
+    if (!(rn > 0.0) || !isfinite(rn)) return 1.0;
+    int e;
+    frexp(rn, &e);
+    return ldexp(1.0, 13 - e);
 }
 
 // shared memory of the bookkeeping code (blocks 0 and 1 of k_omp, the only block of k_resolve)
@@ -118,10 +128,14 @@ struct BookSmem {
 __device__ void rescore_column(const OmpArgs& a, BookSmem& sh, uint32_t idx, const double* r, double* dot_out, double* n2_out) {
     const ColKey key = column_key(a.seed_lo, a.seed_hi, idx);
     double dot = 0.0, n2 = 0.0;
-    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) {
-        const double z = (double)z_from_word(key.ck + (uint32_t)row * key.mk);
-        dot += z * r[row];
-        n2 += z * z;
+    for (int row = 2 * threadIdx.x; row < a.k; row += 2 * kOmpThreads) {            // one generated word = two rows
+        const float2 zz = half2_bits_to_float2(z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk));
+        dot += (double)zz.x * r[row];
+        n2 += (double)zz.x * (double)zz.x;
+        if (row + 1 < a.k) {
+            dot += (double)zz.y * r[row + 1];
+            n2 += (double)zz.y * (double)zz.y;
+        }
     }
     *dot_out = block_sum(dot, sh.red);
     *n2_out = block_sum(n2, sh.red);
@@ -166,7 +180,7 @@ __device__ double rebuild_prefix(const OmpArgs& a, BookSmem& sh, int m, int v, d
     double rn2 = 0.0;
     for (int row = threadIdx.x; row < k; row += kOmpThreads) {
         double acc = 0.0;
-        for (int l = 0; l < v; ++l) acc += sh.xs[l] * (double)bf16_bits_to_float(zs[(size_t)l * k + row]);
+        for (int l = 0; l < v; ++l) acc += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r_out[row] = rv;
         if (r32_out) r32_out[2 * row + m] = (float)rv;
@@ -176,9 +190,13 @@ __device__ double rebuild_prefix(const OmpArgs& a, BookSmem& sh, int m, int v, d
     return sqrt(rn2);
 }
 
-__device__ void write_rt_row(const OmpArgs& a, int m, int c, const double* r) {
-    uint16_t* dst = a.rt + ((size_t)m * a.half_n + c) * a.k;
-    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) dst[row] = bf16_rn_bits((float)r[row]);
+// residual r (norm rn) becomes row c of stream m of the screened batch: binary16, scaled by a power of two
+__device__ void write_rt_row(const OmpArgs& a, int m, int c, const double* r, double rn) {
+    const int n = m * a.half_n + c;
+    uint16_t* dst = a.rt + (size_t)n * a.k;
+    const double sc = residual_scale(rn);
+    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) dst[row] = half_rn_bits(r[row] * sc);
+    if (threadIdx.x == 0) a.inv_scale[n] = (float)(1.0 / sc);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -190,6 +208,7 @@ __device__ void corr_all_columns(const OmpArgs& a, float2* sr, uint32_t (*mask_i
     const float2* r32 = reinterpret_cast<const float2*>(a.r32);
     __syncthreads();
     for (int j = threadIdx.x; j < k; j += kOmpThreads) sr[j] = r32[j];
+    if (threadIdx.x == 0) sr[k] = make_float2(0.0f, 0.0f);          // partner of the last row when k is odd
     Top2 best[2];
     best[0].init(); best[1].init();
     constexpr unsigned int kTileCols = kOmpThreads * kCorrCols;
@@ -213,16 +232,20 @@ __device__ void corr_all_columns(const OmpArgs& a, float2* sr, uint32_t (*mask_i
             am[c] = av[c] = an[c] = 0.0f;
         }
         __syncthreads();
-#pragma unroll 4
-        for (int row = 0; row < k; ++row) {
-            const float2 rr = sr[row];
+#pragma unroll 2
+        for (int row = 0; row < k; row += 2) {                      // one generated word = two rows
+            const float2 r0 = sr[row], r1 = sr[row + 1];
+            const bool both = row + 1 < k;
 #pragma unroll
             for (int c = 0; c < kCorrCols; ++c) {
-                const float z = z_from_word(h[c]);
+                const float2 z = half2_bits_to_float2(z_pair_from_word(h[c]));
                 h[c] += mk[c];
-                am[c] = __fmaf_rn(z, rr.x, am[c]);
-                av[c] = __fmaf_rn(z, rr.y, av[c]);
-                an[c] = __fmaf_rn(z, z, an[c]);
+                am[c] = __fmaf_rn(z.x, r0.x, am[c]);
+                av[c] = __fmaf_rn(z.x, r0.y, av[c]);
+                an[c] = __fmaf_rn(z.x, z.x, an[c]);
+                am[c] = __fmaf_rn(z.y, r1.x, am[c]);
+                av[c] = __fmaf_rn(z.y, r1.y, av[c]);
+                if (both) an[c] = __fmaf_rn(z.y, z.y, an[c]);
             }
         }
 #pragma unroll
@@ -275,13 +298,19 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
         float dm = 0.0f, dv = 0.0f, n2 = 0.0f;
         uint32_t h = key.ck + (uint32_t)lane * key.mk;
         const uint32_t step = 32u * key.mk;
-        for (int row = lane; row < k; row += 32) {
-            const float z = z_from_word(h);
+        for (int row = 2 * lane; row < k; row += 64) {              // one generated word = two rows
+            const float2 z = half2_bits_to_float2(z_pair_from_word(h));
             h += step;
-            const float2 rr = r32[row];
-            dm = __fmaf_rn(z, rr.x, dm);
-            dv = __fmaf_rn(z, rr.y, dv);
-            n2 = __fmaf_rn(z, z, n2);
+            const float2 r0 = r32[row];
+            dm = __fmaf_rn(z.x, r0.x, dm);
+            dv = __fmaf_rn(z.x, r0.y, dv);
+            n2 = __fmaf_rn(z.x, z.x, n2);
+            if (row + 1 < k) {
+                const float2 r1 = r32[row + 1];
+                dm = __fmaf_rn(z.y, r1.x, dm);
+                dv = __fmaf_rn(z.y, r1.y, dv);
+                n2 = __fmaf_rn(z.y, z.y, n2);
+            }
         }
         dm = warp_sum(dm); dv = warp_sum(dv); n2 = warp_sum(n2);
         const float inv = n2 > 0.0f ? 1.0f / n2 : 0.0f;
@@ -364,10 +393,10 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
         if (threadIdx.x == 0) {
             const double ps = sqrt(sh.best_score), rn = sh.cur_rnorm, unit = rn / sqrt((double)k);
             a.pick_score[(size_t)m * s + j] = ps;
-            double t = ps - kScreenMargin * rn;
+            double t = ps - screen_margin(rn, ps);
             if (t > a.z_harvest * unit) t = a.z_harvest * unit;
             if (t < a.z_floor * unit) t = a.z_floor * unit;
-            a.tau[m * a.half_n + spec_c] = (float)t;
+            a.tau[m * a.half_n + spec_c] = (float)(t * residual_scale(rn));     // row spec_c was scaled with this norm
             a.lam[(size_t)m * s + j] = lam_new;
         }
     }
@@ -375,8 +404,11 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     {
         const ColKey key = column_key(a.seed_lo, a.seed_hi, lam_new);
         uint16_t* znew = zs + (size_t)j * k;
-        for (int row = threadIdx.x; row < k; row += kOmpThreads)
-            znew[row] = z_bf16_bits(z_from_word(key.ck + (uint32_t)row * key.mk));
+        for (int row = 2 * threadIdx.x; row < k; row += 2 * kOmpThreads) {
+            const uint32_t z2 = z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk);
+            znew[row] = (uint16_t)(z2 & 0xFFFFu);
+            if (row + 1 < k) znew[row + 1] = (uint16_t)(z2 >> 16);
+        }
     }
     __syncthreads();
     // ---- 4. g = A_Lambda^T a_new  (Gram column; "g_{:,lambda_k}" restricted to the support) --------------
@@ -387,7 +419,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
             const uint16_t* zl = zs + (size_t)l * k;
             double acc = 0.0;
             for (int row = lane; row < k; row += 32)
-                acc += (double)(bf16_bits_to_float(zl[row]) * bf16_bits_to_float(znew[row]));   // product exact in fp32
+                acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));   // product exact in fp32
             acc = warp_sum(acc);
             if (lane == 0) sh.gvec[l] = sig2 * acc;
         }
@@ -432,17 +464,16 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     __syncthreads();
     // ---- 9. r = y - A_Lambda x ---------------------------------------------------------------------------
     double rn2 = 0.0;
-    uint16_t* rt_row = spec_next >= 0 ? a.rt + ((size_t)m * a.half_n + spec_next) * k : nullptr;
     for (int row = threadIdx.x; row < k; row += kOmpThreads) {
         double acc = 0.0;
-        for (int l = 0; l <= j; ++l) acc += sh.xs[l] * (double)bf16_bits_to_float(zs[(size_t)l * k + row]);
+        for (int l = 0; l <= j; ++l) acc += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r[row] = rv;
         a.r32[2 * row + m] = (float)rv;
-        if (rt_row) rt_row[row] = bf16_rn_bits((float)rv);
         rn2 += rv * rv;
     }
     rn2 = block_sum(rn2, sh.red);
+    if (spec_next >= 0) write_rt_row(a, m, spec_next, r, sqrt(rn2));      // each thread re-reads the rows it wrote
     if (threadIdx.x == 0) {
         a.rnorm[(size_t)m * s + j] = sqrt(rn2);
         sh.cur_rnorm = sqrt(rn2);
@@ -483,7 +514,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
                 sh.hi = base[mb]; sh.extra = 0; sh.dep = 0;
                 a.ctl->stop[mb] = 0;
             }
-            if (mode == 0 && forced0[mb] == kNoColumn) write_rt_row(a, mb, 0, a.r64 + (size_t)mb * a.k);
+            if (mode == 0 && forced0[mb] == kNoColumn) write_rt_row(a, mb, 0, a.r64 + (size_t)mb * a.k, rn);
         } else if (threadIdx.x == 0) {
             a.ctl->stop[mb] = 1;
         }
@@ -526,7 +557,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
                     // pick is screened, and the recovery stops there if the pick is confirmed
                     if (rc == 1) {
                         sh.extra = 1;
-                        a.tau[m * a.half_n + c] = (float)(a.z_harvest * sh.cur_rnorm / sqrt((double)a.k));
+                        a.tau[m * a.half_n + c] =
+                            (float)(a.z_harvest * sh.cur_rnorm / sqrt((double)a.k) * residual_scale(sh.cur_rnorm));
                     } else { sh.dep = 1; sh.hi = j + 1; }
                     a.ctl->stop[m] = 1;
                 } else {
@@ -652,7 +684,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             const uint32_t pick = lam[j];
             const double ps = a.pick_score[(size_t)m * s + j];
             const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
-            const float margin = (float)(kScreenMargin * rn);
+            const float margin = (float)screen_margin(rn, ps);
             if (threadIdx.x == 0) sh.cand_idx[0] = pick;
             const int nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, j, pick, (float)ps - margin,
                                                2.0f * margin, 1);
@@ -680,7 +712,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                 const int n = m * a.half_n + (hi - base);
                 const unsigned int count = a.rep_count[n];
                 const double rn = hi == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + hi - 1];
-                const float margin = (float)(kScreenMargin * rn);
+                const float margin = (float)screen_margin(rn, 8.0 * rn / sqrt((double)a.k));    // scores near the noise maximum
                 int nc = -1;
                 if (count >= 1u && count <= (unsigned int)ra.rep_cap)
                     nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, hi, kNoColumn, 0.0f, 2.0f * margin, 0);
@@ -830,7 +862,7 @@ OmpArgs make_args(const sgc_state* st) {
     a.corr_cand = st->corr_cand; a.y64 = st->y64; a.r64 = st->r64; a.r32 = reinterpret_cast<float*>(st->r32);
     a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
     a.cnt = st->cnt; a.ctl = st->ctl;
-    a.rt = st->rt; a.tau = st->tau; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
+    a.rt = st->rt; a.tau = st->tau; a.inv_scale = st->inv_scale; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
     a.cand_list = st->cand_list;
     return a;
 }
@@ -846,7 +878,7 @@ cudaError_t launch_omp(sgc_state* st, const OmpArgs& a, int mode, cudaStream_t s
 }  // namespace
 
 cudaError_t configure_recover(sgc_state* st) {
-    const size_t smem = (size_t)st->k * sizeof(float2);
+    const size_t smem = ((size_t)st->k + 1) * sizeof(float2);
     cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int occ = 0;
@@ -900,8 +932,8 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
             if (e != cudaSuccess) break;
             {
                 PhaseTimer timer(st, stream, kPhasePass, 1);
-                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->rep_count, st->rep, kRepCap,
-                                &st->ctl->round_active, &st->ctl->pass_error, st->sm_count, stream);
+                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale, st->rep_count,
+                                st->rep, kRepCap, &st->ctl->round_active, &st->ctl->pass_error, st->sm_count, stream);
             }
             if (e != cudaSuccess) break;
             {

@@ -2,8 +2,8 @@
 
 Usage: python tests/golden/make_golden.py   (from the repository root)
 Output: tests/golden/z_seed0.txt, z_seed1.txt : 32x32 blocks at (row0, col0) = (0, 0) and one block
-far into the index space, as hex of the upper 16 bits of the float32 bit patterns (the lower 16 are zero by definition), plus an XOR checksum of a
-2^20-entry block.  There is no printed example in the paper to take these from; the paper fixes
+far into the index space, as hex of the binary16 bit patterns (every Z is a binary16 number by definition), plus an XOR
+checksum and a sum of the patterns of a 2^20-entry block.  There is no printed example in the paper to take these from; the paper fixes
 only the distribution (Section 3.3), which tests/test_oracle_a_matrix.py checks separately.
 """
 import os
@@ -23,15 +23,16 @@ def main():
     for seed in (0, 1, 0x123456789ABCDEF):
         name = "z_seed%x.txt" % seed
         with open(os.path.join(here, name), "w") as f:
-            f.write("# Z(seed=%d) golden blocks; rows of 32 hex upper-half float32 bit patterns\n" % seed)
+            f.write("# Z(seed=%d) golden blocks; rows of 32 hex binary16 bit patterns\n" % seed)
             for (r0, c0) in BLOCKS:
-                z = oracle.z_block(seed, r0, 32, c0, 32).view(np.uint32)
-                assert not np.any(z & 0xFFFF)
+                z = oracle.z_block(seed, r0, 32, c0, 32)
+                zh = z.astype(np.float16)
+                assert np.array_equal(zh.astype(np.float32), z)
                 f.write("block %d %d\n" % (r0, c0))
                 for r in range(32):
-                    f.write(" ".join("%04x" % (v >> 16) for v in z[r]) + "\n")
-            big = oracle.z_block(seed, 0, 1024, 1000, 1024).view(np.uint32)
-            f.write("xor1M %08x\n" % int(np.bitwise_xor.reduce(big.ravel())))
+                    f.write(" ".join("%04x" % v for v in zh[r].view(np.uint16)) + "\n")
+            big = oracle.z_block(seed, 0, 1024, 1000, 1024).astype(np.float16).view(np.uint16)
+            f.write("xor1M %04x\n" % int(np.bitwise_xor.reduce(big.ravel())))
             f.write("sum1M %d\n" % int(big.ravel().astype(np.uint64).sum()))
 
 

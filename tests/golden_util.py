@@ -1,4 +1,4 @@
-"""Reader for tests/golden/z_seed*.txt (written by tests/golden/make_golden.py from the oracle)."""
+"""Reader for tests/golden/z_seed*.txt (written by tests/golden/make_golden.py from the oracle): binary16 bit patterns."""
 import os
 
 import numpy as np
@@ -24,5 +24,5 @@ def read_z_golden(seed):
             elif line.startswith("sum1M"):
                 total = int(line.split()[1])
             else:
-                blocks[cur].append([int(v, 16) << 16 for v in line.split()])
-    return {k: np.array(v, dtype=np.uint32) for k, v in blocks.items()}, xor, total
+                blocks[cur].append([int(v, 16) for v in line.split()])
+    return {k: np.array(v, dtype=np.uint16) for k, v in blocks.items()}, xor, total

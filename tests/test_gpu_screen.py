@@ -1,9 +1,10 @@
 """The tensor-core screening pass (sgc_screen) against the plain definition computed from the oracle's A generator.
 
 For every residual j the pass must report exactly the columns i with |<Z_i, R_j>| / ||Z_i|| >= tau_j.  The reference
-takes Z from the oracle (bit-identical generator), R as the very bfloat16 values handed to the GPU, and evaluates the
-definition in fp64.  Pairs whose exact score lies within 1e-4 (relative) of the threshold may fall on either side
-(fp32 accumulation on the tensor cores); every other pair must match, and reported scores must agree to 1e-4.
+takes Z from the oracle (bit-identical generator), R as the very binary16 values handed to the GPU, and evaluates the
+definition in fp64.  The pass accumulates the column norm ||Z_i||^2 in short binary16 partial sums, which the library
+documents as a relative score error of at most 1e-3: pairs whose exact score lies within 1e-3 (relative) of the
+threshold may fall on either side; every other pair must match, and reported scores must agree to 1e-3.
 """
 import numpy as np
 import pytest
@@ -13,11 +14,10 @@ import oracle
 pytestmark = pytest.mark.gpu
 
 
-def bf16_round(x):
-    """float32 array -> (values representable in bfloat16 as float32, their 16-bit patterns); round to nearest even."""
-    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
-    r = ((b + 0x7FFF + ((b >> 16) & 1)) >> 16).astype(np.uint16)
-    return (r.astype(np.uint32) << 16).view(np.float32), r
+def half_round(x):
+    """float32 array -> (the nearest binary16 values as float32, their 16-bit patterns)."""
+    h = np.ascontiguousarray(x, dtype=np.float32).astype(np.float16)
+    return h.astype(np.float32), h.view(np.uint16)
 
 
 @pytest.mark.parametrize("d,k,n,seed", [(5000, 256, 32, 0), (100_003, 256, 128, 1), (40_000, 128, 256, 7),
@@ -27,7 +27,7 @@ def test_screen_reports_exactly_the_columns_above_threshold(d, k, n, seed):
     from paper_2502_00311_b200 import binding
     rng = np.random.default_rng(d + k + n)
     Z = oracle.z_block(seed, 0, k, 0, d).astype(np.float64)              # k x d
-    R, bits = bf16_round(rng.standard_normal((n, k)).astype(np.float32) * rng.uniform(0.01, 3.0, size=(n, 1)).astype(np.float32))
+    R, bits = half_round(rng.standard_normal((n, k)).astype(np.float32) * rng.uniform(0.01, 3.0, size=(n, 1)).astype(np.float32))
     norms = np.sqrt((Z * Z).sum(axis=0))
     scores = np.abs(R.astype(np.float64) @ Z) / norms                       # n x d
     # thresholds: a few dozen expected reports per residual; one residual disabled, one reporting nothing
@@ -48,12 +48,12 @@ def test_screen_reports_exactly_the_columns_above_threshold(d, k, n, seed):
         cols = rep[j, :c, 0].view(np.uint32).astype(np.int64)
         got_sc = rep[j, :c, 1].copy().view(np.float32)
         assert cols.size == np.unique(cols).size and (cols < d).all()
-        sure = set(np.nonzero(scores[j] >= tau[j] * (1 + 1e-4))[0].tolist())
-        maybe = set(np.nonzero(scores[j] >= tau[j] * (1 - 1e-4))[0].tolist())
+        sure = set(np.nonzero(scores[j] >= tau[j] * (1 + 1e-3))[0].tolist())
+        maybe = set(np.nonzero(scores[j] >= tau[j] * (1 - 1e-3))[0].tolist())
         got = set(cols.tolist())
         assert sure <= got <= maybe, (j, sorted(sure - got)[:5], sorted(got - maybe)[:5])
         if c:
-            np.testing.assert_allclose(got_sc, scores[j][cols], rtol=1e-4)
+            np.testing.assert_allclose(got_sc, scores[j][cols], rtol=1e-3)
 
 
 def test_screen_rejects_bad_arguments():
