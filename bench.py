@@ -49,7 +49,7 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU every 200 ms while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons of one GPU every 50 ms while the timed region runs."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -61,7 +61,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -239,7 +239,7 @@ def run_ours(args, wl):
             achieved = 2.0 * k * d * n_pass / pass_avg_s / 1e12
             roof = {"kernel": "k_pass", "bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                     "frac": achieved / pk["bf16_tflops"], "traffic": None, "peak_source": pk["source"],
-                    "note": "2*k*d*N flops per pass (N = %d residuals, bf16 x bf16 -> fp32 on tcgen05); the operand A is "
+                    "note": "2*k*d*N flops per pass (N = %d residuals, f16 x f16 -> fp32 on tcgen05); the operand A is "
                             "regenerated by the CUDA cores (k*d entries per pass), which is what limits the pass" % n_pass,
                     "avg_launch_ms": pass_avg_s * 1e3, "launches": sum(rounds),
                     "generated_entries_per_s": k * d / pass_avg_s}
@@ -288,7 +288,7 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_4096x4096", choices=sorted(WORKLOADS))

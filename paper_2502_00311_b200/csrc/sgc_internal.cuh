@@ -63,9 +63,8 @@ __device__ __forceinline__ uint32_t z_pair_from_word(uint32_t h0) {
     uint32_t h = h0;
     h ^= h >> 16; h *= kMulEntry; h ^= h >> 15;
     // byte pair sums straight into the significand of the half 1024: the halves 1024 + S (exact, S <= 510)
-    const uint32_t e0 = __dp4a(h, 0x00000101u, 0x6400u);
-    const uint32_t e1 = __dp4a(h, 0x01010000u, 0x6400u);
-    const uint32_t s2 = __byte_perm(e0, e1, 0x5410);
+    // (bytes 0 and 2) + (bytes 1 and 3) as two 16-bit fields: byte permutes and one add, all on the integer pipe
+    const uint32_t s2 = __byte_perm(h, 0u, 0x4240) + __byte_perm(h, 0u, 0x4341) + 0x64006400u;
     const uint32_t x = hfma2(s2, kInv256x2, kCentrex2);        // (S - 255)/256, exact
     const uint32_t w = hmul2(x, x);
     uint32_t q = hfma2(w, kC2x2, kC1x2);
@@ -228,7 +227,6 @@ cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set
 cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T
 
 // screening pass (sgc_pass.cu)
-int pass_stages(int n);
 cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,

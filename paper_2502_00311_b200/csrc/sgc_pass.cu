@@ -215,23 +215,27 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         // ---------------- MMA issuer ----------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(a.n);
+            // descriptors differ only in their start-address field (units of 16 bytes): keep that word per stage
+            const uint64_t desc_hi = umma_desc(0) & 0xFFFFFFFF00000000ull;
+            const uint32_t desc_lo0 = (uint32_t)(umma_desc(base) & 0xFFFFFFFFull);
+            const uint32_t stage_step = (uint32_t)stage_bytes >> 4;
             uint32_t st = 0, ph = 0, sweep_i = 0;
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
                 const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
-                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 64)) { ok = false; break; }
+                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 32)) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t acc0 = tmem_base + buf * acc_cols, acc1 = acc0 + a.n;
                 for (int kc = 0; kc < kc_count; ++kc) {
-                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 32)) { ok = false; break; }
+                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 0)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = base + st * stage_bytes;
+                    const uint32_t lo = desc_lo0 + st * stage_step;
+                    const uint32_t first = kc != 0 ? 1u : 0u;
 #pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-#pragma unroll
-                        for (int kk = 0; kk < kChunkRows / 16; ++kk) {
-                            umma_f16(tmem_base + buf * acc_cols + t * a.n, umma_desc(sa + t * kTileBytes + kk * 32),
-                                      umma_desc(sa + 2 * kTileBytes + kk * 32), idesc, (kc | kk) != 0 ? 1u : 0u);
-                        }
+                    for (int kk = 0; kk < kChunkRows / 16; ++kk) {
+                        const uint64_t bdesc = desc_hi | (uint64_t)(lo + (2 * kTileBytes >> 4) + 2 * kk);
+                        umma_f16(acc0, desc_hi | (uint64_t)(lo + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                        umma_f16(acc1, desc_hi | (uint64_t)(lo + (kTileBytes >> 4) + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
                     }
                     umma_commit(bar_empty + 8u * st);        // frees the stage once these MMAs have read it
                     if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
