@@ -31,7 +31,7 @@ size_t layout(sgc_state* st, unsigned char* base) {
     st->r32 = carve<float2>(base, off, k);
     st->sel_cand = carve<unsigned long long>(base, off, sgc::kSelCap);
     st->sel_hist = carve<unsigned int>(base, off, sgc::kSelBins);
-    st->corr_cand = carve<sgc::Cand>(base, off, 2 * (size_t)st->corr_grid * sgc::kCorrTop);
+    st->corr_cand = carve<sgc::Cand>(base, off, 2 * (size_t)(st->corr_grid > 32 ? st->corr_grid : 32) * sgc::kCorrTop);
     st->zsel = carve<uint16_t>(base, off, 2 * s * k);
     st->lam = carve<uint32_t>(base, off, 2 * s);
     st->F = carve<double>(base, off, 2 * s * s);

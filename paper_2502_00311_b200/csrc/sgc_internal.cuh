@@ -105,6 +105,7 @@ constexpr int kBookThreads = 1024;
 constexpr int kOmpThreads = 1024;       // threads per block of the cooperative OMP kernel
 constexpr int kCandCap = 8192;          // candidate columns kept for the restricted (speculative) OMP
 constexpr int kCandKeep = 4096;         // the list is rebuilt from the supports once it grows beyond this
+constexpr int kSmallList = 768;         // lists up to this length are correlated inside the bookkeeping block
 constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
 constexpr int kMaxRounds = 8;           // speculate / screen / resolve rounds enqueued per step
@@ -133,6 +134,7 @@ struct SpecCtl {
     int rounds;             // screening passes that did work in the last step
     int pass_error;         // a wait inside the screening pass expired
     int stop[2];            // scratch of the cooperative kernel: speculation of residual m has ended
+    int list_exact[2];      // 1: the last speculation of residual m compared every list member exactly
     double ynorm[2];        // ||y|| per residual
 };
 

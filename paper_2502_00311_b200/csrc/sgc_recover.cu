@@ -120,7 +120,7 @@ struct BookSmem {
     uint32_t best_idx;
     uint32_t cand_idx[kRescoreCap];
     int n_cand;
-    int hi, extra, dep;               // speculation record of this block's stream
+    int hi, extra, dep, stop;         // speculation record of this block's stream
     unsigned int smax_bits;
 };
 
@@ -172,6 +172,7 @@ __device__ double rebuild_prefix(const OmpArgs& a, BookSmem& sh, int m, int v, d
     if ((int)threadIdx.x < v) {
         const int i = threadIdx.x;
         double acc = 0.0;
+#pragma unroll 8
         for (int l = i; l < v; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
         sh.xs[i] = acc;
         if (x_out) x_out[i] = acc;
@@ -180,6 +181,7 @@ __device__ double rebuild_prefix(const OmpArgs& a, BookSmem& sh, int m, int v, d
     double rn2 = 0.0;
     for (int row = threadIdx.x; row < k; row += kOmpThreads) {
         double acc = 0.0;
+#pragma unroll 8
         for (int l = 0; l < v; ++l) acc += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r_out[row] = rv;
@@ -339,7 +341,7 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
 // recorded); spec_next >= 0: the new residual becomes row spec_next of the screened batch.
 // ------------------------------------------------------------------------------------------------
 __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t forced, int spec_c, int spec_next,
-                         bool final_pick) {
+                         bool final_pick, const Cand* cc, int n_entries) {
     const int k = a.k, s = a.s;
     const double* y = a.y64 + (size_t)m * k;
     double* r = a.r64 + (size_t)m * k;
@@ -355,8 +357,6 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
         __syncthreads();
     } else {
         // ---- 1. screened candidates: everything within 2e-3 (relative, squared scores) of the best fp32 score
-        const Cand* cc = a.corr_cand + (size_t)m * gridDim.x * kCorrTop;
-        const int n_entries = gridDim.x * kCorrTop;
         float mx = -1.0f;
         for (int e = threadIdx.x; e < n_entries; e += kOmpThreads) {
             const Cand c = cc[e];
@@ -418,6 +418,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
         for (int l = warp; l < j; l += kOmpThreads / 32) {
             const uint16_t* zl = zs + (size_t)l * k;
             double acc = 0.0;
+#pragma unroll 8
             for (int row = lane; row < k; row += 32)
                 acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));   // product exact in fp32
             acc = warp_sum(acc);
@@ -430,6 +431,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     if ((int)threadIdx.x < j) {
         const int i = threadIdx.x;
         double acc = 0.0;
+#pragma unroll 8
         for (int l = 0; l <= i; ++l) acc += F[(size_t)l * s + i] * sh.gvec[l];
         sh.cvec[i] = acc;
         csq = acc * acc;
@@ -445,6 +447,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     if ((int)threadIdx.x < j) {
         const int i = threadIdx.x;
         double acc = 0.0;
+#pragma unroll 8
         for (int l = i; l < j; ++l) acc += F[(size_t)i * s + l] * sh.cvec[l];
         F[(size_t)i * s + j] = -gamma * acc;
     } else if ((int)threadIdx.x == j) {
@@ -466,6 +469,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     double rn2 = 0.0;
     for (int row = threadIdx.x; row < k; row += kOmpThreads) {
         double acc = 0.0;
+#pragma unroll 8
         for (int l = 0; l <= j; ++l) acc += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r[row] = rv;
@@ -496,7 +500,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
     volatile SpecCtl* ctl = a.ctl;
     // ---- gate: identical in every block, because nothing below changes the control block before the first barrier
     const int fin[2] = {ctl->finished[0], ctl->finished[1]};
-    if (mode == 0) { if (!ctl->round_active || ctl->fallback) return; }
+    if (mode == 0) { if (!ctl->round_active || ctl->fallback || ctl->n_cand <= kSmallList) return; }
     else { if (fin[0] && fin[1]) return; }
     const int v0[2] = {ctl->v[0], ctl->v[1]};
     const uint32_t forced0[2] = {ctl->forced[0], ctl->forced[1]};
@@ -548,7 +552,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
             const bool speculative = (mode == 0) && forced == kNoColumn;
             const int c = j - base[m];                            // -1 for a forced pick
             const int next = (mode == 0 && c + 1 < a.half_n && j + 1 < a.s) ? c + 1 : -1;
-            const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative);
+            const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative,
+                                     a.corr_cand + (size_t)m * gridDim.x * kCorrTop, (int)gridDim.x * kCorrTop);
             if (threadIdx.x == 0) {
                 if (rc == 0) {
                     sh.hi = j + 1;
@@ -581,10 +586,111 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
             a.ctl->hi[mb] = sh.hi < base[mb] ? base[mb] : sh.hi;
             a.ctl->extra[mb] = sh.extra;
             a.ctl->dep[mb] = sh.dep;
+            a.ctl->list_exact[mb] = 0;    // only the best two candidates of every block reached the fp64 decision
         } else if (!a.ctl->finished[mb]) {
             a.cnt->done[mb] = a.ctl->v[mb];
             a.ctl->finished[mb] = 1;
         }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// speculation on a short candidate list (at most kSmallList columns): block m runs the whole OMP of residual m
+// by itself -- correlation of the list (warp = one column), pick, Algorithm 3 -- without any grid barrier.
+// Same records as k_omp mode 0.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kOmpThreads, 1) k_spec_small(OmpArgs a) {
+    extern __shared__ float2 sr[];
+    __shared__ BookSmem sh;
+    __shared__ Cand scored[kSmallList];                  // screen score of every candidate: the pick is exact within the list
+    float* rs = reinterpret_cast<float*>(sr);            // the residual of this block's stream, fp32
+    volatile SpecCtl* ctl = a.ctl;
+    const int n_cand = ctl->n_cand;
+    if (!ctl->round_active || ctl->fallback || n_cand > kSmallList) return;
+    const int m = blockIdx.x, k = a.k, s = a.s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c = threadIdx.x; c < a.half_n; c += kOmpThreads) {
+        a.rep_count[m * a.half_n + c] = 0u;
+        a.tau[m * a.half_n + c] = __int_as_float(0x7f800000);
+    }
+    if (ctl->finished[m]) return;
+    const int v0 = ctl->v[m];
+    const uint32_t forced0 = ctl->forced[m];
+    const int base = v0 + (forced0 != kNoColumn ? 1 : 0);
+    const double rn0 = rebuild_prefix(a, sh, m, v0, a.r64 + (size_t)m * k, a.r32, a.x + (size_t)m * s);
+    if (threadIdx.x == 0) {
+        sh.cur_rnorm = rn0;
+        if (v0 == 0) a.ctl->ynorm[m] = rn0;
+        sh.hi = base; sh.extra = 0; sh.dep = 0; sh.stop = 0;
+    }
+    if (forced0 == kNoColumn) write_rt_row(a, m, 0, a.r64 + (size_t)m * k, rn0);
+    __syncthreads();
+    for (int j = v0; j < s; ++j) {
+        const int c = j - base;                                       // -1 for the forced pick
+        if (c >= a.half_n || sh.stop) break;
+        const uint32_t forced = (j == v0) ? forced0 : kNoColumn;
+        if (forced == kNoColumn) {
+            // phase A inside the block: every candidate column against this residual
+            __syncthreads();
+            for (int row = threadIdx.x; row < k; row += kOmpThreads) rs[row] = a.r32[2 * row + m];
+            if (threadIdx.x == 0) rs[k] = 0.0f;
+            __syncthreads();
+            for (int e = warp; e < n_cand; e += kOmpThreads / 32) {
+                const uint32_t col = a.cand_list[e];
+                bool taken = false;
+                for (int q = lane; q < j; q += 32) taken |= (a.lam[(size_t)m * s + q] == col);
+                if (__any_sync(0xffffffffu, taken)) {
+                    if (lane == 0) { scored[e].score = -1.0f; scored[e].idx = kNoColumn; }
+                    continue;
+                }
+                const ColKey key = column_key(a.seed_lo, a.seed_hi, col);
+                float dot = 0.0f, n2 = 0.0f;
+                uint32_t h = key.ck + (uint32_t)lane * key.mk;
+                const uint32_t step = 32u * key.mk;
+                for (int row = 2 * lane; row < k; row += 64) {         // one generated word = two rows
+                    const float2 z = half2_bits_to_float2(z_pair_from_word(h));
+                    h += step;
+                    dot = __fmaf_rn(z.x, rs[row], dot);
+                    n2 = __fmaf_rn(z.x, z.x, n2);
+                    dot = __fmaf_rn(z.y, rs[row + 1], dot);
+                    if (row + 1 < k) n2 = __fmaf_rn(z.y, z.y, n2);
+                }
+                dot = warp_sum(dot); n2 = warp_sum(n2);
+                if (lane == 0) { scored[e].score = n2 > 0.0f ? dot * dot / n2 : 0.0f; scored[e].idx = col; }
+            }
+            __syncthreads();
+        }
+        const bool speculative = forced == kNoColumn;
+        const int next = (c + 1 < a.half_n && j + 1 < s) ? c + 1 : -1;
+        const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative, scored, n_cand);
+        if (threadIdx.x == 0) {
+            if (rc == 0) {
+                sh.hi = j + 1;
+            } else if (speculative) {
+                if (rc == 1) {
+                    sh.extra = 1;
+                    a.tau[m * a.half_n + c] =
+                        (float)(a.z_harvest * sh.cur_rnorm / sqrt((double)k) * residual_scale(sh.cur_rnorm));
+                } else { sh.dep = 1; sh.hi = j + 1; }
+                sh.stop = 1;
+            } else {
+                a.cnt->stopped[m] = 1;
+                atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN);
+                a.cnt->done[m] = j;
+                a.ctl->v[m] = j;
+                a.ctl->finished[m] = 1;
+                sh.stop = 1;
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        a.ctl->base[m] = base;
+        a.ctl->hi[m] = sh.hi < base ? base : sh.hi;
+        a.ctl->extra[m] = sh.extra;
+        a.ctl->dep[m] = sh.dep;
+        // every list member was scored, and all near-maximal ones decided in fp64 unless their buffer overflowed
+        a.ctl->list_exact[m] = (a.cnt->status & (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW) ? 0 : 1;
     }
 }
 
@@ -667,9 +773,36 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         if (threadIdx.x == 0) { ctl->fallback = 1; ctl->round_active = 0; }
         return;
     }
+    __shared__ int contested[kPassMaxN];        // per screened residual: some report comes within the margin of its pick
     if (threadIdx.x == 0) { give_up = 0; ctl->rounds = ctl->rounds + 1; }
+    for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = 0;
     __syncthreads();
     const int s = a.s;
+    // one parallel sweep over all report lists; the walk below only stops at contested picks
+    for (int m = 0; m < 2; ++m) {
+        if (ctl->finished[m]) continue;
+        const int base = ctl->base[m], hi = ctl->hi[m];
+        for (int j = base + (threadIdx.x >> 5); j < hi; j += kOmpThreads / 32) {      // warp per residual
+            const int n = m * a.half_n + (j - base);
+            const unsigned int count = a.rep_count[n];
+            if (count > (unsigned int)ra.rep_cap) { if ((threadIdx.x & 31) == 0) contested[n] = 1; continue; }
+            const uint32_t pick = a.lam[(size_t)m * s + j];
+            const double ps = a.pick_score[(size_t)m * s + j];
+            const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
+            const float floor_sc = (float)ps - (float)screen_margin(rn, ps);
+            const bool skip_members = ctl->list_exact[m] != 0;
+            bool hit = false;
+            for (unsigned int e = threadIdx.x & 31; e < count; e += 32) {
+                const uint2 rp = ra.rep[(size_t)n * ra.rep_cap + e];
+                if (__uint_as_float(rp.y) < floor_sc || rp.x == pick) continue;
+                // a list member lost the exact comparison against the pick during the speculation (or is in the support)
+                if (skip_members && ((ra.cand_bits[rp.x >> 5] >> (rp.x & 31u)) & 1u)) continue;
+                if (!in_support(a.lam + (size_t)m * s, j, rp.x)) hit = true;
+            }
+            if (__any_sync(0xffffffffu, hit) && (threadIdx.x & 31) == 0) contested[n] = 1;
+        }
+    }
+    __syncthreads();
     for (int m = 0; m < 2; ++m) {
         if (ctl->finished[m]) continue;
         const int base = ctl->base[m], hi = ctl->hi[m], extra = ctl->extra[m], dep = ctl->dep[m];
@@ -679,6 +812,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         bool failed = false, bad = false;
         for (int j = base; j < hi && !failed && !bad; ++j) {
             const int n = m * a.half_n + (j - base);
+            if (!contested[n]) { v = j + 1; continue; }           // nobody comes close: the pick is the argmax
             const unsigned int count = a.rep_count[n];
             if (count > (unsigned int)ra.rep_cap) { bad = true; break; }
             const uint32_t pick = lam[j];
@@ -762,7 +896,9 @@ __global__ void __launch_bounds__(kOmpThreads, 1)
 k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uint32_t* cand_list, unsigned int* cand_bits) {
     __shared__ int n_s;
     int n = ctl->n_cand;
-    if (n > kCandKeep) {
+    // rebuild from the supports alone when the list has outgrown its bound, or when it holds far more than the
+    // supports although a single round confirmed every pick (harvested columns of an earlier cold start)
+    if (n > kCandKeep || (ctl->rounds <= 1 && !ctl->fallback && n > 4 * s)) {
         for (int e = threadIdx.x; e < n; e += kOmpThreads) {
             const uint32_t col = cand_list[e];
             atomicAnd(&cand_bits[col >> 5], ~(1u << (col & 31u)));
@@ -882,6 +1018,8 @@ cudaError_t configure_recover(sgc_state* st) {
     cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int occ = 0;
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_spec_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_omp, kOmpThreads, smem);
     if (e != cudaSuccess) return e;
     if (occ < 1) return cudaErrorInvalidConfiguration;
@@ -926,8 +1064,9 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
         ra.rtmp = st->rtmp;
         for (int round = 0; round < kMaxRounds && e == cudaSuccess; ++round) {
             {
-                PhaseTimer timer(st, stream, kPhaseCorr, 1);
-                e = launch_omp(st, a, 0, stream);
+                PhaseTimer timer(st, stream, kPhaseCorr, 2);
+                k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
+                e = launch_omp(st, a, 0, stream);                                // long candidate list
             }
             if (e != cudaSuccess) break;
             {
@@ -940,7 +1079,7 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
                 PhaseTimer timer(st, stream, kPhaseBook, 1);
                 k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
             }
-            *launches += 3;
+            *launches += 4;
         }
         if (e != cudaSuccess) return e;
     }
