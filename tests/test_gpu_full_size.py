@@ -1,0 +1,172 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times.
+
+A full oracle recovery costs k*d*s generated entries per residual (hours at d = 16.7M), so at these sizes the
+comparison is split:
+  * a1-a3 (top-s support and values, p, q, M, V, t): element by element against the oracle, every step;
+  * a4: the first picks of both recoveries against the oracle's own OMP over ALL d columns (one full pass per pick);
+    for all picks, properties that pin the result at any size, computed from the oracle's A generator:
+      - replayed on the GPU's support, OMP selects the same columns in the same order (fp64, numpy);
+      - the coefficients are the least-squares solution on that support (numpy lstsq);
+      - no column of a random sample of the other d - s columns scores above the pick, at sampled iterations;
+      - on the planted (exactly recoverable) workloads the support is the planted one;
+  * a5: the weight update against Eq. (8) evaluated with numpy on the recovered coefficients.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2502_00311_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_STATE = 1e-5
+TOL_UPDATE = 1e-4
+
+
+def rel(a, b):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    return np.abs(a - b).max() / max(np.abs(b).max(), 1e-300)
+
+
+def columns(seed, k, cols):
+    """A[:, cols] (without sigma) as float64 [k, len(cols)] from the oracle's generator."""
+    out = np.empty((k, len(cols)), dtype=np.float64)
+    for i, c in enumerate(cols):
+        out[:, i] = oracle.z_block(seed, 0, k, int(c), 1)[:, 0]
+    return out
+
+
+def check_recovery(seed, d, k, s, y, lam, x, done, rng, sample_iters=(0, 1, 7, -1)):
+    """Properties of one recovery (lam, x, done) of the target y; returns the per-iteration residuals."""
+    assert done == s
+    lam = lam[:done].astype(np.int64)
+    assert np.unique(lam).size == done and lam.max() < d
+    sigma = float(oracle.sigma(k))
+    Z = columns(seed, k, lam)
+    A = sigma * Z
+    norms = np.sqrt((Z * Z).sum(axis=0))
+    # replay: on these columns OMP must choose them in this very order
+    r = y.copy()
+    residuals = []
+    for j in range(done):
+        residuals.append(r.copy())
+        sc = np.abs(Z.T @ r) / norms
+        sc[:j] = -1.0
+        assert int(np.argmax(sc)) == j, "pick %d is not the best of the support" % j
+        xj = np.linalg.lstsq(A[:, :j + 1], y, rcond=None)[0]
+        r = y - A[:, :j + 1] @ xj
+    xls = np.linalg.lstsq(A, y, rcond=None)[0]
+    assert rel(x[:done], xls) < TOL_UPDATE
+    # a random sample of the other columns never beats the pick (contiguous blocks are cheap to generate)
+    n_blocks = max(4, min(32, (1 << 25) // (k * 512)))
+    for it in sample_iters:
+        j = it % done
+        rj = residuals[j]
+        pick_score = abs(Z[:, j] @ rj) / norms[j]
+        for b in rng.integers(0, max(1, d - 512), size=n_blocks):
+            blk = oracle.z_block(seed, 0, k, int(b), 512).astype(np.float64)
+            sc = np.abs(rj @ blk) / np.sqrt((blk * blk).sum(axis=0))
+            idx = np.arange(int(b), int(b) + 512)
+            sc[np.isin(idx, lam[:j + 1])] = 0.0
+            assert float(sc.max()) <= pick_score, (j, float(sc.max()), pick_score)
+    return residuals
+
+
+def run_config(sgc, d, k, s, seed, cfg_id, steps, planted, full_oracle_picks=0, mode=None):
+    import torch
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    if mode is not None:
+        st.set_mode(mode)
+    ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0))
+    w0 = inputs.weights(d, 99)
+    w_gpu = torch.from_numpy(w0.copy()).cuda()
+    rng = np.random.default_rng(1234 + cfg_id)
+    rounds = []
+    seen = set()                                                # every index that was ever kept by Sparsify_s
+    for step in range(1, steps + 1):
+        g = inputs.gradient(d, "student", supp, sign, inputs.step_seed(cfg_id, 0, step))
+        w_before = w_gpu.cpu().numpy()
+        st.step(torch.from_numpy(g).cuda(), w_gpu)
+        ref.step_compress(g)                                    # a1-a3 of the oracle
+        assert st.get("t") == step == ref.get("t")
+        assert np.array_equal(st.get("sel_idx"), ref.get("sel_idx"))
+        assert np.array_equal(st.get("sel_val"), ref.get("sel_val"))
+        for name in ("p", "q", "M", "V"):
+            assert rel(st.get(name), ref.get(name)) < TOL_STATE, name
+        rounds.append((int(st.get("rounds")), int(st.get("fallback"))))
+        seen |= set(ref.get("sel_idx").tolist())
+        targets = dict(M=ref.get("Mhat"), V=ref.get("Vhat"))
+        rec = {}
+        for name in ("M", "V"):
+            lam, x, done = st.get("lam" + name), st.get("x" + name), int(st.get("done" + name))
+            if step in (1, steps):
+                check_recovery(seed, d, k, s, targets[name], lam, x, done, rng)
+            if planted:
+                # exact-recovery regime: M^ and V^ are combinations of the columns kept so far, and OMP finds only those
+                assert set(lam.tolist()) <= seen, "recovered support leaves the kept indices"
+                if step == 1:
+                    assert sorted(lam.tolist()) == ref.get("sel_idx").tolist()
+            rec[name] = (lam[:done], x[:done])
+            if step == 1 and full_oracle_picks:
+                o = oracle.omp(seed, d, k, full_oracle_picks, targets[name])     # full passes over all d columns
+                assert np.array_equal(o["lam"], lam[:full_oracle_picks]), name
+                assert rel(st.get("rnorm" + name)[:full_oracle_picks], o["rnorm"]) < 1e-6
+        # a5: Eq. (8) on the common support where x^V > 0, nothing else touched
+        lamM, xM = rec["M"]
+        lamV, xV = rec["V"]
+        upd = {}
+        for i, col in enumerate(lamM.tolist()):
+            hit = np.nonzero(lamV == col)[0]
+            if hit.size and xV[hit[0]] > 0:
+                upd[col] = hp["lr"] * xM[i] / (np.sqrt(xV[hit[0]]) + hp["eps"])
+        n = int(st.get("n_upd"))
+        assert n == len(upd) and sorted(upd) == st.get("upd_idx")[:n].tolist()
+        want = np.array([upd[c] for c in sorted(upd)])
+        assert rel(st.get("upd_val")[:n], want) < TOL_UPDATE
+        w_after = w_gpu.cpu().numpy()
+        touched = np.zeros(d, dtype=bool)
+        touched[sorted(upd)] = True
+        assert np.array_equal(w_after[~touched], w_before[~touched])
+        dw = w_after[touched].astype(np.float64) - w_before[touched]
+        assert np.abs(dw + want).max() <= TOL_UPDATE * np.abs(want).max() + 1.2e-7 * np.abs(w_before[touched]).max()
+    status = int(st.get("status"))
+    st.close()
+    ref.close()
+    return rounds, status
+
+
+@pytest.fixture(scope="module")
+def sgc():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2502_00311_b200 import binding
+    binding.lib()
+    return binding
+
+
+def test_config2_full_size(sgc):
+    # 4096 x 4096, k = 2048, s = 64, seed 1: the benchmark's workload; exact-recovery regime
+    rounds, status = run_config(sgc, 4096 * 4096, 2048, 64, 1, 2, steps=3, planted=True, full_oracle_picks=1)
+    assert all(fb == 0 for _, fb in rounds), rounds
+    assert rounds[-1][0] == 1, rounds            # warm candidate list: one screening pass per step
+    assert not status & (sgc.STATUS_CANDIDATE_OVERFLOW | sgc.STATUS_SELECT_FALLBACK)
+
+
+@pytest.mark.parametrize("rows,cols", [(4096, 4096), (11008, 4096)])
+def test_config3_shapes_full_size(sgc, rows, cols):
+    # one Llama-2-7B layer: k = 2048, s = 128 per matrix (recovery is inexact here: noise columns get picked)
+    run_config(sgc, rows * cols, 2048, 128, 1, 3, steps=2, planted=False)
+
+
+def test_config4_matrix_full_size(sgc):
+    # the 32-layer stack uses k = 1024, s = 64 for every matrix
+    run_config(sgc, 4096 * 4096, 1024, 64, 1, 4, steps=2, planted=False)
+
+
+@pytest.mark.parametrize("k,s,planted", [(256, 16, False), (4096, 64, True), (16384, 64, True)])
+def test_config5_sweep_points_full_size(sgc, k, s, planted):
+    # 4096 x 11008 matrix at three points of the (k, s) sweep
+    run_config(sgc, 4096 * 11008, k, s, 1, 5, steps=2, planted=planted)
