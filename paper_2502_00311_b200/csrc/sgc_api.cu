@@ -53,6 +53,7 @@ size_t layout(sgc_state* st, unsigned char* base) {
         st->cand_list = carve<uint32_t>(base, off, sgc::kCandCap);
         st->cand_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
         st->rtmp = carve<double>(base, off, k);
+        st->inv_norm = carve<uint16_t>(base, off, (size_t)st->d);
     }
     return off;
 }
@@ -93,8 +94,13 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
         e = cudaMemset(st->base, 0, st->bytes);        // M_0 = V_0 = 0, counters, histogram, empty candidate list
     }
     if (e == cudaSuccess) e = sgc::finish_recover_setup(st);
+    if (e == cudaSuccess) {
+        e = cudaHostAlloc(reinterpret_cast<void**>(&st->h_rounds), sizeof(int), cudaHostAllocMapped);
+        if (e == cudaSuccess) { st->h_rounds[0] = 0; e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st->d_rounds), st->h_rounds, 0); }
+    }
     if (e != cudaSuccess) {
         if (st->base) cudaFree(st->base);
+        if (st->h_rounds) cudaFreeHost(st->h_rounds);
         delete st->ev_pool; delete st->ev_phase;
         delete st;
         return (int)e;
@@ -139,6 +145,7 @@ SGC_API int sgc_destroy(sgc_state* st) {
     cudaError_t e = cudaSuccess;
     if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
     cudaError_t e2 = cudaFree(st->base);
+    if (st->h_rounds) cudaFreeHost(st->h_rounds);
     for (cudaEvent_t ev : *st->ev_pool) cudaEventDestroy(ev);
     delete st->ev_pool; delete st->ev_phase;
     delete st;
@@ -287,7 +294,7 @@ SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uin
     if (e == cudaSuccess) e = cudaMemsetAsync(rep_count, 0, sizeof(uint32_t) * (size_t)n, cs);
     if (e == cudaSuccess) e = cudaMemsetAsync(error_flag, 0, sizeof(int32_t), cs);
     if (e == cudaSuccess)
-        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
+        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
                              nullptr, error_flag, sms, cs);
     return (int)e;
 }

@@ -103,12 +103,12 @@ constexpr int kCorrTop = 2;             // candidates kept per block and residua
 constexpr int kRescoreCap = 16;         // candidates rescored in fp64 per iteration and residual
 constexpr int kBookThreads = 1024;
 constexpr int kOmpThreads = 1024;       // threads per block of the cooperative OMP kernel
-constexpr int kCandCap = 8192;          // candidate columns kept for the restricted (speculative) OMP
-constexpr int kCandKeep = 4096;         // the list is rebuilt from the supports once it grows beyond this
+constexpr int kCandCap = 16384;         // candidate columns kept for the restricted (speculative) OMP
+constexpr int kCandKeep = 12288;        // the list is rebuilt from the supports once it grows beyond this
 constexpr int kSmallList = 768;         // lists up to this length are correlated inside the bookkeeping block
 constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
-constexpr int kMaxRounds = 8;           // speculate / screen / resolve rounds enqueued per step
+constexpr int kMaxRounds = 24;          // speculate / screen / resolve rounds enqueued per step
 constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
 // |score computed by the screening pass - exact score| <= kScreenMargin * ||r|| + kScreenNormMargin * score:
 // the residual is rounded to binary16 (relative error 2^-11 per element, hence at most 2^-11 ||r|| by
@@ -192,6 +192,9 @@ struct sgc_state {
     uint32_t* cand_list;        // [kCandCap]
     unsigned int* cand_bits;    // bitmap over [0, d): membership in cand_list
     double* rtmp;               // [k] scratch residual of the resolve kernel
+    uint16_t* inv_norm;         // [d] 1 / ||Z_i|| as binary16, filled once at creation (the screening pass reads it)
+    int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
+    int* d_rounds;              // device alias of h_rounds
 };
 
 namespace sgc {
@@ -232,6 +235,7 @@ cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: 
 cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
-                        unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error, int sm_count,
-                        cudaStream_t stream);
+                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error,
+                        int sm_count, cudaStream_t stream);
+cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream);
 }  // namespace sgc

@@ -45,6 +45,7 @@ struct PassArgs {
     unsigned int num_super;      // ceil(d / 256)
     const float* tau;            // [n] thresholds (+inf = unused residual), in the units of the (scaled) rows of R^T
     const float* inv_scale;      // [n] factor that turns a score back into the caller's units, or nullptr for 1
+    const uint16_t* inv_norm;    // [d] 1 / ||Z_i|| as binary16 (TABLE variant); otherwise the generators accumulate the norms
     unsigned int* rep_count;     // [n]
     uint2* rep;                  // [n][rep_cap]  (column, score bits)
     int rep_cap;
@@ -154,6 +155,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 //   norms  float[kNormRing][256][2]      partial ||Z_i||^2 of the two generator threads of each column
 //   tau    float[256]
 //   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
+template <bool TABLE>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
     if (a.gate != nullptr && *a.gate == 0) return;
     extern __shared__ unsigned char smem_raw[];
@@ -257,8 +259,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             for (int t = 0; t < 2; ++t) {
                 const int col_local = t * kTileCols + quad * 32 + lane;
                 const unsigned long long col = (unsigned long long)sweep * kSuperCols + col_local;
-                const float n2 = nr[col_local * 2] + nr[col_local * 2 + 1];
-                const float inv = (col < a.d && n2 > 0.0f) ? 1.0f / sqrtf(n2) : 0.0f;
+                float inv = 0.0f;
+                if (TABLE) {
+                    if (col < a.d) inv = half_bits_to_float(a.inv_norm[col]);
+                } else {
+                    const float n2 = nr[col_local * 2] + nr[col_local * 2 + 1];
+                    if (col < a.d && n2 > 0.0f) inv = 1.0f / sqrtf(n2);
+                }
 #pragma unroll 1
                 for (int c0 = 0; c0 < a.n; c0 += 16) {
                     uint32_t v[16];
@@ -308,15 +315,17 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                     for (int e = 0; e < 8; ++e) {
                         w[e] = z_pair_from_word(h);
                         h += key.mk;
-                        n2 = hfma2(w[e], w[e], n2);
+                        if (!TABLE) n2 = hfma2(w[e], w[e], n2);
                     }
                     st_shared_v4(dst + off[c], w[0], w[1], w[2], w[3]);
                     st_shared_v4(dst + off[c + 1], w[4], w[5], w[6], w[7]);
-                    const float2 part = half2_bits_to_float2(n2);
-                    norm += part.x + part.y;
+                    if (!TABLE) {
+                        const float2 part = half2_bits_to_float2(n2);
+                        norm += part.x + part.y;
+                    }
                 }
                 h += skip;
-                if (kc == kc_count - 1) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
+                if (!TABLE && kc == kc_count - 1) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full + 8u * st);
@@ -338,6 +347,26 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
+}
+
+// 1 / ||Z_i|| for every column, once per state: thread = column, fp32 sum of the exact squares
+__global__ void __launch_bounds__(256) k_inv_norms(uint32_t seed_lo, uint32_t seed_hi, unsigned long long d, int k, uint16_t* out) {
+    const unsigned long long col = (unsigned long long)blockIdx.x * 256 + threadIdx.x;
+    if (col >= d) return;
+    const ColKey key = column_key(seed_lo, seed_hi, (uint32_t)col);
+    float n2 = 0.0f;
+    uint32_t h = key.ck;
+#pragma unroll 4
+    for (int row = 0; row < k; row += 2) {
+        const float2 z = half2_bits_to_float2(z_pair_from_word(h));
+        h += key.mk;
+        n2 = __fmaf_rn(z.x, z.x, n2);
+        if (row + 1 < k) n2 = __fmaf_rn(z.y, z.y, n2);
+    }
+    const float inv = n2 > 0.0f ? 1.0f / sqrtf(n2) : 0.0f;
+    unsigned short bits;
+    asm("cvt.rn.f16.f32 %0, %1;" : "=h"(bits) : "f"(inv));
+    out[col] = bits;
 }
 
 // ---- host side --------------------------------------------------------------------------------------------
@@ -387,23 +416,31 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
 
 cudaError_t pass_configure(int n) {
     static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map storage");
-    return cudaFuncSetAttribute(k_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+    cudaError_t e = cudaFuncSetAttribute(k_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+}
+
+cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream) {
+    k_inv_norms<<<(unsigned int)((d + 255) / 256), 256, 0, stream>>>((uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), d, k, out);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
-                        unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error, int sm_count,
-                        cudaStream_t stream) {
+                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error,
+                        int sm_count, cudaStream_t stream) {
     PassArgs a;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
     a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;
     a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
-    a.tau = tau; a.inv_scale = inv_scale; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
+    a.tau = tau; a.inv_scale = inv_scale; a.inv_norm = inv_norm; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
     unsigned int grid = (unsigned int)sm_count;
     if (grid > a.num_super) grid = a.num_super;
     CUtensorMap map;
     memcpy(&map, tmap, sizeof(map));
-    k_pass<<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    if (inv_norm) k_pass<true><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    else k_pass<false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
     return cudaGetLastError();
 }
 

@@ -893,8 +893,11 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate) {
 
 // end of the step: the supports found stay (or become) candidates of the next step
 __global__ void __launch_bounds__(kOmpThreads, 1)
-k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uint32_t* cand_list, unsigned int* cand_bits) {
+k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uint32_t* cand_list, unsigned int* cand_bits,
+              int* rounds_out) {
     __shared__ int n_s;
+    // how many rounds this step took (the enqueued rounds if even they were not enough): sizes the next step's launches
+    if (threadIdx.x == 0) *rounds_out = ctl->fallback ? kMaxRounds : ctl->rounds;
     int n = ctl->n_cand;
     // rebuild from the supports alone when the list has outgrown its bound, or when it holds far more than the
     // supports although a single round confirmed every pick (harvested columns of an earlier cold start)
@@ -1035,8 +1038,8 @@ cudaError_t configure_recover(sgc_state* st) {
     int half = st->s < 128 ? st->s : 128;
     half = (half + 15) / 16 * 16;
     st->pass_n = 2 * half;
-    st->z_harvest = normal_tail_threshold((double)st->d, 256.0);
-    st->z_floor = normal_tail_threshold((double)st->d, 1024.0);
+    st->z_harvest = normal_tail_threshold((double)st->d, 1024.0);
+    st->z_floor = normal_tail_threshold((double)st->d, 1792.0);
     if (st->spec_ok) {
         e = pass_configure(st->pass_n);
         if (e != cudaSuccess) return e;
@@ -1046,7 +1049,11 @@ cudaError_t configure_recover(sgc_state* st) {
 
 cudaError_t finish_recover_setup(sgc_state* st) {
     if (!st->spec_ok) return cudaSuccess;
-    return pass_encode_map(st->tmap, st->rt, st->pass_n, st->k);
+    cudaError_t e = pass_encode_map(st->tmap, st->rt, st->pass_n, st->k);
+    if (e != cudaSuccess) return e;
+    e = launch_inv_norms(st->seed, (uint64_t)st->d, st->k, st->inv_norm, 0);     // column norms: a property of (seed, k)
+    if (e != cudaSuccess) return e;
+    return cudaDeviceSynchronize();
 }
 
 cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches) {
@@ -1062,7 +1069,12 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
         ResolveArgs ra;
         ra.o = a; ra.rep = st->rep; ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list;
         ra.rtmp = st->rtmp;
-        for (int round = 0; round < kMaxRounds && e == cudaSuccess; ++round) {
+        // rounds to enqueue: twice what the last finished step needed plus slack (read from pinned memory without
+        // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
+        const int last = *reinterpret_cast<volatile int*>(st->h_rounds);
+        int n_rounds = last <= 0 ? 8 : 2 * last + 4;
+        if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
+        for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
             {
                 PhaseTimer timer(st, stream, kPhaseCorr, 2);
                 k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
@@ -1071,7 +1083,7 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
             if (e != cudaSuccess) break;
             {
                 PhaseTimer timer(st, stream, kPhasePass, 1);
-                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale, st->rep_count,
+                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale, st->inv_norm, st->rep_count,
                                 st->rep, kRepCap, &st->ctl->round_active, &st->ctl->pass_error, st->sm_count, stream);
             }
             if (e != cudaSuccess) break;
@@ -1095,7 +1107,8 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
                                                   (double)st->alpha, (double)st->eps, (double)st->lr);
         *launches += 1;
         if (speculate) {
-            k_cand_update<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->cnt, st->lam, st->s, st->cand_list, st->cand_bits);
+            k_cand_update<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->cnt, st->lam, st->s, st->cand_list, st->cand_bits,
+                                                         st->d_rounds);
             *launches += 1;
         }
     }
