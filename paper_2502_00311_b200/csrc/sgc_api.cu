@@ -54,6 +54,10 @@ size_t layout(sgc_state* st, unsigned char* base) {
         st->cand_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
         st->rtmp = carve<double>(base, off, k);
         st->inv_norm = carve<uint16_t>(base, off, (size_t)st->d);
+        st->zlist = carve<uint16_t>(base, off, (size_t)sgc::kGramList * k);
+        st->gram = carve<double>(base, off, (size_t)sgc::kGramList * sgc::kGramList);
+        st->p0 = carve<double>(base, off, 2 * (size_t)sgc::kGramList);
+        st->pick_li = carve<int>(base, off, 2 * s);
     }
     return off;
 }

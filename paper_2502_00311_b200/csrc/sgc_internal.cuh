@@ -106,6 +106,7 @@ constexpr int kOmpThreads = 1024;       // threads per block of the cooperative 
 constexpr int kCandCap = 16384;         // candidate columns kept for the restricted (speculative) OMP
 constexpr int kCandKeep = 12288;        // the list is rebuilt from the supports once it grows beyond this
 constexpr int kSmallList = 768;         // lists up to this length are correlated inside the bookkeeping block
+constexpr int kGramList = 256;          // lists up to this length run OMP on their Gram matrix (Algorithm 3 as printed)
 constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
 constexpr int kMaxRounds = 24;          // speculate / screen / resolve rounds enqueued per step
@@ -135,6 +136,11 @@ struct SpecCtl {
     int pass_error;         // a wait inside the screening pass expired
     int stop[2];            // scratch of the cooperative kernel: speculation of residual m has ended
     int list_exact[2];      // 1: the last speculation of residual m compared every list member exactly
+    int list_version;       // bumped whenever the candidate list changes
+    int gram_version;       // list version the stored Gram matrix belongs to
+    int gram_pending;       // list version seen by the round in flight
+    int gram_todo;          // 1: the Gram matrix must be recomputed in this round
+    int gram_ok;            // 0: the Gram path gave up in this step (a pick is missing from the list)
     double ynorm[2];        // ||y|| per residual
 };
 
@@ -193,6 +199,10 @@ struct sgc_state {
     unsigned int* cand_bits;    // bitmap over [0, d): membership in cand_list
     double* rtmp;               // [k] scratch residual of the resolve kernel
     uint16_t* inv_norm;         // [d] 1 / ||Z_i|| as binary16, filled once at creation (the screening pass reads it)
+    uint16_t* zlist;            // [kGramList][k] the candidate columns as binary16 (Gram path)
+    double* gram;               // [kGramList][kGramList] Z_C^T Z_C
+    double* p0;                 // [2][kGramList] Z_C^T y per residual
+    int* pick_li;               // [2][s] list position of every pick (Gram path)
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };

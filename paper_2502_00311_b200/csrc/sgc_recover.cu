@@ -45,6 +45,7 @@ struct OmpArgs {
     Counters* cnt; SpecCtl* ctl;
     uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; double* pick_score;
     const uint32_t* cand_list;
+    uint16_t* zlist; double* gram; double* p0; int* pick_li;     // Gram path
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -606,7 +607,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_spec_small(OmpArgs a) {
     float* rs = reinterpret_cast<float*>(sr);            // the residual of this block's stream, fp32
     volatile SpecCtl* ctl = a.ctl;
     const int n_cand = ctl->n_cand;
-    if (!ctl->round_active || ctl->fallback || n_cand > kSmallList) return;
+    if (!ctl->round_active || ctl->fallback || n_cand > kSmallList || (n_cand <= kGramList && ctl->gram_ok)) return;
     const int m = blockIdx.x, k = a.k, s = a.s;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int c = threadIdx.x; c < a.half_n; c += kOmpThreads) {
@@ -695,6 +696,330 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_spec_small(OmpArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// speculation on a very short candidate list (at most kGramList columns): Algorithm 3 as printed in Appendix B,
+// i.e. on the Gram matrix G = Z_C^T Z_C of the list and the correlations p = Z_C^T r, which it updates without
+// touching the k-dimensional residual.  Four kernels per round:
+//   k_gram_prepare  the list's columns as binary16 (zlist) and p0 = Z_C^T y for both residuals
+//   k_gram_matrix   G, only when the list has changed since G was computed (in a steady state: never)
+//   k_omp_gram      block m: all picks of residual m, O(|C| * j) fp64 work per pick
+//   k_spec_rows     one block per pick: the residual r_j = y - A_Lambda x_j it was made from (binary16 row of
+//                   the screened batch, norm, threshold), and the picked column for the later kernels
+// The records are those of k_omp mode 0 / k_spec_small.  Scores from G differ from scores computed against r_j
+// only by fp64 rounding; should that ever flip a pick, the screening pass reports the better column as a
+// challenger and k_resolve decides with the directly computed scores.
+// ------------------------------------------------------------------------------------------------
+constexpr int kGramThreads = 256;
+
+__device__ __forceinline__ bool gram_round(volatile SpecCtl* ctl) {
+    return ctl->round_active && !ctl->fallback && ctl->gram_ok && ctl->n_cand <= kGramList;
+}
+
+__device__ double block_sum_256(double v, double* red) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = (lane < kGramThreads / 32) ? red[lane] : 0.0;
+    t = warp_sum(t);
+    return t;
+}
+
+__global__ void __launch_bounds__(kGramThreads) k_gram_prepare(OmpArgs a) {
+    volatile SpecCtl* ctl = a.ctl;
+    if (!gram_round(ctl)) return;
+    __shared__ double red[32];
+    const int n = ctl->n_cand, b = blockIdx.x, k = a.k;
+    if (b == 0 && threadIdx.x == 0) {
+        a.ctl->gram_todo = (ctl->gram_version != ctl->list_version) ? 1 : 0;
+        a.ctl->gram_pending = ctl->list_version;
+    }
+    if (b >= n) return;
+    const ColKey key = column_key(a.seed_lo, a.seed_hi, a.cand_list[b]);
+    uint32_t* dst = reinterpret_cast<uint32_t*>(a.zlist + (size_t)b * k);          // k is a multiple of 64 on this path
+    double dm = 0.0, dv = 0.0;
+    for (int p = threadIdx.x; p < (k >> 1); p += kGramThreads) {
+        const uint32_t z2 = z_pair_from_word(key.ck + (uint32_t)p * key.mk);
+        dst[p] = z2;
+        const float2 z = half2_bits_to_float2(z2);
+        dm += (double)z.x * a.y64[2 * p] + (double)z.y * a.y64[2 * p + 1];
+        dv += (double)z.x * a.y64[k + 2 * p] + (double)z.y * a.y64[k + 2 * p + 1];
+    }
+    dm = block_sum_256(dm, red);
+    dv = block_sum_256(dv, red);
+    if (threadIdx.x == 0) { a.p0[b] = dm; a.p0[kGramList + b] = dv; }
+}
+
+__global__ void __launch_bounds__(kGramThreads) k_gram_matrix(OmpArgs a) {
+    volatile SpecCtl* ctl = a.ctl;
+    if (!gram_round(ctl) || !ctl->gram_todo) return;
+    extern __shared__ uint4 colb[];                                   // column b of the list
+    const int n = ctl->n_cand, b = blockIdx.x, k = a.k;
+    if (b >= n) return;
+    const uint4* src = reinterpret_cast<const uint4*>(a.zlist + (size_t)b * k);
+    for (int v = threadIdx.x; v < (k >> 3); v += kGramThreads) colb[v] = src[v];
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c = b + warp; c < n; c += kGramThreads / 32) {
+        const uint4* pc = reinterpret_cast<const uint4*>(a.zlist + (size_t)c * k);
+        double acc = 0.0;
+#pragma unroll 4
+        for (int v = lane; v < (k >> 3); v += 32) {
+            const uint4 x = pc[v], y4 = colb[v];
+            const uint32_t xw[4] = {x.x, x.y, x.z, x.w}, yw[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {                              // products of two binary16 numbers are exact in fp32
+                const float2 fa = half2_bits_to_float2(xw[e]), fb = half2_bits_to_float2(yw[e]);
+                acc += (double)(fa.x * fb.x);
+                acc += (double)(fa.y * fb.y);
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) { a.gram[(size_t)b * kGramList + c] = acc; a.gram[(size_t)c * kGramList + b] = acc; }
+    }
+}
+
+__global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
+    volatile SpecCtl* ctl = a.ctl;
+    if (!gram_round(ctl)) return;
+    __shared__ double red[32];
+    __shared__ double p[kGramList], gdiag[kGramList];
+    __shared__ double xs[kMaxS], gvec[kMaxS], cvec[kMaxS];
+    __shared__ int li[kMaxS];
+    __shared__ unsigned char taken[kGramList];
+    __shared__ int found, best_i, stop, hi_s, extra_s, dep_s;
+    __shared__ double wsc[kGramThreads / 32];
+    __shared__ uint32_t wcol[kGramThreads / 32];
+    __shared__ int widx[kGramThreads / 32];
+    static_assert(kGramThreads == kGramList, "one thread per list member");
+    const int m = blockIdx.x, s = a.s, n = ctl->n_cand, t = threadIdx.x;
+    const int lane = t & 31, warp = t >> 5;
+    if (m == 0 && t == 0 && ctl->gram_todo) a.ctl->gram_version = ctl->gram_pending;   // k_gram_matrix has run
+    for (int c = t; c < a.half_n; c += kGramThreads) {
+        a.rep_count[m * a.half_n + c] = 0u;
+        a.tau[m * a.half_n + c] = __int_as_float(0x7f800000);
+    }
+    if (ctl->finished[m]) return;
+    const int v0 = ctl->v[m];
+    const uint32_t forced0 = ctl->forced[m];
+    const int base = v0 + (forced0 != kNoColumn ? 1 : 0);
+    const double sigma = a.sigma, sig2 = sigma * sigma;
+    const double* G = a.gram;
+    double* F = a.F + (size_t)m * s * s;
+    double* ac = a.acoef + (size_t)m * s;
+    uint32_t* lam = a.lam + (size_t)m * s;
+    const uint32_t my_col = t < n ? a.cand_list[t] : kNoColumn;
+    // list positions of the verified picks (and of the forced one); a missing one sends the step to the direct kernels
+    if (t == 0) { found = 0; stop = 0; hi_s = base; extra_s = 0; dep_s = 0; }
+    taken[t] = 0;
+    __syncthreads();
+    int forced_li = -1;
+    if (t < n) {
+        gdiag[t] = G[(size_t)t * kGramList + t];
+        for (int l = 0; l < v0; ++l) if (lam[l] == my_col) { li[l] = t; taken[t] = 1; atomicAdd(&found, 1); }
+        if (forced0 != kNoColumn && my_col == forced0) { li[v0] = t; atomicAdd(&found, 1); }
+    }
+    __syncthreads();
+    if (found != base) {
+        if (t == 0) a.ctl->gram_ok = 0;
+        return;
+    }
+    if (forced0 != kNoColumn) forced_li = li[v0];
+    for (int i = t; i < v0; i += kGramThreads) {
+        double acc = 0.0;
+        for (int l = i; l < v0; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
+        xs[i] = acc;
+        a.x[(size_t)m * s + i] = acc;
+        a.pick_li[(size_t)m * s + i] = li[i];
+    }
+    __syncthreads();
+    for (int j = v0; j < s; ++j) {
+        const int c = j - base;                                         // -1 for the forced pick
+        if (c >= a.half_n || stop) break;
+        // correlations of the list with the current residual: p = p0 - sigma * G[:, Lambda] x   (G is symmetric)
+        double pi = 0.0;
+        if (t < n) {
+            double acc = 0.0;
+#pragma unroll 8
+            for (int l = 0; l < j; ++l) acc += G[(size_t)li[l] * kGramList + t] * xs[l];
+            pi = a.p0[m * kGramList + t] - sigma * acc;
+            p[t] = pi;
+        }
+        int q;
+        const bool forced = (j == v0) && forced0 != kNoColumn;
+        if (forced) {
+            q = forced_li;
+            __syncthreads();
+        } else {
+            // "Select": argmax of p_i^2 / g_ii over the free list members, lowest column index on ties
+            double sc = (t < n && !taken[t] && gdiag[t] > 0.0) ? pi * pi / gdiag[t] : -1.0;
+            uint32_t col = sc >= 0.0 ? my_col : kNoColumn;
+            int idx = t;
+            for (int o = 16; o > 0; o >>= 1) {
+                const double s2 = __shfl_xor_sync(0xffffffffu, sc, o);
+                const uint32_t c2 = __shfl_xor_sync(0xffffffffu, col, o);
+                const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (s2 > sc || (s2 == sc && c2 < col)) { sc = s2; col = c2; idx = i2; }
+            }
+            __syncthreads();
+            if (lane == 0) { wsc[warp] = sc; wcol[warp] = col; widx[warp] = idx; }
+            __syncthreads();
+            if (t == 0) {
+                double bs = -1.0; uint32_t bc = kNoColumn; int bi = -1;
+                for (int w = 0; w < kGramThreads / 32; ++w)
+                    if (wsc[w] > bs || (wsc[w] == bs && wcol[w] < bc)) { bs = wsc[w]; bc = wcol[w]; bi = widx[w]; }
+                best_i = bs >= 0.0 ? bi : -1;
+            }
+            __syncthreads();
+            q = best_i;
+            if (q < 0) {                                                // every list member is in the support already
+                if (t == 0) { extra_s = 1; stop = 1; }
+                __syncthreads();
+                break;
+            }
+        }
+        const double pq = p[q], gqq = gdiag[q];
+        if (t == 0) {
+            lam[j] = a.cand_list[q];
+            li[j] = q;
+            a.pick_li[(size_t)m * s + j] = q;
+            if (!forced) a.pick_score[(size_t)m * s + j] = fabs(pq) / sqrt(gqq);
+        }
+        // Gram column of the pick restricted to the support, c = F^T g, pivot
+        for (int l = t; l < j; l += kGramThreads) gvec[l] = sig2 * G[(size_t)li[l] * kGramList + q];
+        __syncthreads();
+        double csq = 0.0;
+        for (int i0 = 0; i0 < j; i0 += kGramThreads / 16) {
+            const int i = i0 + (t >> 4), sub = t & 15;
+            double acc = 0.0;
+            if (i < j)
+                for (int l = sub; l <= i; l += 16) acc += F[(size_t)l * s + i] * gvec[l];
+            for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (i < j && sub == 0) { cvec[i] = acc; csq += acc * acc; }
+        }
+        csq = block_sum_256(csq, red);
+        const double gnn = sig2 * gqq, piv = gnn - csq;
+        if (!(piv > 1e-10 * gnn)) {
+            // dependent column: a speculative one is screened and ends the recovery if confirmed; a forced one ends it now
+            if (t == 0) {
+                if (forced) {
+                    a.cnt->stopped[m] = 1;
+                    atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN);
+                    a.cnt->done[m] = j; a.ctl->v[m] = j; a.ctl->finished[m] = 1;
+                } else { dep_s = 1; hi_s = j + 1; }
+                stop = 1;
+            }
+            __syncthreads();
+            break;
+        }
+        const double gamma = 1.0 / sqrt(piv);
+        for (int i0 = 0; i0 < j; i0 += kGramThreads / 16) {
+            const int i = i0 + (t >> 4), sub = t & 15;
+            double acc = 0.0;
+            if (i < j)
+                for (int l = i + sub; l < j; l += 16) acc += F[(size_t)i * s + l] * cvec[l];
+            for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (i < j && sub == 0) F[(size_t)i * s + j] = -gamma * acc;
+        }
+        if (t == 0) F[(size_t)j * s + j] = gamma;
+        const double aj = gamma * sigma * pq;
+        __syncthreads();
+        for (int i = t; i <= j; i += kGramThreads) {
+            const double xo = (i < j) ? xs[i] : 0.0;
+            const double xn = xo + aj * F[(size_t)i * s + j];
+            xs[i] = xn;
+            a.x[(size_t)m * s + i] = xn;
+        }
+        if (t == 0) {
+            ac[j] = aj;
+            taken[q] = 1;
+            hi_s = j + 1;
+            if (forced) { a.cnt->done[m] = j + 1; a.ctl->v[m] = j + 1; }
+        }
+        __syncthreads();
+    }
+    if (t == 0 && !a.ctl->finished[m]) {
+        a.ctl->base[m] = base;
+        a.ctl->hi[m] = hi_s < base ? base : hi_s;
+        a.ctl->extra[m] = extra_s;
+        a.ctl->dep[m] = dep_s;
+        a.ctl->list_exact[m] = 1;
+    }
+}
+
+// block (m, c): the state after j = base + c picks of residual m
+__global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
+    volatile SpecCtl* ctl = a.ctl;
+    if (!gram_round(ctl)) return;
+    __shared__ double red[32];
+    __shared__ double xs[kMaxS];
+    __shared__ int li[kMaxS];
+    const int per = a.half_n + 1;
+    const int m = blockIdx.x / per, c = blockIdx.x % per, k = a.k, s = a.s, t = threadIdx.x;
+    if (ctl->finished[m]) return;
+    const int base = ctl->base[m], hi = ctl->hi[m], extra = ctl->extra[m], dep = ctl->dep[m];
+    const int j = base + c;
+    if (j > hi || (dep && j == hi)) return;               // a dependent pick leaves no new state behind
+    const double* F = a.F + (size_t)m * s * s;
+    const double* ac = a.acoef + (size_t)m * s;
+    const double* y = a.y64 + (size_t)m * k;
+    const int n_coef = j;
+    for (int i = t; i < n_coef; i += kGramThreads) {
+        double acc = 0.0;
+        for (int l = i; l < n_coef; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
+        xs[i] = acc;
+        li[i] = a.pick_li[(size_t)m * s + i];
+    }
+    __syncthreads();
+    // the picked column of pick j, for the kernels that rebuild residuals from the stored columns
+    if (j < hi) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(a.zlist + (size_t)a.pick_li[(size_t)m * s + j] * k);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(a.zsel + ((size_t)m * s + j) * k);
+        for (int pr = t; pr < (k >> 1); pr += kGramThreads) dst[pr] = src[pr];
+    }
+    const bool screened = c < a.half_n && (j < hi || (j == hi && extra));
+    // r_j = y - sigma * Z_Lambda x_j: first its norm, then (for a screened state) the scaled binary16 row
+    double rn2 = 0.0;
+    for (int row = t; row < k; row += kGramThreads) {
+        double acc = 0.0;
+#pragma unroll 8
+        for (int l = 0; l < n_coef; ++l) acc += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
+        const double r1 = y[row] - a.sigma * acc;
+        rn2 += r1 * r1;
+    }
+    rn2 = block_sum_256(rn2, red);
+    const double rn = sqrt(rn2);
+    if (t == 0) {
+        if (j == 0) a.ctl->ynorm[m] = rn;
+        else a.rnorm[(size_t)m * s + j - 1] = rn;            // ||r|| after pick j-1 (verified entries are rewritten with equal values)
+    }
+    if (!screened) return;
+    const int nrow = m * a.half_n + c;
+    const double sc = residual_scale(rn);
+    uint16_t* dst = a.rt + (size_t)nrow * k;
+    for (int row = t; row < k; row += kGramThreads) {
+        double acc = 0.0;
+#pragma unroll 8
+        for (int l = 0; l < n_coef; ++l) acc += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
+        dst[row] = half_rn_bits((y[row] - a.sigma * acc) * sc);
+    }
+    if (t == 0) {
+        a.inv_scale[nrow] = (float)(1.0 / sc);
+        const double unit = rn / sqrt((double)k);
+        double tau;
+        if (j < hi) {
+            const double ps = a.pick_score[(size_t)m * s + j];
+            tau = ps - screen_margin(rn, ps);
+            if (tau > a.z_harvest * unit) tau = a.z_harvest * unit;
+            if (tau < a.z_floor * unit) tau = a.z_floor * unit;
+        } else {
+            tau = a.z_harvest * unit;
+        }
+        a.tau[nrow] = (float)(tau * sc);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // resolve: confirm or refute the speculated picks with the reports of the screening pass
 // ------------------------------------------------------------------------------------------------
 struct ResolveArgs {
@@ -759,7 +1084,7 @@ __device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, u
         else atomicAnd(&ra.cand_bits[col >> 5], ~bit);
     }
     __syncthreads();
-    if (threadIdx.x == 0) ctl->n_cand = sh.n_cand < kCandCap ? sh.n_cand : kCandCap;
+    if (threadIdx.x == 0) { ctl->n_cand = sh.n_cand < kCandCap ? sh.n_cand : kCandCap; ctl->list_version = ctl->list_version + 1; }
     __syncthreads();
 }
 
@@ -888,6 +1213,8 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate) {
         ctl->finished[0] = ctl->finished[1] = 0;
         ctl->stop[0] = ctl->stop[1] = 0;
         ctl->rounds = 0; ctl->pass_error = 0;
+        ctl->gram_ok = 1;
+        if (ctl->list_version == 0) ctl->list_version = 1;      // a fresh state: no Gram matrix yet
     }
 }
 
@@ -921,7 +1248,11 @@ k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uin
         else atomicAnd(&cand_bits[col >> 5], ~bit);
     }
     __syncthreads();
-    if (threadIdx.x == 0) ctl->n_cand = n_s < kCandCap ? n_s : kCandCap;
+    if (threadIdx.x == 0) {
+        const int n_new = n_s < kCandCap ? n_s : kCandCap;
+        if (n_new != ctl->n_cand || n == 0) ctl->list_version = ctl->list_version + 1;     // rebuilt or extended
+        ctl->n_cand = n_new;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1003,6 +1334,7 @@ OmpArgs make_args(const sgc_state* st) {
     a.cnt = st->cnt; a.ctl = st->ctl;
     a.rt = st->rt; a.tau = st->tau; a.inv_scale = st->inv_scale; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
     a.cand_list = st->cand_list;
+    a.zlist = st->zlist; a.gram = st->gram; a.p0 = st->p0; a.pick_li = st->pick_li;
     return a;
 }
 
@@ -1022,6 +1354,8 @@ cudaError_t configure_recover(sgc_state* st) {
     if (e != cudaSuccess) return e;
     int occ = 0;
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_spec_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && (size_t)st->k * 2 > 48 * 1024)
+        e = cudaFuncSetAttribute(k_gram_matrix, cudaFuncAttributeMaxDynamicSharedMemorySize, st->k * 2);
     if (e != cudaSuccess) return e;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_omp, kOmpThreads, smem);
     if (e != cudaSuccess) return e;
@@ -1076,7 +1410,11 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
         if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
         for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
             {
-                PhaseTimer timer(st, stream, kPhaseCorr, 2);
+                PhaseTimer timer(st, stream, kPhaseCorr, 6);
+                k_gram_prepare<<<kGramList, kGramThreads, 0, stream>>>(a);       // very short list: Gram-matrix OMP
+                k_gram_matrix<<<kGramList, kGramThreads, (size_t)st->k * 2, stream>>>(a);
+                k_omp_gram<<<2, kGramThreads, 0, stream>>>(a);
+                k_spec_rows<<<2 * (a.half_n + 1), kGramThreads, 0, stream>>>(a);
                 k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
                 e = launch_omp(st, a, 0, stream);                                // long candidate list
             }
@@ -1091,7 +1429,7 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
                 PhaseTimer timer(st, stream, kPhaseBook, 1);
                 k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
             }
-            *launches += 4;
+            *launches += 8;
         }
         if (e != cudaSuccess) return e;
     }
