@@ -43,7 +43,7 @@ size_t layout(sgc_state* st, unsigned char* base) {
     st->cnt = carve<sgc::Counters>(base, off, 1);
     st->ctl = carve<sgc::SpecCtl>(base, off, 1);
     if (st->spec_ok) {
-        const size_t n = (size_t)st->pass_n;
+        const size_t n = (size_t)sgc::kPassMaxN;          // room for a whole batch of same-A states (sgc_step_group)
         st->rt = carve<uint16_t>(base, off, n * k);
         st->tau = carve<float>(base, off, n);
         st->inv_scale = carve<float>(base, off, n);
@@ -137,11 +137,23 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
         if (((uintptr_t)grads[i] & 15u) || ((uintptr_t)weights[i] & 15u)) return SGC_ERR_ALIGN;
         for (int32_t j = 0; j < i; ++j) if (states[j] == states[i]) return SGC_ERR_GROUP;
     }
-    for (int32_t i = 0; i < n; ++i) {
-        const int rc = sgc_step(states[i], grads[i], weights[i], stream);
-        if (rc != 0) return rc;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    std::vector<int> launches((size_t)n, 0);
+    cudaError_t e = cudaSuccess;
+    for (int32_t i = 0; i < n && e == cudaSuccess; ++i) {           // a1-a3 per state
+        sgc_state* st = states[i];
+        st->t += 1;
+        e = sgc::launch_select(st, grads[i], cs, &launches[i]);
+        if (e == cudaSuccess) e = sgc::launch_project_adam(st, cs, &launches[i]);
     }
-    return SGC_OK;
+    int shared = 0;
+    if (e == cudaSuccess) e = sgc::launch_recover_group(states, weights, n, cs, &shared);   // a4 + a5, passes shared per batch
+    for (int32_t i = 0; i < n; ++i) {
+        sgc_state* st = states[i];
+        st->last_stream = cs; st->has_stream = true; st->stepped = true;
+        st->last_launches = launches[i] + (i == 0 ? shared : 0);     // the shared launches are booked on the first state
+    }
+    return (int)e;
 }
 
 SGC_API int sgc_destroy(sgc_state* st) {
@@ -297,9 +309,12 @@ SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uin
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(rep_count, 0, sizeof(uint32_t) * (size_t)n, cs);
     if (e == cudaSuccess) e = cudaMemsetAsync(error_flag, 0, sizeof(int32_t), cs);
-    if (e == cudaSuccess)
-        e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
-                             nullptr, error_flag, sms, cs);
+    {
+        int* errors[sgc::kPassMaxBatch] = {error_flag};
+        if (e == cudaSuccess)
+            e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
+                                 nullptr, errors, sms, cs);
+    }
     return (int)e;
 }
 

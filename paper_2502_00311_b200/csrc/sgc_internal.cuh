@@ -109,6 +109,7 @@ constexpr int kSmallList = 768;         // lists up to this length are correlate
 constexpr int kGramList = 256;          // lists up to this length run OMP on their Gram matrix (Algorithm 3 as printed)
 constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
+constexpr int kPassMaxBatch = 8;        // states whose residuals one screening pass can serve (kPassMaxN / 32)
 constexpr int kMaxRounds = 24;          // speculate / screen / resolve rounds enqueued per step
 constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
 // |score computed by the screening pass - exact score| <= kScreenMargin * ||r|| + kScreenNormMargin * score:
@@ -168,7 +169,7 @@ struct sgc_state {
     bool spec_ok;               // speculative recovery usable for this (d, k)
     int pass_n;                 // residuals per screening pass (multiple of 32, <= 256); pass_n / 2 per residual stream
     double z_harvest, z_floor;  // thresholds of the screening pass in units of ||r|| / sqrt(k)
-    unsigned char tmap[128];    // CUtensorMap of the residual matrix R^T
+    unsigned char tmap[8][128]; // CUtensorMaps of the residual matrix R^T, one per number of states batched into a pass
     // optional per-kernel timing (sgc_set_profile)
     bool profile;
     std::vector<cudaEvent_t>* ev_pool; size_t ev_used;
@@ -236,6 +237,7 @@ struct PhaseTimer {
 cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches);
 cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launches);
 cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches);
+cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches);
 cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
                            cudaStream_t stream);
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
@@ -245,7 +247,7 @@ cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: 
 cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
-                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error,
-                        int sm_count, cudaStream_t stream);
+                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
+                        int* const* errors, int sm_count, cudaStream_t stream);
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream);
 }  // namespace sgc

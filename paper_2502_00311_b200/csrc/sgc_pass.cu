@@ -49,8 +49,8 @@ struct PassArgs {
     unsigned int* rep_count;     // [n]
     uint2* rep;                  // [n][rep_cap]  (column, score bits)
     int rep_cap;
-    const int* gate;             // optional: the kernel returns at once when *gate == 0
-    int* error;                  // set to 1 when a wait expired
+    const int* gate[kPassMaxBatch];   // optional: the kernel returns at once when every *gate is 0 (one per batched state)
+    int* error[kPassMaxBatch];        // set to 1 when a wait expired (one per batched state)
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------------
@@ -157,7 +157,12 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 //   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
 template <bool TABLE>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
-    if (a.gate != nullptr && *a.gate == 0) return;
+    if (a.gate[0] != nullptr) {
+        bool any = false;
+#pragma unroll
+        for (int q = 0; q < kPassMaxBatch; ++q) any = any || (a.gate[q] != nullptr && *a.gate[q] != 0);
+        if (!any) return;
+    }
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -337,7 +342,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
-        if (threadIdx.x == 0) atomicExch(a.error, 1);
+        if (threadIdx.x == 0)
+            for (int q = 0; q < kPassMaxBatch; ++q) if (a.error[q]) atomicExch(a.error[q], 1);
         // give copies and MMAs still in flight time to land before shared and tensor memory are released
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
@@ -414,11 +420,16 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-cudaError_t pass_configure(int n) {
+cudaError_t pass_configure(int) {
     static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map storage");
-    cudaError_t e = cudaFuncSetAttribute(k_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+    size_t need = 0;                              // one setting that serves every width the kernel is launched with
+    for (int n = 32; n <= kPassMaxN; n += 32) {
+        const size_t b = pass_smem_bytes(n, pass_stages(n));
+        if (b > need) need = b;
+    }
+    cudaError_t e = cudaFuncSetAttribute(k_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pass_smem_bytes(n, pass_stages(n)));
+    return cudaFuncSetAttribute(k_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
 }
 
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream) {
@@ -427,14 +438,15 @@ cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cu
 }
 
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
-                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* gate, int* error,
-                        int sm_count, cudaStream_t stream) {
+                        const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
+                        int* const* errors, int sm_count, cudaStream_t stream) {
     PassArgs a;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
     a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;
     a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
-    a.tau = tau; a.inv_scale = inv_scale; a.inv_norm = inv_norm; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap; a.gate = gate; a.error = error;
+    a.tau = tau; a.inv_scale = inv_scale; a.inv_norm = inv_norm; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap;
+    for (int q = 0; q < kPassMaxBatch; ++q) { a.gate[q] = gates ? gates[q] : nullptr; a.error[q] = errors ? errors[q] : nullptr; }
     unsigned int grid = (unsigned int)sm_count;
     if (grid > a.num_super) grid = a.num_super;
     CUtensorMap map;

@@ -1375,7 +1375,7 @@ cudaError_t configure_recover(sgc_state* st) {
     st->z_harvest = normal_tail_threshold((double)st->d, 1024.0);
     st->z_floor = normal_tail_threshold((double)st->d, 1792.0);
     if (st->spec_ok) {
-        e = pass_configure(st->pass_n);
+        e = pass_configure(kPassMaxN);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
@@ -1383,65 +1383,105 @@ cudaError_t configure_recover(sgc_state* st) {
 
 cudaError_t finish_recover_setup(sgc_state* st) {
     if (!st->spec_ok) return cudaSuccess;
-    cudaError_t e = pass_encode_map(st->tmap, st->rt, st->pass_n, st->k);
+    cudaError_t e = cudaSuccess;
+    for (int g = 1; g <= kPassMaxN / st->pass_n && e == cudaSuccess; ++g)      // one map per number of states in a batch
+        e = pass_encode_map(st->tmap[g - 1], st->rt, g * st->pass_n, st->k);
     if (e != cudaSuccess) return e;
     e = launch_inv_norms(st->seed, (uint64_t)st->d, st->k, st->inv_norm, 0);     // column norms: a property of (seed, k)
     if (e != cudaSuccess) return e;
     return cudaDeviceSynchronize();
 }
 
-cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches) {
-    const OmpArgs a = make_args(st);
-    const bool speculate = st->spec_ok && (st->mode == 2 || (st->mode == 0 && st->d >= (1ll << 16)));
+// Recovery (a4 + a5) of n states that share (d, k, s, seed), hence A.  The states' screened residuals are laid out side by
+// side in the screening buffers of the first state of each batch (a batch = as many states as fit kPassMaxN columns), so
+// one pass over A serves a whole batch; everything else runs per state.  n = 1 is the plain sgc_step.
+cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches) {
+    sgc_state* st0 = sts[0];
+    bool speculate = true;
+    for (int i = 0; i < n; ++i)
+        speculate = speculate && sts[i]->spec_ok && (sts[i]->mode == 2 || (sts[i]->mode == 0 && sts[i]->d >= (1ll << 16)));
+    const int per_batch = speculate ? kPassMaxN / st0->pass_n : 1;
+    std::vector<OmpArgs> args((size_t)n);
     cudaError_t e = cudaSuccess;
-    {
-        PhaseTimer timer(st, stream, kPhaseBook, 1);
-        k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0);
-        *launches += 1;
-    }
-    if (speculate) {
-        ResolveArgs ra;
-        ra.o = a; ra.rep = st->rep; ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list;
-        ra.rtmp = st->rtmp;
+    int n_rounds = 0;
+    for (int i = 0; i < n; ++i) {
+        sgc_state* st = sts[i];
+        sgc_state* lead = sts[i - i % per_batch];
+        const int slot = i % per_batch;
+        OmpArgs a = make_args(st);
+        // this state's slice of the batch's screening buffers
+        a.rt = lead->rt + (size_t)slot * st->pass_n * st->k;
+        a.tau = lead->tau + slot * st->pass_n;
+        a.inv_scale = lead->inv_scale + slot * st->pass_n;
+        a.rep_count = lead->rep_count + slot * st->pass_n;
+        args[i] = a;
+        {
+            PhaseTimer timer(st, stream, kPhaseBook, 1);
+            k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0);
+            *launches += 1;
+        }
         // rounds to enqueue: twice what the last finished step needed plus slack (read from pinned memory without
         // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
-        const int last = *reinterpret_cast<volatile int*>(st->h_rounds);
-        int n_rounds = last <= 0 ? 8 : 2 * last + 4;
-        if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
+        const int last = speculate ? *reinterpret_cast<volatile int*>(st->h_rounds) : 0;
+        const int want = last <= 0 ? 8 : 2 * last + 4;
+        if (want > n_rounds) n_rounds = want;
+    }
+    if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
+    if (speculate) {
         for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
-            {
-                PhaseTimer timer(st, stream, kPhaseCorr, 6);
-                k_gram_prepare<<<kGramList, kGramThreads, 0, stream>>>(a);       // very short list: Gram-matrix OMP
-                k_gram_matrix<<<kGramList, kGramThreads, (size_t)st->k * 2, stream>>>(a);
-                k_omp_gram<<<2, kGramThreads, 0, stream>>>(a);
-                k_spec_rows<<<2 * (a.half_n + 1), kGramThreads, 0, stream>>>(a);
-                k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
-                e = launch_omp(st, a, 0, stream);                                // long candidate list
+            for (int b0 = 0; b0 < n && e == cudaSuccess; b0 += per_batch) {
+                const int nb = n - b0 < per_batch ? n - b0 : per_batch;
+                for (int i = b0; i < b0 + nb && e == cudaSuccess; ++i) {
+                    sgc_state* st = sts[i];
+                    const OmpArgs& a = args[i];
+                    PhaseTimer timer(st, stream, kPhaseCorr, 6);
+                    k_gram_prepare<<<kGramList, kGramThreads, 0, stream>>>(a);       // very short list: Gram-matrix OMP
+                    k_gram_matrix<<<kGramList, kGramThreads, (size_t)st->k * 2, stream>>>(a);
+                    k_omp_gram<<<2, kGramThreads, 0, stream>>>(a);
+                    k_spec_rows<<<2 * (a.half_n + 1), kGramThreads, 0, stream>>>(a);
+                    k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
+                    e = launch_omp(st, a, 0, stream);                                // long candidate list
+                    *launches += 6;
+                }
+                if (e != cudaSuccess) break;
+                sgc_state* lead = sts[b0];
+                {
+                    PhaseTimer timer(lead, stream, kPhasePass, 1);
+                    const int* gates[kPassMaxBatch];
+                    int* errors[kPassMaxBatch];
+                    for (int q = 0; q < kPassMaxBatch; ++q) {
+                        gates[q] = q < nb ? &sts[b0 + q]->ctl->round_active : nullptr;
+                        errors[q] = q < nb ? &sts[b0 + q]->ctl->pass_error : nullptr;
+                    }
+                    e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
+                                    lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
+                                    lead->sm_count, stream);
+                    *launches += 1;
+                }
+                for (int i = b0; i < b0 + nb && e == cudaSuccess; ++i) {
+                    sgc_state* st = sts[i];
+                    ResolveArgs ra;
+                    ra.o = args[i];
+                    ra.rep = lead->rep + (size_t)(i - b0) * st->pass_n * kRepCap;
+                    ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list; ra.rtmp = st->rtmp;
+                    PhaseTimer timer(st, stream, kPhaseBook, 1);
+                    k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
+                    *launches += 1;
+                }
             }
-            if (e != cudaSuccess) break;
-            {
-                PhaseTimer timer(st, stream, kPhasePass, 1);
-                e = launch_pass(st->tmap, st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale, st->inv_norm, st->rep_count,
-                                st->rep, kRepCap, &st->ctl->round_active, &st->ctl->pass_error, st->sm_count, stream);
-            }
-            if (e != cudaSuccess) break;
-            {
-                PhaseTimer timer(st, stream, kPhaseBook, 1);
-                k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
-            }
-            *launches += 8;
         }
         if (e != cudaSuccess) return e;
     }
-    {
-        PhaseTimer timer(st, stream, kPhaseCorr, 1);
-        e = launch_omp(st, a, 1, stream);
-        *launches += 1;
-    }
-    if (e != cudaSuccess) return e;
-    {
+    for (int i = 0; i < n; ++i) {
+        sgc_state* st = sts[i];
+        {
+            PhaseTimer timer(st, stream, kPhaseCorr, 1);
+            e = launch_omp(st, args[i], 1, stream);
+            *launches += 1;
+        }
+        if (e != cudaSuccess) return e;
         PhaseTimer timer(st, stream, kPhaseScatter, 1);
-        k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weight, st->upd_idx, st->upd_val,
+        k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weights[i], st->upd_idx, st->upd_val,
                                                   (double)st->alpha, (double)st->eps, (double)st->lr);
         *launches += 1;
         if (speculate) {
@@ -1451,6 +1491,10 @@ cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, in
         }
     }
     return cudaGetLastError();
+}
+
+cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches) {
+    return launch_recover_group(&st, &weight, 1, stream, launches);
 }
 
 }  // namespace sgc

@@ -296,6 +296,34 @@ def test_group_equals_independent_steps(sgc):
         st.close()
 
 
+@pytest.mark.parametrize("d,k,s,n", [(300_000, 512, 64, 3), (200_000, 256, 8, 5), (150_000, 2048, 128, 2)])
+def test_group_shares_screening_passes_and_equals_independent_steps(sgc, d, k, s, n):
+    # speculative recovery: the residuals of several same-A states are screened by one tensor-core pass per batch
+    # (two states at s = 64, up to eight at s <= 16, one at s = 128); supports and weights must equal independent steps
+    hp = inputs.ADAM
+    solo = [sgc.Sgc(d, k, s, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(n)]
+    grp = [sgc.Sgc(d, k, s, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(n)]
+    for st in solo + grp:
+        st.set_mode(sgc.MODE_SPECULATIVE)
+    ws = [cuda(inputs.weights(d, 10 + i)) for i in range(n)]
+    wg = [w.clone() for w in ws]
+    supports = [inputs.planted_support(d, s, 50 + i) for i in range(n)]
+    for step in range(3):
+        gr = [cuda(inputs.gradient(d, "student", supports[i][0], supports[i][1], 1000 * i + step)) for i in range(n)]
+        for i in range(n):
+            solo[i].step(gr[i], ws[i])
+        sgc.step_group(grp, gr, wg)
+        for i in range(n):
+            assert grp[i].get("fallback") == 0
+            for name in ("sel_idx", "lamM", "lamV", "upd_idx"):
+                assert np.array_equal(solo[i].get(name), grp[i].get(name)), (name, i, step)
+            assert rel(grp[i].get("xM"), solo[i].get("xM")) < 1e-9
+            assert np.array_equal(ws[i].cpu().numpy(), wg[i].cpu().numpy())
+            assert grp[i].get("t") == step + 1
+    for st in solo + grp:
+        st.close()
+
+
 def test_step_rejects_misaligned_pointers(sgc):
     import torch
     st = sgc.Sgc(1000, 16, 2, 0, 1e-3, 0.9, 0.999, 1e-8)
