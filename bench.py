@@ -256,7 +256,9 @@ def run_ours(args, wl):
             pass_avg_s = pass_ms / working * 1e-3
             achieved = 2.0 * k * d * n_pass / pass_avg_s / 1e12
             roof = {"kernel": "k_pass", "bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / pk["bf16_tflops"], "traffic": None, "peak_source": pk["source"],
+                    "frac": achieved / pk["bf16_tflops"], "traffic": 2.0 * d + 0.56e6, "peak_source": pk["source"],
+                    "traffic_note": "DRAM bytes per launch: 2 bytes per column of the 1/norm table plus R^T (0.56 MB); ncu "
+                                    "measured 4.75 MB at d = 2^21 (profiles/k_pass_small_2M_k2048_s64.md), scaled by d",
                     "note": "2*k*d*N flops per pass (N = %d residuals, f16 x f16 -> fp32 on tcgen05); the operand A is "
                             "regenerated by the CUDA cores (k*d entries per pass), which is what limits the pass" % n_pass,
                     "avg_launch_ms": pass_avg_s * 1e3, "launches": sum(rounds),
