@@ -134,6 +134,13 @@ SGC_API int sgc_destroy(sgc_state* st);
 /* alpha of Eq. (8) ("a scaling factor"); must be finite. */
 SGC_API int sgc_set_alpha(sgc_state* st, float alpha);
 
+/* SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): replaces the measurement matrix by the one that new_seed
+ * names and re-aligns the optimizer state with it, M <- A' OMP_A(M), V <- A' OMP_A(V).  Call it after the sgc_step of
+ * an iteration t with t mod T = 0: the recoveries of that step are reused, since OMP_A(M) = (1 - beta1^t) OMP_A(M^)
+ * (OMP is scale-equivariant; the paper itself notes that the results of the first call can be kept).  From the next
+ * step on, p, q and both recoveries use A'.  Enqueued on stream; SGC_ERR_NOSTEP before the first step. */
+SGC_API int sgc_reproject(sgc_state* st, uint64_t new_seed, void* stream);
+
 /* Chooses the recovery strategy (SGC_MODE_*).  Both strategies return the picks of Algorithm 3 (Appendix B):
  * the speculative one runs OMP on a short candidate list and then proves, with one tensor-core pass over all
  * d columns against the residuals of all iterations at once, that no other column would have been picked; a

@@ -73,6 +73,8 @@ def lib():
                 getattr(L, name).argtypes = [C.c_void_p, f32p]
             L.orc_step_recover.restype = None
             L.orc_step_recover.argtypes = [C.c_void_p, f32p]
+            L.orc_reproject.restype = None
+            L.orc_reproject.argtypes = [C.c_void_p, C.c_uint64]
             L.orc_step.restype = None
             L.orc_step.argtypes = [C.c_void_p, f32p, f32p]
             L.orc_get.restype = C.c_int32
@@ -214,6 +216,10 @@ class Oracle:
     def step(self, grad, weight):
         self.step_compress(grad)
         self.step_recover(weight)
+
+    def reproject(self, new_seed):
+        """SGCA (Algorithm 4, lines 9-12): M <- A' OMP_A(M), V <- A' OMP_A(V), A <- A' with A' named by new_seed."""
+        lib().orc_reproject(self._h, C.c_uint64(new_seed))
 
     def get(self, name):
         what, dt, dim = _GET[name]

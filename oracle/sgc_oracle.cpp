@@ -427,6 +427,31 @@ void orc_step(orc_state* st, const float* grad, float* weight) {
     orc_step_recover(st, weight);
 }
 
+// SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): with a new matrix A' (here: a new seed),
+//   M <- A' OMP_A(M),  V <- A' OMP_A(V),  A <- A'.
+// Reading: M and V are the stored moments (bias correction yields temporaries, as everywhere in this oracle); both
+// recoveries are run afresh on them with the old A, s iterations each, and the s-sparse results are projected with A'.
+void orc_reproject(orc_state* st, uint64_t new_seed) {
+    const int32_t k = st->k, s = st->s;
+    std::vector<double> y((size_t)k), x((size_t)s), t1((size_t)s), t2((size_t)s), rn((size_t)s), out((size_t)k), unused((size_t)k);
+    std::vector<uint32_t> lam((size_t)s);
+    std::vector<float> val((size_t)s);
+    for (int pass = 0; pass < 2; ++pass) {
+        std::vector<float>& state = pass == 0 ? st->M : st->V;
+        for (int32_t j = 0; j < k; ++j) y[j] = (double)state[j];
+        const int32_t done = orc_omp(st->seed, st->d, k, s, y.data(), lam.data(), x.data(), t1.data(), t2.data(), rn.data());
+        // A' x with x supported on the recovered columns: sum in fp64 in the order of selection
+        for (int32_t j = 0; j < k; ++j) out[j] = 0.0;
+        const double sigma = (double)sigma_of_k(k);
+        for (int32_t l = 0; l < done; ++l) {
+            const uint32_t ck = column_key(new_seed, lam[l]);
+            for (int32_t j = 0; j < k; ++j) out[j] += a_entry(ck, (uint32_t)j, sigma) * x[l];
+        }
+        for (int32_t j = 0; j < k; ++j) state[j] = (float)out[j];
+    }
+    st->seed = new_seed;
+}
+
 // Read-back of the last step's records.  what: see the Python binding for the list.
 int32_t orc_get(orc_state* st, int32_t what, void* dst, int64_t bytes) {
     const void* src = nullptr; int64_t n = 0;

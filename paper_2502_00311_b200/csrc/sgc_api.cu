@@ -175,6 +175,17 @@ SGC_API int sgc_set_alpha(sgc_state* st, float alpha) {
     return SGC_OK;
 }
 
+SGC_API int sgc_reproject(sgc_state* st, uint64_t new_seed, void* stream) {
+    if (!st) return SGC_ERR_NULL;
+    if (!st->stepped) return SGC_ERR_NOSTEP;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    cudaError_t e = sgc::launch_reproject(st, new_seed, cs);
+    st->seed = new_seed;
+    if (e == cudaSuccess && st->spec_ok) e = sgc::launch_inv_norms(new_seed, (uint64_t)st->d, st->k, st->inv_norm, cs);
+    st->last_stream = cs; st->has_stream = true;
+    return (int)e;
+}
+
 SGC_API int sgc_set_mode(sgc_state* st, int32_t mode) {
     if (!st) return SGC_ERR_NULL;
     if (mode < SGC_MODE_AUTO || mode > SGC_MODE_SPECULATIVE) return SGC_ERR_WHAT;

@@ -237,6 +237,7 @@ struct PhaseTimer {
 cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches);
 cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launches);
 cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches);
+cudaError_t launch_reproject(sgc_state* st, uint64_t new_seed, cudaStream_t stream);
 cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches);
 cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
                            cudaStream_t stream);

@@ -48,6 +48,33 @@ k_project_adam(uint32_t seed_lo, uint32_t seed_hi, int k, int s, const uint32_t*
     r32[row] = make_float2((float)mh, (float)vh);
 }
 
+// SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): M <- A' OMP_A(M), V <- A' OMP_A(V) for a new matrix A'.
+// OMP is scale-equivariant, OMP_A(M) = (1 - beta1^t) OMP_A(M^), so the recoveries of the step that has just run are
+// reused (the paper notes that the results of the first call can be stored): row j of the new state is
+// c * sum_l A'[j][lambda_l] x_l over the recovered support, summed in fp64 in the order of selection.
+__global__ void __launch_bounds__(kProjThreads)
+k_reproject(uint32_t seed_lo, uint32_t seed_hi, int k, int s, const uint32_t* __restrict__ lam, const double* __restrict__ x,
+            const Counters* __restrict__ cnt, float* __restrict__ M, float* __restrict__ V, double sigma, double c1, double c2,
+            SpecCtl* ctl) {
+    extern __shared__ unsigned char smem_raw[];
+    ColKey* keys = reinterpret_cast<ColKey*>(smem_raw);
+    double* xs = reinterpret_cast<double*>(keys + 2 * s);
+    const int done[2] = {cnt->done[0], cnt->done[1]};
+    for (int i = threadIdx.x; i < 2 * s; i += kProjThreads) {
+        const int m = i / s, l = i % s;
+        if (l < done[m]) { keys[i] = column_key(seed_lo, seed_hi, lam[i]); xs[i] = x[i]; }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) ctl->list_version = ctl->list_version + 1;   // Gram matrix of the old A is void
+    __syncthreads();
+    const int row = blockIdx.x * kProjThreads + threadIdx.x;
+    if (row >= k) return;
+    for (int m = 0; m < 2; ++m) {
+        double acc = 0.0;
+        for (int l = 0; l < done[m]; ++l) acc = acc + sigma * (double)z_at(keys[m * s + l], (uint32_t)row) * xs[m * s + l];
+        if (m == 0) M[row] = (float)(c1 * acc); else V[row] = (float)(c2 * acc);
+    }
+}
+
 __global__ void k_z_block(uint32_t seed_lo, uint32_t seed_hi, long long row0, long long nrows, long long col0,
                           long long ncols, float* __restrict__ out) {
     const long long n = nrows * ncols;
@@ -71,6 +98,17 @@ cudaError_t launch_project_adam(sgc_state* st, cudaStream_t stream, int* launche
                                                          st->k, st->s, st->sel_idx, st->sel_val, st->M, st->V, st->p,
                                                          st->q, st->y64, st->r64, st->r32, st->cnt, sigma, b1, b2, c1, c2);
     *launches += 1;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reproject(sgc_state* st, uint64_t new_seed, cudaStream_t stream) {
+    const double b1 = (double)st->beta1, b2 = (double)st->beta2;
+    const double c1 = 1.0 - pow(b1, (double)st->t), c2 = 1.0 - pow(b2, (double)st->t);
+    const double sigma = (double)(float)(1.0 / sqrt((double)st->k));
+    const int grid = (st->k + kProjThreads - 1) / kProjThreads;
+    const size_t smem = 2 * (size_t)st->s * (sizeof(ColKey) + sizeof(double));
+    k_reproject<<<grid, kProjThreads, smem, stream>>>((uint32_t)(new_seed & 0xFFFFFFFFu), (uint32_t)(new_seed >> 32), st->k, st->s,
+                                                      st->lam, st->x, st->cnt, st->M, st->V, sigma, c1, c2, st->ctl);
     return cudaGetLastError();
 }
 

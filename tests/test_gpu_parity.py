@@ -324,6 +324,38 @@ def test_group_shares_screening_passes_and_equals_independent_steps(sgc, d, k, s
         st.close()
 
 
+@pytest.mark.parametrize("mode", [1, 2])
+def test_sgca_reprojection_matches_the_oracle(sgc, mode):
+    # Algorithm 4: every T = 2 steps the matrix is replaced and M, V are re-aligned; the steps after that run under the
+    # new matrix on both sides (the oracle recovers the stored moments afresh, the GPU rescales the step's recoveries)
+    d, k, s = 120_000, 512, 12
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, 21, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    st.set_mode(mode)
+    ref = oracle.Oracle(d, k, s, 21, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    supp, sign = inputs.planted_support(d, s, 31)
+    w_gpu, w_ref = cuda(inputs.weights(d, 4)), inputs.weights(d, 4)
+    for step in range(1, 7):
+        g = inputs.gradient(d, "student", supp, sign, 500 + step)
+        st.step(cuda(g), w_gpu)
+        ref.step(g, w_ref)
+        assert np.array_equal(st.get("lamM"), ref.get("lamM")) and np.array_equal(st.get("lamV"), ref.get("lamV")), step
+        assert rel(st.get("p"), ref.get("p")) < TOL_STATE
+        if step % 2 == 0:
+            new_seed = 1000 + step
+            st.reproject(new_seed)
+            ref.reproject(new_seed)
+        assert rel(st.get("M"), ref.get("M")) < TOL_STATE and rel(st.get("V"), ref.get("V")) < TOL_STATE, step
+        assert rel(w_gpu.cpu().numpy(), w_ref) < 1e-6
+    st.close()
+    ref.close()
+    fresh = sgc.Sgc(1000, 64, 2, 0, 1e-3, 0.9, 0.999, 1e-8)
+    with pytest.raises(sgc.SgcError) as e:
+        fresh.reproject(5)
+    assert e.value.code == -8
+    fresh.close()
+
+
 def test_step_rejects_misaligned_pointers(sgc):
     import torch
     st = sgc.Sgc(1000, 16, 2, 0, 1e-3, 0.9, 0.999, 1e-8)

@@ -126,3 +126,32 @@ def test_combine_scatter_definition_and_guards():
     want[2] -= uv[0]
     want[7] -= uv[1]
     assert np.array_equal(W, want.astype(np.float32))
+
+
+# ---- SGCA re-projection (Appendix C, Algorithm 4, lines 9-12) ------------------------------------------------
+def test_reprojection_moves_an_exactly_sparse_state_to_the_new_matrix():
+    # constant sparse gradient: M_t = (1 - b1^t) A g and V_t = (1 - b2^t) A g^2 exactly (closed form of the EMA), so
+    # OMP recovers (1 - b^t) g and the re-projected states must be (1 - b^t) A' g, A' materialised with numpy
+    d, k, s, seed, new_seed = 3000, 256, 6, 3, 0xABCDEF0123
+    rng = np.random.default_rng(5)
+    supp = np.sort(rng.choice(d, size=s, replace=False)).astype(np.uint32)
+    g = np.zeros(d, dtype=np.float32)
+    g[supp] = (rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
+    o = oracle.Oracle(d, k, s, seed, 1e-3, 0.9, 0.999, 1e-8)
+    w = np.zeros(d, dtype=np.float32)
+    steps = 3
+    for _ in range(steps):
+        o.step(g, w)
+    o.reproject(new_seed)
+    Anew = oracle.z_block(new_seed, 0, k, 0, d).astype(np.float64) * float(oracle.sigma(k))
+    gd = g.astype(np.float64)
+    b1, b2 = float(np.float32(0.9)), float(np.float32(0.999))          # the betas are fp32 numbers
+    np.testing.assert_allclose(o.get("M"), (1 - b1 ** steps) * (Anew @ gd), rtol=0, atol=2e-6 * np.abs(Anew @ gd).max())
+    np.testing.assert_allclose(o.get("V"), (1 - b2 ** steps) * (Anew @ (gd * gd)), rtol=0,
+                               atol=2e-6 * (1 - b2 ** steps) * np.abs(Anew @ (gd * gd)).max())
+    # the method carries on under the new matrix: same support, same update direction
+    w2 = np.zeros(d, dtype=np.float32)
+    o.step(g, w2)
+    assert sorted(o.get("lamM").tolist()) == supp.tolist() == sorted(o.get("lamV").tolist())
+    np.testing.assert_allclose(w2[supp], -1e-3 * np.sign(g[supp]), rtol=0, atol=2e-8)
+    o.close()
