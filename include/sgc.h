@@ -128,6 +128,13 @@ SGC_API int sgc_step(sgc_state* st, const float* grad, float* weight, void* stre
 SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, float* const* weights, int32_t n,
                    void* stream);
 
+/* Memory-efficient SGC (MESGC, Section 4.4 "Efficient SGC"): the gradient is split into c equal chunks, SGC with
+ * s_c = s / c entries runs on every chunk, and all chunks share one small matrix A (k x d/c).  The caller creates c
+ * states with sgc_create(d / c, k, s_c, seed, ...) -- the same seed, hence the same A -- and passes the whole vectors:
+ *   grad, weight   device pointers, c * (d / c) floats; chunk i occupies [i * d/c, (i + 1) * d/c)
+ * d / c must be a multiple of 4 (16-byte aligned chunks).  Equivalent to sgc_step_group on the c chunk pointers. */
+SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* grad, float* weight, void* stream);
+
 /* Waits for the state's last enqueued work, then frees everything.  NULL is accepted. */
 SGC_API int sgc_destroy(sgc_state* st);
 

@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
 _lib = None
 
-EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
+EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
            "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
            "sgc_set_mode", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version"]
 
@@ -58,6 +58,8 @@ def lib():
         L.sgc_step.argtypes = [vp, vp, vp, vp]
         L.sgc_step_group.restype = C.c_int
         L.sgc_step_group.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int32, vp]
+        L.sgc_step_chunked.restype = C.c_int
+        L.sgc_step_chunked.argtypes = [C.POINTER(vp), C.c_int32, vp, vp, vp]
         L.sgc_destroy.restype = C.c_int
         L.sgc_destroy.argtypes = [vp]
         L.sgc_set_alpha.restype = C.c_int
@@ -236,6 +238,26 @@ class Sgc:
             self.close()
         except Exception:
             pass
+
+
+class Mesgc:
+    """Memory-efficient SGC (Section 4.4): c chunks of one flat vector, each with its own optimizer state and
+    s_c entries per step, all sharing the matrix A (k x d/c) named by one seed (sgc_step_chunked)."""
+
+    def __init__(self, d, c, k, s_c, seed, lr, beta1, beta2, eps, alpha=None):
+        if d % c:
+            raise ValueError("d must be a multiple of the number of chunks")
+        self.d, self.c = int(d), int(c)
+        self.chunks = [Sgc(d // c, k, s_c, seed, lr, beta1, beta2, eps, alpha=alpha) for _ in range(c)]
+
+    def step(self, grad, weight, stream=None):
+        hs = (C.c_void_p * self.c)(*[st._h for st in self.chunks])
+        _check(lib().sgc_step_chunked(hs, self.c, _dev_ptr(grad, self.d, "grad"), _dev_ptr(weight, self.d, "weight"),
+                                      _stream_ptr(stream)), "sgc_step_chunked")
+
+    def close(self):
+        for st in self.chunks:
+            st.close()
 
 
 def step_group(states, grads, weights, stream=None):

@@ -156,6 +156,18 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
     return (int)e;
 }
 
+SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* grad, float* weight, void* stream) {
+    if (!states || !grad || !weight) return SGC_ERR_NULL;
+    if (c < 1) return SGC_ERR_DIM;
+    if (!states[0]) return SGC_ERR_NULL;
+    const int64_t dc = states[0]->d;
+    if ((dc * 4) % 16 != 0 && c > 1) return SGC_ERR_ALIGN;          // every chunk must start on a 16-byte boundary
+    std::vector<const float*> gs((size_t)c);
+    std::vector<float*> ws((size_t)c);
+    for (int32_t i = 0; i < c; ++i) { gs[i] = grad + (size_t)i * dc; ws[i] = weight + (size_t)i * dc; }
+    return sgc_step_group(states, gs.data(), ws.data(), c, stream);
+}
+
 SGC_API int sgc_destroy(sgc_state* st) {
     if (!st) return SGC_OK;
     cudaError_t e = cudaSuccess;

@@ -324,6 +324,39 @@ def test_group_shares_screening_passes_and_equals_independent_steps(sgc, d, k, s
         st.close()
 
 
+def test_mesgc_chunks_share_one_matrix_and_match_independent_oracles(sgc):
+    # Section 4.4: c chunks, s_c entries each, one A of size k x d/c; every chunk is an SGC problem of its own
+    c, dc, k, sc = 6, 70_000, 256, 4
+    d = c * dc
+    hp = inputs.ADAM
+    m = sgc.Mesgc(d, c, k, sc, 8, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    for st in m.chunks:
+        st.set_mode(sgc.MODE_SPECULATIVE)
+    refs = [oracle.Oracle(dc, k, sc, 8, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(c)]
+    supp, sign = inputs.planted_support(d, c * sc, 17)
+    w0 = inputs.weights(d, 2)
+    w_gpu, w_ref = cuda(w0.copy()), w0.copy()
+    for step in range(1, 4):
+        g = inputs.gradient(d, "student", supp, sign, 40 + step)
+        m.step(cuda(g), w_gpu)
+        for i in range(c):
+            refs[i].step(g[i * dc:(i + 1) * dc], w_ref[i * dc:(i + 1) * dc])
+            for name in ("sel_idx", "lamM", "lamV"):
+                assert np.array_equal(m.chunks[i].get(name), refs[i].get(name)), (name, i, step)
+            assert rel(m.chunks[i].get("M"), refs[i].get("M")) < TOL_STATE
+        wg = w_gpu.cpu().numpy()
+        changed = wg != w0
+        assert np.array_equal(changed, w_ref != w0)
+        assert np.abs(wg[changed].astype(np.float64) - w_ref[changed]).max() <= TOL_UPDATE * np.abs(w_ref[changed] - w0[changed]).max() + 2e-9
+    with pytest.raises(sgc.SgcError):
+        odd = sgc.Mesgc(6 * 1002, 6, 64, 2, 0, 1e-3, 0.9, 0.999, 1e-8)       # chunks of 1002 floats are not 16-byte aligned
+        import torch
+        odd.step(torch.zeros(6 * 1002, device="cuda"), torch.zeros(6 * 1002, device="cuda"))
+    m.close()
+    for r in refs:
+        r.close()
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 def test_sgca_reprojection_matches_the_oracle(sgc, mode):
     # Algorithm 4: every T = 2 steps the matrix is replaced and M, V are re-aligned; the steps after that run under the
