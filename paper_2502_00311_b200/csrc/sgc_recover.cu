@@ -9,7 +9,7 @@
 //   generated entry; fp32 screen, fp64 decision among the near-maximal candidates, then the inverse-Cholesky
 //   recurrences of Algorithm 3 (c = F^T g, gamma, new column of F, a_j, x = F a) in fp64 and r = y - A_Lambda x.
 //
-// Speculative (rounds of k_omp mode 0, the tensor-core screening pass, k_resolve): OMP first runs on a short
+// Speculative (rounds of speculation kernels, the tensor-core screening pass, k_resolve): OMP first runs on a short
 //   candidate list only (the supports of the previous step plus harvested columns), which costs next to
 //   nothing, and records the residual before every pick.  ONE pass over all d columns then correlates A with
 //   all those residuals at once (sgc_pass.cu) and reports every column whose score comes within the rounding
@@ -17,10 +17,15 @@
 //   that wins the fp64 rescoring against its challengers, is the true argmax; at the first pick that loses,
 //   the global winner (known from the same pass) is forced, the columns reported for that residual join the
 //   candidate list and the next round continues from there.  Every round fixes at least one more pick; what is
-//   still open after kMaxRounds rounds, or after any overflow, is finished in lock-step.
+//   still open after the enqueued rounds, or after any overflow, is finished in lock-step.
+//   The speculation itself has three forms, chosen on the device by the length of the list: Algorithm 3 on the
+//   list's Gram matrix (k_gram_prepare, k_gram_matrix, k_omp_gram, k_spec_rows; up to kGramList columns), one
+//   block per residual correlating the list itself (k_spec_small; up to kSmallList), and k_omp mode 0 beyond.
 //
-// Both modes run inside one cooperative kernel: all blocks correlate (phase A), grid barrier, blocks 0 and 1
-// keep the books of M^ and V^ (phase B), grid barrier.  k_scatter applies Eq. (8) on the common support.
+// k_omp is one cooperative kernel for lock-step and long lists: all blocks correlate (phase A), grid barrier,
+// blocks 0 and 1 keep the books of M^ and V^ (phase B), grid barrier.  k_scatter applies Eq. (8) on the common
+// support.  Several states that share A are recovered together (launch_recover_group): their residuals sit side by
+// side in one screened batch, so one pass serves them all.
 #include <cooperative_groups.h>
 #include <cuda_fp16.h>
 
@@ -401,7 +406,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
             a.lam[(size_t)m * s + j] = lam_new;
         }
     }
-    // ---- 3. store the new column (bfloat16 bits, exact) ------------------------------------------------
+    // ---- 3. store the new column (binary16 bits, exact) --------------------------------------------------
     {
         const ColKey key = column_key(a.seed_lo, a.seed_hi, lam_new);
         uint16_t* znew = zs + (size_t)j * k;
@@ -575,7 +580,6 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
                     a.ctl->v[m] = j;
                     a.ctl->finished[m] = 1;
                     a.ctl->stop[m] = 1;
-                    sh.hi = base[m] > j ? j : sh.hi;
                 }
             }
         }
