@@ -103,11 +103,11 @@ constexpr int kCorrTop = 2;             // candidates kept per block and residua
 constexpr int kRescoreCap = 16;         // candidates rescored in fp64 per iteration and residual
 constexpr int kBookThreads = 1024;
 constexpr int kOmpThreads = 1024;       // threads per block of the cooperative OMP kernel
-constexpr int kCandCap = 16384;         // candidate columns kept for the restricted (speculative) OMP
-constexpr int kCandKeep = 12288;        // the list is rebuilt from the supports once it grows beyond this
+constexpr int kCandCap = 32768;         // candidate columns kept for the restricted (speculative) OMP
+constexpr int kCandKeep = 24576;        // the list is rebuilt from the supports once it grows beyond this
 constexpr int kSmallList = 768;         // lists up to this length are correlated inside the bookkeeping block
 constexpr int kGramList = 256;          // lists up to this length run OMP on their Gram matrix (Algorithm 3 as printed)
-constexpr int kRepCap = 2048;           // report slots per residual of one screening pass
+constexpr int kRepCap = 8192;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
 constexpr int kPassMaxBatch = 8;        // states whose residuals one screening pass can serve (kPassMaxN / 32)
 constexpr int kMaxRounds = 24;          // speculate / screen / resolve rounds enqueued per step

@@ -1376,8 +1376,8 @@ cudaError_t configure_recover(sgc_state* st) {
     int half = st->s < 128 ? st->s : 128;
     half = (half + 15) / 16 * 16;
     st->pass_n = 2 * half;
-    st->z_harvest = normal_tail_threshold((double)st->d, 1024.0);
-    st->z_floor = normal_tail_threshold((double)st->d, 1792.0);
+    st->z_harvest = normal_tail_threshold((double)st->d, 3072.0);
+    st->z_floor = normal_tail_threshold((double)st->d, 6144.0);
     if (st->spec_ok) {
         e = pass_configure(kPassMaxN);
         if (e != cudaSuccess) return e;
