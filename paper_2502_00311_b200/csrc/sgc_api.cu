@@ -58,6 +58,9 @@ size_t layout(sgc_state* st, unsigned char* base) {
         st->gram = carve<double>(base, off, (size_t)sgc::kGramList * sgc::kGramList);
         st->p0 = carve<double>(base, off, 2 * (size_t)sgc::kGramList);
         st->pick_li = carve<int>(base, off, 2 * s);
+        st->hist_slots = sgc::kHistColumns / (int)s < sgc::kHistSteps ? sgc::kHistColumns / (int)s : sgc::kHistSteps;
+        if (st->hist_slots < 1) st->hist_slots = 1;
+        st->kept_ring = carve<uint32_t>(base, off, (size_t)st->hist_slots * s);
     }
     return off;
 }
@@ -241,6 +244,7 @@ SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
         case SGC_GET_ROUNDS: src = &st->ctl->rounds; n = 4; break;
         case SGC_GET_FALLBACK: src = &st->ctl->fallback; n = 4; break;
         case SGC_GET_N_CAND: src = &st->ctl->n_cand; n = 4; break;
+        case SGC_GET_ROUND_TRACE: src = &st->ctl->trace[0][0]; n = 4 * 3 * sgc::kMaxRounds; break;
         default: return SGC_ERR_WHAT;
     }
     if (needs_step && !st->stepped) return SGC_ERR_NOSTEP;

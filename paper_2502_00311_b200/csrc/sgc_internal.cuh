@@ -106,6 +106,10 @@ constexpr int kOmpThreads = 1024;       // threads per block of the cooperative 
 constexpr int kCandCap = 32768;         // candidate columns kept for the restricted (speculative) OMP
 constexpr int kCandKeep = 24576;        // the list is rebuilt from the supports once it grows beyond this
 constexpr int kSmallList = 768;         // lists up to this length are correlated inside the bookkeeping block
+constexpr int kHistSteps = 64;          // steps whose kept indices (Sparsify_s) stay candidates ...
+constexpr int kHistColumns = 8192;      // ... as long as they are at most this many columns
+constexpr int kLookAhead = 12;          // after a refuted pick, every kLookAhead-th later residual is harvested too
+constexpr double kLookAheadShare = 0.78; // ... as far as its columns reach this share of the residual's pick score
 constexpr int kGramList = 256;          // lists up to this length run OMP on their Gram matrix (Algorithm 3 as printed)
 constexpr int kRepCap = 8192;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
@@ -142,6 +146,8 @@ struct SpecCtl {
     int gram_pending;       // list version seen by the round in flight
     int gram_todo;          // 1: the Gram matrix must be recomputed in this round
     int gram_ok;            // 0: the Gram path gave up in this step (a pick is missing from the list)
+    int hist_count, hist_next;  // ring of the kept index sets of the last steps: valid slots, slot of the next step
+    int trace[kMaxRounds][3];   // per round: confirmed picks of both streams and the list length after it
     double ynorm[2];        // ||y|| per residual
 };
 
@@ -204,6 +210,8 @@ struct sgc_state {
     double* gram;               // [kGramList][kGramList] Z_C^T Z_C
     double* p0;                 // [2][kGramList] Z_C^T y per residual
     int* pick_li;               // [2][s] list position of every pick (Gram path)
+    uint32_t* kept_ring;         // [hist_slots][s] kept indices of the last steps (all of them are columns M^ and V^ are made of)
+    int hist_slots;
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };

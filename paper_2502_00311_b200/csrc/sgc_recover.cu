@@ -1030,6 +1030,7 @@ struct ResolveArgs {
     OmpArgs o;
     const uint2* rep; int rep_cap;
     unsigned int* cand_bits; uint32_t* cand_list; double* rtmp;
+    const uint32_t* kept_ring;
 };
 
 __device__ __forceinline__ bool in_support(const uint32_t* lam, int n, uint32_t col) {
@@ -1067,28 +1068,67 @@ __device__ int collect_challengers(BookSmem& sh, const uint2* rep, unsigned int 
     return n > kRescoreCap ? -1 : n;
 }
 
-// the reported columns of one residual join the candidate list (the forced winner first)
-__device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, unsigned int count, uint32_t first) {
-    volatile SpecCtl* ctl = ra.o.ctl;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        sh.n_cand = ctl->n_cand;
-        if (first != kNoColumn && sh.n_cand < kCandCap) {
-            const unsigned int bit = 1u << (first & 31u);
-            if (!(atomicOr(&ra.cand_bits[first >> 5], bit) & bit)) ra.cand_list[sh.n_cand++] = first;
-        }
+// appends the columns `cols` that the list does not hold yet; n_s is the running length (shared memory)
+__device__ void cand_append(const uint32_t* cols, int n_cols, int* n_s, uint32_t* cand_list, unsigned int* cand_bits) {
+    for (int e = threadIdx.x; e < n_cols; e += blockDim.x) {
+        const uint32_t col = cols[e];
+        if (col == kNoColumn) continue;
+        const unsigned int bit = 1u << (col & 31u);
+        if (atomicOr(&cand_bits[col >> 5], bit) & bit) continue;
+        const int slot = atomicAdd(n_s, 1);
+        if (slot < kCandCap) cand_list[slot] = col;
+        else atomicAnd(&cand_bits[col >> 5], ~bit);
     }
+}
+
+// Cuts the candidate list back to what is certain to matter when `incoming` more columns would let it outgrow kCandKeep:
+// the ring of kept index sets and the picks made so far (columns harvested for earlier residuals have lost most of
+// their value: the residual has moved on).
+__device__ void make_room(const ResolveArgs& ra, int incoming) {
+    volatile SpecCtl* ctl = ra.o.ctl;
+    __shared__ int n_s;
+    __syncthreads();
+    const int n0 = ctl->n_cand;
+    if (n0 + incoming <= kCandKeep) return;
+    for (int e = threadIdx.x; e < n0; e += kOmpThreads) {
+        const uint32_t col = ra.cand_list[e];
+        atomicAnd(&ra.cand_bits[col >> 5], ~(1u << (col & 31u)));
+    }
+    if (threadIdx.x == 0) n_s = 0;
+    __syncthreads();
+    cand_append(ra.kept_ring, ctl->hist_count * ra.o.s, &n_s, ra.cand_list, ra.cand_bits);
+    __syncthreads();
+    for (int m = 0; m < 2; ++m) {
+        cand_append(ra.o.lam + (size_t)m * ra.o.s, ctl->finished[m] ? ra.o.cnt->done[m] : ctl->hi[m], &n_s, ra.cand_list,
+                    ra.cand_bits);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) { ctl->n_cand = n_s < kCandCap ? n_s : kCandCap; ctl->list_version = ctl->list_version + 1; }
+    __syncthreads();
+}
+
+// the reported columns of one residual that score at least `floor_sc` join the candidate list (the forced winner first)
+__device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, unsigned int count, uint32_t first,
+                        float floor_sc = 0.0f) {
+    volatile SpecCtl* ctl = ra.o.ctl;
+    __shared__ int n_s;
+    __syncthreads();
+    if (threadIdx.x == 0) n_s = ctl->n_cand;
+    __syncthreads();
+    if (first != kNoColumn) cand_append(&first, 1, &n_s, ra.cand_list, ra.cand_bits);
     __syncthreads();
     for (unsigned int e = threadIdx.x; e < count; e += kOmpThreads) {
-        const uint32_t col = rep[e].x;
+        const uint2 rp = rep[e];
+        if (__uint_as_float(rp.y) < floor_sc) continue;
+        const uint32_t col = rp.x;
         const unsigned int bit = 1u << (col & 31u);
         if (atomicOr(&ra.cand_bits[col >> 5], bit) & bit) continue;
-        const int slot = atomicAdd(&sh.n_cand, 1);
+        const int slot = atomicAdd(&n_s, 1);
         if (slot < kCandCap) ra.cand_list[slot] = col;
         else atomicAnd(&ra.cand_bits[col >> 5], ~bit);
     }
     __syncthreads();
-    if (threadIdx.x == 0) { ctl->n_cand = sh.n_cand < kCandCap ? sh.n_cand : kCandCap; ctl->list_version = ctl->list_version + 1; }
+    if (threadIdx.x == 0) { ctl->n_cand = n_s < kCandCap ? n_s : kCandCap; ctl->list_version = ctl->list_version + 1; }
     __syncthreads();
 }
 
@@ -1157,7 +1197,18 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             rescore_candidates(a, sh, nc, ra.rtmp);
             if (sh.best_idx == pick) { v = j + 1; continue; }
             forced = sh.best_idx; v = j; failed = true;
+            make_room(ra, (int)count + 1 + ((hi - j) / kLookAhead) * 1024);
             harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
+            // look ahead: the later residuals of this speculation are off the true path by a pick or a few, yet close
+            // to it, so the columns that come near their picks are the likely picks of the next round
+            for (int jj = j + kLookAhead; jj < hi; jj += kLookAhead) {
+                const int nn = m * a.half_n + (jj - base);
+                const unsigned int cc = a.rep_count[nn];
+                if (cc > (unsigned int)ra.rep_cap) continue;
+                harvest(ra, sh, ra.rep + (size_t)nn * ra.rep_cap, cc, kNoColumn,
+                        (float)(kLookAheadShare * a.pick_score[(size_t)m * s + jj]));        // reports hold unscaled scores
+            }
+
         }
         if (!failed && !bad) {
             if (dep) {
@@ -1184,6 +1235,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                     rebuild_prefix(a, sh, m, hi, ra.rtmp, nullptr, nullptr);
                     rescore_candidates(a, sh, nc, ra.rtmp);
                     forced = sh.best_idx; v = hi;
+                    make_room(ra, (int)count + 1);
                     harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
                 }
             } else {
@@ -1205,6 +1257,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         } else if (ctl->finished[0] && ctl->finished[1]) {
             ctl->round_active = 0;
         }
+        const int r = ctl->rounds - 1;
+        if (r >= 0 && r < kMaxRounds) { ctl->trace[r][0] = ctl->v[0]; ctl->trace[r][1] = ctl->v[1]; ctl->trace[r][2] = ctl->n_cand; }
     }
 }
 
@@ -1217,22 +1271,46 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate) {
         ctl->finished[0] = ctl->finished[1] = 0;
         ctl->stop[0] = ctl->stop[1] = 0;
         ctl->rounds = 0; ctl->pass_error = 0;
+        for (int r = 0; r < kMaxRounds; ++r) ctl->trace[r][0] = ctl->trace[r][1] = ctl->trace[r][2] = 0;
         ctl->gram_ok = 1;
         if (ctl->list_version == 0) ctl->list_version = 1;      // a fresh state: no Gram matrix yet
+    }
+}
+
+// start of the step, after Sparsify_s: M^ and V^ are combinations of the columns kept in this and in earlier steps
+// (Eq. 4, 5), so the indices just kept are candidates, and they enter the ring of recent index sets
+__global__ void __launch_bounds__(kOmpThreads, 1)
+k_cand_begin(SpecCtl* ctl, const uint32_t* sel_idx, int s, uint32_t* kept_ring, int hist_slots, uint32_t* cand_list,
+             unsigned int* cand_bits) {
+    __shared__ int n_s;
+    const int n0 = ctl->n_cand;
+    const int slot = ctl->hist_next % hist_slots;
+    if (threadIdx.x == 0) n_s = n0;
+    for (int e = threadIdx.x; e < s; e += kOmpThreads) kept_ring[(size_t)slot * s + e] = sel_idx[e];
+    __syncthreads();
+    cand_append(sel_idx, s, &n_s, cand_list, cand_bits);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int n_new = n_s < kCandCap ? n_s : kCandCap;
+        if (n_new != n0) { ctl->n_cand = n_new; ctl->list_version = ctl->list_version + 1; }
+        ctl->hist_next = (slot + 1) % hist_slots;
+        if (ctl->hist_count < hist_slots) ctl->hist_count = ctl->hist_count + 1;
     }
 }
 
 // end of the step: the supports found stay (or become) candidates of the next step
 __global__ void __launch_bounds__(kOmpThreads, 1)
 k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uint32_t* cand_list, unsigned int* cand_bits,
-              int* rounds_out) {
+              const uint32_t* kept_ring, int* rounds_out) {
     __shared__ int n_s;
     // how many rounds this step took (the enqueued rounds if even they were not enough): sizes the next step's launches
     if (threadIdx.x == 0) *rounds_out = ctl->fallback ? kMaxRounds : ctl->rounds;
     int n = ctl->n_cand;
-    // rebuild from the supports alone when the list has outgrown its bound, or when it holds far more than the
-    // supports although a single round confirmed every pick (harvested columns of an earlier cold start)
-    if (n > kCandKeep || (ctl->rounds <= 1 && !ctl->fallback && n > 4 * s)) {
+    // rebuild from the supports and the ring of kept index sets when the list has outgrown its bound, or when it holds
+    // far more than those although a single round confirmed every pick (harvested columns of an earlier cold start)
+    const int n_hist = ctl->hist_count * s;
+    const bool rebuild = n > kCandKeep || (ctl->rounds <= 1 && !ctl->fallback && n > 4 * s + n_hist);
+    if (rebuild) {
         for (int e = threadIdx.x; e < n; e += kOmpThreads) {
             const uint32_t col = cand_list[e];
             atomicAnd(&cand_bits[col >> 5], ~(1u << (col & 31u)));
@@ -1241,16 +1319,11 @@ k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uin
     }
     if (threadIdx.x == 0) n_s = n;
     __syncthreads();
-    for (int e = threadIdx.x; e < 2 * s; e += kOmpThreads) {
-        const int m = e / s, j = e % s;
-        if (j >= cnt->done[m]) continue;
-        const uint32_t col = lam[e];
-        const unsigned int bit = 1u << (col & 31u);
-        if (atomicOr(&cand_bits[col >> 5], bit) & bit) continue;
-        const int slot = atomicAdd(&n_s, 1);
-        if (slot < kCandCap) cand_list[slot] = col;
-        else atomicAnd(&cand_bits[col >> 5], ~bit);
+    for (int m = 0; m < 2; ++m) {
+        cand_append(lam + (size_t)m * s, cnt->done[m] < s ? cnt->done[m] : s, &n_s, cand_list, cand_bits);
+        __syncthreads();
     }
+    if (rebuild) cand_append(kept_ring, n_hist, &n_s, cand_list, cand_bits);
     __syncthreads();
     if (threadIdx.x == 0) {
         const int n_new = n_s < kCandCap ? n_s : kCandCap;
@@ -1423,6 +1496,11 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
             PhaseTimer timer(st, stream, kPhaseBook, 1);
             k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0);
             *launches += 1;
+            if (speculate) {
+                k_cand_begin<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->sel_idx, st->s, st->kept_ring, st->hist_slots,
+                                                            st->cand_list, st->cand_bits);
+                *launches += 1;
+            }
         }
         // rounds to enqueue: twice what the last finished step needed plus slack (read from pinned memory without
         // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
@@ -1468,6 +1546,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     ra.o = args[i];
                     ra.rep = lead->rep + (size_t)(i - b0) * st->pass_n * kRepCap;
                     ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list; ra.rtmp = st->rtmp;
+                    ra.kept_ring = st->kept_ring;
                     PhaseTimer timer(st, stream, kPhaseBook, 1);
                     k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
                     *launches += 1;
@@ -1490,7 +1569,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
         *launches += 1;
         if (speculate) {
             k_cand_update<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->cnt, st->lam, st->s, st->cand_list, st->cand_bits,
-                                                         st->d_rounds);
+                                                         st->kept_ring, st->d_rounds);
             *launches += 1;
         }
     }
