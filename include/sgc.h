@@ -92,6 +92,7 @@ enum {
     SGC_GET_ROUNDS = 21,    /* int32      screening passes over all d columns that the last step needed (speculative recovery) */
     SGC_GET_FALLBACK = 22,  /* int32      1 when the last step finished (or ran entirely) in lock-step  */
     SGC_GET_N_CAND = 23,    /* int32      length of the candidate list kept for the next step           */
+    SGC_GET_LIST_ROUNDS = 25, /* int32     list passes (screening passes over the wide lists only) that the last step resolved */
     SGC_GET_ROUND_TRACE = 24 /* int32[24][3] per screening pass of the last step: picks of M^ confirmed so far, picks of V^ confirmed so
                                 far, length of the candidate list after it (rows past SGC_GET_ROUNDS are zero)               */
 };

@@ -24,7 +24,7 @@ RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, 
                status=(14, np.uint32, None), mismatch=(15, np.int32, None), negv=(16, np.int32, None),
                doneM=(17, np.int32, None), doneV=(18, np.int32, None), rnormM=(19, np.float64, "s"),
                rnormV=(20, np.float64, "s"), rounds=(21, np.int32, None), fallback=(22, np.int32, None),
-               n_cand=(23, np.int32, None), round_trace=(24, np.int32, 72))
+               n_cand=(23, np.int32, None), round_trace=(24, np.int32, 72), list_rounds=(25, np.int32, None))
 
 MODE_AUTO, MODE_LOCKSTEP, MODE_SPECULATIVE = 0, 1, 2
 

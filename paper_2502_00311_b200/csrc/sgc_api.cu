@@ -61,6 +61,10 @@ size_t layout(sgc_state* st, unsigned char* base) {
         st->hist_slots = sgc::kHistColumns / (int)s < sgc::kHistSteps ? sgc::kHistColumns / (int)s : sgc::kHistSteps;
         if (st->hist_slots < 1) st->hist_slots = 1;
         st->kept_ring = carve<uint32_t>(base, off, (size_t)st->hist_slots * s);
+        st->wide_tau = carve<float>(base, off, sgc::kPassMaxN / 8);
+        st->wide_list = carve<uint32_t>(base, off, 2 * (size_t)sgc::kWideCap);
+        st->wide_count = carve<unsigned int>(base, off, 2);
+        st->wide_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
     }
     return off;
 }
@@ -244,6 +248,7 @@ SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
         case SGC_GET_ROUNDS: src = &st->ctl->rounds; n = 4; break;
         case SGC_GET_FALLBACK: src = &st->ctl->fallback; n = 4; break;
         case SGC_GET_N_CAND: src = &st->ctl->n_cand; n = 4; break;
+        case SGC_GET_LIST_ROUNDS: src = &st->ctl->list_rounds; n = 4; break;
         case SGC_GET_ROUND_TRACE: src = &st->ctl->trace[0][0]; n = 4 * 3 * sgc::kMaxRounds; break;
         default: return SGC_ERR_WHAT;
     }

@@ -110,6 +110,9 @@ constexpr int kHistSteps = 64;          // steps whose kept indices (Sparsify_s)
 constexpr int kHistColumns = 8192;      // ... as long as they are at most this many columns
 constexpr int kLookAhead = 12;          // after a refuted pick, every kLookAhead-th later residual is harvested too
 constexpr double kLookAheadShare = 0.78; // ... as far as its columns reach this share of the residual's pick score
+constexpr int kWideCap = 2097152;       // columns per wide list (two-level screening)
+constexpr int kMiniRounds = 8;          // list passes between two full passes, at most
+constexpr int kMiniDepth = 32;          // picks speculated ahead of one list pass
 constexpr int kGramList = 256;          // lists up to this length run OMP on their Gram matrix (Algorithm 3 as printed)
 constexpr int kRepCap = 8192;           // report slots per residual of one screening pass
 constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
@@ -146,6 +149,11 @@ struct SpecCtl {
     int gram_pending;       // list version seen by the round in flight
     int gram_todo;          // 1: the Gram matrix must be recomputed in this round
     int gram_ok;            // 0: the Gram path gave up in this step (a pick is missing from the list)
+    int tv[2];              // tentative picks: confirmed against the wide lists only (tv >= v)
+    uint32_t tforced[2];    // column imposed as pick tv[m] by a list pass, or kNoColumn
+    int mini_done;          // 1: list passes rest until the next full pass
+    int list_rounds;        // list passes of the last step that were resolved
+    int list_refuted;       // picks that those list passes refuted
     int hist_count, hist_next;  // ring of the kept index sets of the last steps: valid slots, slot of the next step
     int trace[kMaxRounds][3];   // per round: confirmed picks of both streams and the list length after it
     double ynorm[2];        // ||y|| per residual
@@ -175,6 +183,7 @@ struct sgc_state {
     bool spec_ok;               // speculative recovery usable for this (d, k)
     int pass_n;                 // residuals per screening pass (multiple of 32, <= 256); pass_n / 2 per residual stream
     double z_harvest, z_floor;  // thresholds of the screening pass in units of ||r|| / sqrt(k)
+    double z_wide;              // threshold of the wide lists, same units
     unsigned char tmap[8][128]; // CUtensorMaps of the residual matrix R^T, one per number of states batched into a pass
     // optional per-kernel timing (sgc_set_profile)
     bool profile;
@@ -212,6 +221,11 @@ struct sgc_state {
     int* pick_li;               // [2][s] list position of every pick (Gram path)
     uint32_t* kept_ring;         // [hist_slots][s] kept indices of the last steps (all of them are columns M^ and V^ are made of)
     int hist_slots;
+    bool two_level;             // host: wide lists and list passes are in use (steps that need several full passes)
+    float* wide_tau;            // [kPassMaxN / 8] thresholds of the wide lists, one per 8th screened residual
+    uint32_t* wide_list;        // [2][kWideCap]
+    unsigned int* wide_count;   // [2]
+    unsigned int* wide_bits;    // bitmap over [0, d): the column is in one of the wide lists
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };
@@ -252,11 +266,22 @@ cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t c
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
 cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T
 
+// wide lists of the two-level screening (sgc_pass.cu): a full pass fills them, a list pass screens only their columns
+struct PassWide {
+    const float* tau;            // [n / 8] thresholds of the wide lists (scaled units of rows 0, 8, 16, ...)
+    uint32_t* list;              // [2][cap]
+    unsigned int* count;         // [2]
+    unsigned int* bits;          // bitmap over [0, d): a column enters the lists once
+    int cap, half_n;
+    const SpecCtl* ctl;
+    bool list_pass;              // true: screen the lists' columns; false: full pass that feeds the lists
+};
+
 // screening pass (sgc_pass.cu)
 cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
-                        int* const* errors, int sm_count, cudaStream_t stream);
+                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide = nullptr);
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream);
 }  // namespace sgc

@@ -49,6 +49,16 @@ struct PassArgs {
     unsigned int* rep_count;     // [n]
     uint2* rep;                  // [n][rep_cap]  (column, score bits)
     int rep_cap;
+    // Two-level screening (single state only).  A full pass also collects, for every 8th residual of each stream,
+    // every column scoring at least big_tau[row / 8] into the stream's "wide list" (some 10^5 columns; the bitmap lets a
+    // column in once).  A list pass (list_ctl != nullptr) then screens only the columns of the two wide lists: a few
+    // percent of the work of a full pass.
+    const float* big_tau;        // [n / 8] or nullptr
+    uint32_t* big_list;          // [2][big_cap]
+    unsigned int* big_count;     // [2]
+    unsigned int* big_bits;      // bitmap over [0, d)
+    int big_cap, big_half;
+    const SpecCtl* list_ctl;     // list pass: gate and list lengths come from the control block
     const int* gate[kPassMaxBatch];   // optional: the kernel returns at once when every *gate is 0 (one per batched state)
     int* error[kPassMaxBatch];        // set to 1 when a wait expired (one per batched state)
 };
@@ -155,7 +165,8 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 //   norms  float[kNormRing][256][2]      partial ||Z_i||^2 of the two generator threads of each column
 //   tau    float[256]
 //   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
-template <bool TABLE>
+// WIDE: the two-level screening code (wide-list harvest, list passes) is compiled in
+template <bool TABLE, bool WIDE>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
     if (a.gate[0] != nullptr) {
         bool any = false;
@@ -163,6 +174,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         for (int q = 0; q < kPassMaxBatch; ++q) any = any || (a.gate[q] != nullptr && *a.gate[q] != 0);
         if (!any) return;
     }
+    // list pass: the columns are the concatenation of the two wide lists (every block reads the same lengths: nothing
+    // writes them while a list pass runs)
+    unsigned int list_n0 = 0, list_n = 0, num_super = a.num_super;
+    if (WIDE && a.list_ctl != nullptr) {
+        const volatile SpecCtl* lc = a.list_ctl;
+        if (!lc->round_active || lc->fallback || lc->mini_done || lc->n_cand <= kSmallList) return;
+        list_n0 = min(a.big_count[0], (unsigned int)a.big_cap);
+        list_n = list_n0 + min(a.big_count[1], (unsigned int)a.big_cap);
+        if (list_n == 0) return;
+        num_super = (list_n + kSuperCols - 1) / kSuperCols;
+        if (blockIdx.x >= num_super) return;
+    }
+    const bool listed = WIDE && a.list_ctl != nullptr;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -209,7 +233,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         if (lane == 0) {
             uint32_t st = 0, ph = 0;
             bool ok = true;
-            for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x) {
+            for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x) {
                 for (int kc = 0; kc < kc_count; ++kc) {
                     if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 256)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u);
@@ -228,7 +252,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             const uint32_t stage_step = (uint32_t)stage_bytes >> 4;
             uint32_t st = 0, ph = 0, sweep_i = 0;
             bool ok = true;
-            for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
+            for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x, ++sweep_i) {
                 const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
                 if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 32)) { ok = false; break; }
                 tc_fence_after();
@@ -255,7 +279,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         const int quad = warp & 3;
         uint32_t sweep_i = 0;
         bool ok = true;
-        for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
+        for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x, ++sweep_i) {
             const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
             if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag, 512))) { ok = false; break; }
             tc_fence_after();
@@ -263,7 +287,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
 #pragma unroll 1
             for (int t = 0; t < 2; ++t) {
                 const int col_local = t * kTileCols + quad * 32 + lane;
-                const unsigned long long col = (unsigned long long)sweep * kSuperCols + col_local;
+                unsigned long long col = (unsigned long long)sweep * kSuperCols + col_local;
+                if (listed) {
+                    const unsigned int idx = (unsigned int)col;
+                    col = idx < list_n0 ? a.big_list[idx] : (idx < list_n ? a.big_list[(size_t)a.big_cap + idx - list_n0] : a.d);
+                }
                 float inv = 0.0f;
                 if (TABLE) {
                     if (col < a.d) inv = half_bits_to_float(a.inv_norm[col]);
@@ -275,6 +303,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                 for (int c0 = 0; c0 < a.n; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * acc_cols + t * a.n + c0, v);
+                    if (WIDE && a.big_tau != nullptr && !listed && inv > 0.0f) {
+                        // every 8th residual feeds the wide list of its stream
+                        const bool w0 = fabsf(__uint_as_float(v[0])) * inv >= a.big_tau[c0 >> 3];
+                        const bool w8 = fabsf(__uint_as_float(v[8])) * inv >= a.big_tau[(c0 >> 3) + 1];
+                        if (w0 || w8) {
+                            const unsigned int bit = 1u << ((unsigned int)col & 31u);
+                            if (!(atomicOr(&a.big_bits[col >> 5], bit) & bit)) {
+                                const int m = c0 >= a.big_half ? 1 : 0;
+                                const unsigned int slot = atomicAdd(&a.big_count[m], 1u);
+                                if (slot < (unsigned int)a.big_cap) a.big_list[(size_t)m * a.big_cap + slot] = (uint32_t)col;
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float sc = fabsf(__uint_as_float(v[i])) * inv;
@@ -304,8 +345,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         for (int c = 0; c < 4; ++c) off[c] = row_off + ((((uint32_t)(half * 4 + c)) ^ sw) << 4);
         uint32_t st = 0, ph = 0, sweep_i = 0;
         bool ok = true;
-        for (unsigned int sweep = blockIdx.x; ok && sweep < a.num_super; sweep += gridDim.x, ++sweep_i) {
-            const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)((unsigned long long)sweep * kSuperCols + col_local));
+        for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x, ++sweep_i) {
+            uint32_t gcol = (uint32_t)((unsigned long long)sweep * kSuperCols + col_local);
+            if (listed) gcol = gcol < list_n0 ? a.big_list[gcol] : (gcol < list_n ? a.big_list[(size_t)a.big_cap + gcol - list_n0] : 0u);
+            const ColKey key = column_key(a.seed_lo, a.seed_hi, gcol);
             float norm = 0.0f;
             uint32_t h = key.ck + (uint32_t)(half * 16) * key.mk;   // one word per row pair
             const uint32_t skip = 16u * key.mk;                  // the other generator thread of this column owns the next 32 rows
@@ -427,9 +470,11 @@ cudaError_t pass_configure(int) {
         const size_t b = pass_smem_bytes(n, pass_stages(n));
         if (b > need) need = b;
     }
-    cudaError_t e = cudaFuncSetAttribute(k_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    cudaError_t e = cudaFuncSetAttribute(k_pass<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    e = cudaFuncSetAttribute(k_pass<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_pass<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
 }
 
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream) {
@@ -439,7 +484,7 @@ cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cu
 
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
-                        int* const* errors, int sm_count, cudaStream_t stream) {
+                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide) {
     PassArgs a;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
@@ -447,12 +492,20 @@ cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int 
     a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
     a.tau = tau; a.inv_scale = inv_scale; a.inv_norm = inv_norm; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap;
     for (int q = 0; q < kPassMaxBatch; ++q) { a.gate[q] = gates ? gates[q] : nullptr; a.error[q] = errors ? errors[q] : nullptr; }
+    a.big_tau = nullptr; a.big_list = nullptr; a.big_count = nullptr; a.big_bits = nullptr; a.big_cap = 0; a.big_half = 0;
+    a.list_ctl = nullptr;
+    if (wide) {
+        a.big_tau = wide->tau; a.big_list = wide->list; a.big_count = wide->count; a.big_bits = wide->bits;
+        a.big_cap = wide->cap; a.big_half = wide->half_n;
+        a.list_ctl = wide->list_pass ? wide->ctl : nullptr;
+    }
     unsigned int grid = (unsigned int)sm_count;
     if (grid > a.num_super) grid = a.num_super;
     CUtensorMap map;
     memcpy(&map, tmap, sizeof(map));
-    if (inv_norm) k_pass<true><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
-    else k_pass<false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    if (inv_norm && wide) k_pass<true, true><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    else if (inv_norm) k_pass<true, false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    else k_pass<false, false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
     return cudaGetLastError();
 }
 

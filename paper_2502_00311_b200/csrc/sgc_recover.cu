@@ -49,6 +49,10 @@ struct OmpArgs {
     uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
     Counters* cnt; SpecCtl* ctl;
     uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; double* pick_score;
+    // two-level screening
+    float* wide_tau; double z_wide; unsigned int* wide_count; unsigned int* wide_bits;
+    int mini;                          // 1: speculation ahead of a list pass (at most `depth` picks)
+    int depth;
     const uint32_t* cand_list;
     uint16_t* zlist; double* gram; double* p0; int* pick_li;     // Gram path
 };
@@ -112,6 +116,12 @@ __device__ __forceinline__ double residual_scale(double rn) {
     int e;
     frexp(rn, &e);
     return ldexp(1.0, 13 - e);
+}
+
+// threshold of a wide list: every column scoring at least z_wide noise deviations against a screened residual (norm rn)
+// whose row index is a multiple of 8, in the scaled units of that row
+__device__ __forceinline__ float wide_threshold(const OmpArgs& a, double rn) {
+    return (float)(a.z_wide * rn / sqrt((double)a.k) * residual_scale(rn));
 }
 
 // shared memory of the bookkeeping code (blocks 0 and 1 of k_omp, the only block of k_resolve)
@@ -403,6 +413,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
             if (t > a.z_harvest * unit) t = a.z_harvest * unit;
             if (t < a.z_floor * unit) t = a.z_floor * unit;
             a.tau[m * a.half_n + spec_c] = (float)(t * residual_scale(rn));     // row spec_c was scaled with this norm
+            if ((spec_c & 7) == 0) a.wide_tau[(m * a.half_n + spec_c) >> 3] = wide_threshold(a, rn);
             a.lam[(size_t)m * s + j] = lam_new;
         }
     }
@@ -487,7 +498,8 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     if (threadIdx.x == 0) {
         a.rnorm[(size_t)m * s + j] = sqrt(rn2);
         sh.cur_rnorm = sqrt(rn2);
-        if (final_pick) { a.cnt->done[m] = j + 1; a.ctl->v[m] = j + 1; }
+        // a prescribed column, if there was one, is consumed with this pick
+        if (final_pick) { a.cnt->done[m] = j + 1; a.ctl->v[m] = j + 1; a.ctl->forced[m] = kNoColumn; }
     }
     __syncthreads();
     return 0;
@@ -506,32 +518,60 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
     volatile SpecCtl* ctl = a.ctl;
     // ---- gate: identical in every block, because nothing below changes the control block before the first barrier
     const int fin[2] = {ctl->finished[0], ctl->finished[1]};
-    if (mode == 0) { if (!ctl->round_active || ctl->fallback || ctl->n_cand <= kSmallList) return; }
-    else { if (fin[0] && fin[1]) return; }
-    const int v0[2] = {ctl->v[0], ctl->v[1]};
-    const uint32_t forced0[2] = {ctl->forced[0], ctl->forced[1]};
+    if (mode == 0) {
+        if (!ctl->round_active || ctl->fallback || ctl->n_cand <= kSmallList) return;
+        if (a.mini && (ctl->mini_done || (a.wide_count[0] == 0u && a.wide_count[1] == 0u))) return;
+    } else if (fin[0] && fin[1]) return;
+    const int vc[2] = {ctl->v[0], ctl->v[1]};                            // confirmed picks
+    const uint32_t fc[2] = {ctl->forced[0], ctl->forced[1]};             // confirmed winner for pick vc, if any
     const int n_cand = ctl->n_cand;
-    const int base[2] = {v0[0] + (forced0[0] != kNoColumn ? 1 : 0), v0[1] + (forced0[1] != kNoColumn ? 1 : 0)};
+    const int base[2] = {vc[0] + (fc[0] != kNoColumn ? 1 : 0), vc[1] + (fc[1] != kNoColumn ? 1 : 0)};
+    // where this kernel starts: the speculation resumes after the tentative picks (those confirmed against the wide
+    // lists only), lock-step after the confirmed ones.  The first pick may be prescribed: confirmed (final) or imposed
+    // by a list pass (still speculative).
+    int v0[2]; uint32_t first_col[2]; bool first_final[2];
+    for (int m = 0; m < 2; ++m) {
+        const int tv = ctl->tv[m];
+        v0[m] = (mode == 0 && tv > vc[m]) ? tv : vc[m];
+        first_final[m] = v0[m] == vc[m] && fc[m] != kNoColumn;
+        uint32_t first = 0xFFFFFFFFu;                  // kNoColumn
+        if (first_final[m]) first = fc[m];
+        else if (mode == 0 && v0[m] == tv) first = ctl->tforced[m];
+        first_col[m] = first;
+    }
     grid.sync();
     const int mb = blockIdx.x;                           // blocks 0 and 1 keep the books of M^ and V^
+    // the first full pass of a step starts the wide lists afresh; later ones add what their residuals bring (the lists then
+    // cover the whole path of this step, which is where the next step's path runs, too)
+    if (mode == 0 && !a.mini && a.wide_count != nullptr && ctl->rounds == 0) {
+        if (mb == 0 && threadIdx.x == 0) a.wide_count[0] = a.wide_count[1] = 0u;
+        const size_t words = ((size_t)a.d + 31) / 32;
+        for (size_t w = (size_t)blockIdx.x * kOmpThreads + threadIdx.x; w < words; w += (size_t)gridDim.x * kOmpThreads)
+            a.wide_bits[w] = 0u;
+    }
     if (mb < 2) {
         if (!fin[mb]) {
-            // state after the verified picks (a failed speculation left later values behind)
+            // state after the picks made so far (a refuted speculation left later values behind)
             const double rn = rebuild_prefix(a, sh, mb, v0[mb], a.r64 + (size_t)mb * a.k, a.r32, a.x + (size_t)mb * a.s);
             if (threadIdx.x == 0) {
                 sh.cur_rnorm = rn;
                 if (v0[mb] == 0) a.ctl->ynorm[mb] = rn;
-                sh.hi = base[mb]; sh.extra = 0; sh.dep = 0;
+                sh.hi = v0[mb] > base[mb] ? v0[mb] : base[mb]; sh.extra = 0; sh.dep = 0;
                 a.ctl->stop[mb] = 0;
             }
-            if (mode == 0 && forced0[mb] == kNoColumn) write_rt_row(a, mb, 0, a.r64 + (size_t)mb * a.k, rn);
+            const int c0 = v0[mb] - base[mb];
+            if (mode == 0 && !first_final[mb] && c0 >= 0 && c0 < a.half_n) write_rt_row(a, mb, c0, a.r64 + (size_t)mb * a.k, rn);
         } else if (threadIdx.x == 0) {
             a.ctl->stop[mb] = 1;
         }
         if (mode == 0) {
+            const int keep = fin[mb] ? 0 : (v0[mb] - base[mb] > 0 ? v0[mb] - base[mb] : 0);   // rows of earlier tentative picks stay
             for (int c = threadIdx.x; c < a.half_n; c += kOmpThreads) {
                 a.rep_count[mb * a.half_n + c] = 0u;
-                a.tau[mb * a.half_n + c] = __int_as_float(0x7f800000);
+                if (c >= keep) {
+                    a.tau[mb * a.half_n + c] = __int_as_float(0x7f800000);
+                    if ((c & 7) == 0) a.wide_tau[(mb * a.half_n + c) >> 3] = __int_as_float(0x7f800000);
+                }
             }
         }
     }
@@ -542,9 +582,9 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
         for (int m = 0; m < 2; ++m) {
             jm[m] = v0[m] + i;
             act[m] = !fin[m] && jm[m] < a.s && !ctl->stop[m];
-            if (mode == 0 && jm[m] - base[m] >= a.half_n) act[m] = false;
+            if (mode == 0 && (jm[m] - base[m] >= a.half_n || i >= a.depth)) act[m] = false;
             picks[m] = jm[m] < a.s ? jm[m] : a.s;
-            if (act[m] && !(i == 0 && forced0[m] != kNoColumn)) need_corr = true;
+            if (act[m] && !(i == 0 && first_col[m] != kNoColumn)) need_corr = true;
         }
         if (!act[0] && !act[1]) break;
         if (need_corr) {
@@ -554,9 +594,9 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
         grid.sync();
         if (mb < 2 && act[mb]) {
             const int m = mb, j = jm[m];
-            const uint32_t forced = (i == 0) ? forced0[m] : kNoColumn;
-            const bool speculative = (mode == 0) && forced == kNoColumn;
-            const int c = j - base[m];                            // -1 for a forced pick
+            const uint32_t forced = (i == 0) ? first_col[m] : kNoColumn;
+            const bool speculative = (mode == 0) && !(i == 0 && first_final[m]);
+            const int c = j - base[m];                            // -1 for a confirmed prescribed pick
             const int next = (mode == 0 && c + 1 < a.half_n && j + 1 < a.s) ? c + 1 : -1;
             const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative,
                                      a.corr_cand + (size_t)m * gridDim.x * kCorrTop, (int)gridDim.x * kCorrTop);
@@ -570,6 +610,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
                         sh.extra = 1;
                         a.tau[m * a.half_n + c] =
                             (float)(a.z_harvest * sh.cur_rnorm / sqrt((double)a.k) * residual_scale(sh.cur_rnorm));
+                        if ((c & 7) == 0) a.wide_tau[(m * a.half_n + c) >> 3] = wide_threshold(a, sh.cur_rnorm);
                     } else { sh.dep = 1; sh.hi = j + 1; }
                     a.ctl->stop[m] = 1;
                 } else {
@@ -1031,6 +1072,8 @@ struct ResolveArgs {
     const uint2* rep; int rep_cap;
     unsigned int* cand_bits; uint32_t* cand_list; double* rtmp;
     const uint32_t* kept_ring;
+    int mini;                              // 1: the reports come from a list pass (two-level screening)
+    const unsigned int* wide_count;
 };
 
 __device__ __forceinline__ bool in_support(const uint32_t* lam, int n, uint32_t col) {
@@ -1132,18 +1175,34 @@ __device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, u
     __syncthreads();
 }
 
+// Full mode (reports of a pass over all d columns): confirms the speculated picks in order; the first refuted pick of a
+// stream gets its true winner, which becomes final.  Mini mode (reports of a list pass over the wide lists): the same
+// walk, but what it establishes is tentative -- tv / tforced tell the next speculation where to resume, while v, forced,
+// the round count and everything a finished recovery records are left alone; the next full pass judges all of it.
 __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
     const OmpArgs& a = ra.o;
     __shared__ BookSmem sh;
-    __shared__ int give_up;
+    __shared__ int give_up, any_failed;
     volatile SpecCtl* ctl = a.ctl;
+    const bool mini = ra.mini != 0;
     if (!ctl->round_active) return;
     if (ctl->fallback || ctl->pass_error) {
         if (threadIdx.x == 0) { ctl->fallback = 1; ctl->round_active = 0; }
         return;
     }
+    if (mini) {
+        if (ctl->mini_done || ctl->n_cand <= kSmallList) return;
+        if (ra.wide_count[0] == 0u && ra.wide_count[1] == 0u) {
+            if (threadIdx.x == 0) ctl->mini_done = 1;
+            return;
+        }
+    }
     __shared__ int contested[kPassMaxN];        // per screened residual: some report comes within the margin of its pick
-    if (threadIdx.x == 0) { give_up = 0; ctl->rounds = ctl->rounds + 1; }
+    if (threadIdx.x == 0) {
+        give_up = 0; any_failed = 0;
+        if (mini) ctl->list_rounds = ctl->list_rounds + 1;
+        else ctl->rounds = ctl->rounds + 1;
+    }
     for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = 0;
     __syncthreads();
     const int s = a.s;
@@ -1151,7 +1210,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
     for (int m = 0; m < 2; ++m) {
         if (ctl->finished[m]) continue;
         const int base = ctl->base[m], hi = ctl->hi[m];
-        for (int j = base + (threadIdx.x >> 5); j < hi; j += kOmpThreads / 32) {      // warp per residual
+        const int lo = (mini && ctl->tv[m] > base) ? ctl->tv[m] : base;
+        for (int j = lo + (threadIdx.x >> 5); j < hi; j += kOmpThreads / 32) {         // warp per residual
             const int n = m * a.half_n + (j - base);
             const unsigned int count = a.rep_count[n];
             if (count > (unsigned int)ra.rep_cap) { if ((threadIdx.x & 31) == 0) contested[n] = 1; continue; }
@@ -1176,10 +1236,11 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         if (ctl->finished[m]) continue;
         const int base = ctl->base[m], hi = ctl->hi[m], extra = ctl->extra[m], dep = ctl->dep[m];
         const uint32_t* lam = a.lam + (size_t)m * s;
-        int v = base;
+        const int lo = (mini && ctl->tv[m] > base) ? ctl->tv[m] : base;
+        int v = lo;
         uint32_t forced = kNoColumn;
         bool failed = false, bad = false;
-        for (int j = base; j < hi && !failed && !bad; ++j) {
+        for (int j = lo; j < hi && !failed && !bad; ++j) {
             const int n = m * a.half_n + (j - base);
             if (!contested[n]) { v = j + 1; continue; }           // nobody comes close: the pick is the argmax
             const unsigned int count = a.rep_count[n];
@@ -1209,6 +1270,19 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                         (float)(kLookAheadShare * a.pick_score[(size_t)m * s + jj]));        // reports hold unscaled scores
             }
 
+        }
+        if (mini) {
+            // tentative outcome only
+            if (!failed && !bad) v = dep ? hi - 1 : hi;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                ctl->tv[m] = v;
+                ctl->tforced[m] = forced;
+                if (failed) { any_failed = 1; ctl->list_refuted = ctl->list_refuted + 1; }
+                if (bad) give_up = 1;
+            }
+            __syncthreads();
+            continue;
         }
         if (!failed && !bad) {
             if (dep) {
@@ -1246,11 +1320,29 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         if (threadIdx.x == 0) {
             ctl->v[m] = v;
             ctl->forced[m] = forced;
+            ctl->tv[m] = v;
+            ctl->tforced[m] = kNoColumn;
             if (bad) give_up = 1;
         }
         __syncthreads();
     }
+    if (mini) {
+        // list passes rest until the next full pass once every screened window is full and nothing in it was refuted, or
+        // when the reports overflowed (the full pass has to sort that out)
+        if (threadIdx.x == 0 && give_up) ctl->mini_done = 1;
+        if (threadIdx.x == 0 && !any_failed && !give_up) {
+            bool full = true;
+            for (int m = 0; m < 2; ++m) {
+                if (ctl->finished[m]) continue;
+                const int base = ctl->base[m], hi = ctl->hi[m];
+                if (!(hi - base >= a.half_n || hi >= s || ctl->dep[m] || ctl->extra[m])) full = false;
+            }
+            if (full) ctl->mini_done = 1;
+        }
+        return;
+    }
     if (threadIdx.x == 0) {
+        ctl->mini_done = 0;
         if (give_up) {
             ctl->fallback = 1; ctl->round_active = 0;
             atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
@@ -1263,8 +1355,13 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
 }
 
 // start of the recovery of one step
-__global__ void k_spec_init(SpecCtl* ctl, int speculate) {
+__global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau) {
     if (threadIdx.x == 0) {
+        ctl->tv[0] = ctl->tv[1] = 0;
+        ctl->tforced[0] = ctl->tforced[1] = kNoColumn;
+        ctl->mini_done = 0; ctl->list_rounds = 0; ctl->list_refuted = 0;
+        // no wide list unless a long-list speculation asks for one
+        if (wide_tau != nullptr) for (int g = 0; g < kPassMaxN / 8; ++g) wide_tau[g] = __int_as_float(0x7f800000);
         ctl->round_active = speculate; ctl->fallback = speculate ? 0 : 1;
         ctl->v[0] = ctl->v[1] = 0;
         ctl->forced[0] = ctl->forced[1] = kNoColumn;
@@ -1304,7 +1401,8 @@ k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uin
               const uint32_t* kept_ring, int* rounds_out) {
     __shared__ int n_s;
     // how many rounds this step took (the enqueued rounds if even they were not enough): sizes the next step's launches
-    if (threadIdx.x == 0) *rounds_out = ctl->fallback ? kMaxRounds : ctl->rounds;
+    // bit 8: a list pass refuted a pick (the wide lists earned their keep)
+    if (threadIdx.x == 0) *rounds_out = (ctl->fallback ? kMaxRounds : ctl->rounds) | (ctl->list_refuted > 0 ? 256 : 0);
     int n = ctl->n_cand;
     // rebuild from the supports and the ring of kept index sets when the list has outgrown its bound, or when it holds
     // far more than those although a single round confirmed every pick (harvested columns of an earlier cold start)
@@ -1412,6 +1510,8 @@ OmpArgs make_args(const sgc_state* st) {
     a.rt = st->rt; a.tau = st->tau; a.inv_scale = st->inv_scale; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
     a.cand_list = st->cand_list;
     a.zlist = st->zlist; a.gram = st->gram; a.p0 = st->p0; a.pick_li = st->pick_li;
+    a.wide_tau = st->wide_tau; a.z_wide = st->z_wide; a.wide_count = nullptr; a.wide_bits = st->wide_bits; a.mini = 0;
+    a.depth = 1 << 30;
     return a;
 }
 
@@ -1451,6 +1551,7 @@ cudaError_t configure_recover(sgc_state* st) {
     st->pass_n = 2 * half;
     st->z_harvest = normal_tail_threshold((double)st->d, 3072.0);
     st->z_floor = normal_tail_threshold((double)st->d, 6144.0);
+    st->z_wide = normal_tail_threshold((double)st->d, 100000.0);
     if (st->spec_ok) {
         e = pass_configure(kPassMaxN);
         if (e != cudaSuccess) return e;
@@ -1494,7 +1595,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
         args[i] = a;
         {
             PhaseTimer timer(st, stream, kPhaseBook, 1);
-            k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0);
+            k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0, st->wide_tau);
             *launches += 1;
             if (speculate) {
                 k_cand_begin<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->sel_idx, st->s, st->kept_ring, st->hist_slots,
@@ -1504,13 +1605,56 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
         }
         // rounds to enqueue: twice what the last finished step needed plus slack (read from pinned memory without
         // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
-        const int last = speculate ? *reinterpret_cast<volatile int*>(st->h_rounds) : 0;
+        const int hint = speculate ? *reinterpret_cast<volatile int*>(st->h_rounds) : 0;
+        const int last = hint & 255;
         const int want = last <= 0 ? 8 : 2 * last + 4;
         if (want > n_rounds) n_rounds = want;
+        // two-level screening pays where steps need several full passes (recovery picks columns outside the kept sets);
+        // it is dropped again when a step needed one pass and its list passes refuted nothing
+        if (last >= 3) st->two_level = true;
+        else if (last == 1 && !(hint & 256)) st->two_level = false;
     }
     if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
+    const bool two_level = speculate && n == 1 && st0->two_level;
+    PassWide wide;
+    if (two_level) {
+        args[0].wide_count = st0->wide_count;
+        wide.tau = st0->wide_tau; wide.list = st0->wide_list; wide.count = st0->wide_count; wide.bits = st0->wide_bits;
+        wide.cap = kWideCap; wide.half_n = st0->pass_n / 2; wide.ctl = st0->ctl; wide.list_pass = false;
+    }
     if (speculate) {
         for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
+            // list passes first: speculate a few picks ahead, screen the wide lists only, keep what they confirm as
+            // tentative picks; every kernel of this loop returns at once when there is nothing (more) to do
+            for (int mini = 0; two_level && mini < kMiniRounds && e == cudaSuccess; ++mini) {
+                sgc_state* st = st0;
+                {
+                    PhaseTimer timer(st, stream, kPhaseCorr, 1);
+                    OmpArgs am = args[0];
+                    am.mini = 1; am.depth = kMiniDepth;
+                    e = launch_omp(st, am, 0, stream);
+                    *launches += 1;
+                }
+                if (e != cudaSuccess) break;
+                {
+                    PhaseTimer timer(st, stream, kPhasePass, 1);
+                    const int* gates[kPassMaxBatch] = {&st->ctl->round_active};
+                    int* errors[kPassMaxBatch] = {&st->ctl->pass_error};
+                    PassWide lp = wide;
+                    lp.list_pass = true;
+                    e = launch_pass(st->tmap[0], st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale,
+                                    st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp);
+                    *launches += 1;
+                }
+                if (e != cudaSuccess) break;
+                ResolveArgs ra;
+                ra.o = args[0];
+                ra.rep = st->rep; ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list;
+                ra.rtmp = st->rtmp; ra.kept_ring = st->kept_ring; ra.mini = 1; ra.wide_count = st->wide_count;
+                PhaseTimer timer(st, stream, kPhaseBook, 1);
+                k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
+                *launches += 1;
+            }
             for (int b0 = 0; b0 < n && e == cudaSuccess; b0 += per_batch) {
                 const int nb = n - b0 < per_batch ? n - b0 : per_batch;
                 for (int i = b0; i < b0 + nb && e == cudaSuccess; ++i) {
@@ -1537,7 +1681,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     }
                     e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
                                     lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
-                                    lead->sm_count, stream);
+                                    lead->sm_count, stream, two_level ? &wide : nullptr);
                     *launches += 1;
                 }
                 for (int i = b0; i < b0 + nb && e == cudaSuccess; ++i) {
@@ -1546,7 +1690,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     ra.o = args[i];
                     ra.rep = lead->rep + (size_t)(i - b0) * st->pass_n * kRepCap;
                     ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list; ra.rtmp = st->rtmp;
-                    ra.kept_ring = st->kept_ring;
+                    ra.kept_ring = st->kept_ring; ra.mini = 0; ra.wide_count = st->wide_count;
                     PhaseTimer timer(st, stream, kPhaseBook, 1);
                     k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
                     *launches += 1;

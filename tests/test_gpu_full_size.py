@@ -96,7 +96,7 @@ def run_config(sgc, d, k, s, seed, cfg_id, steps, planted, full_oracle_picks=0, 
         assert np.array_equal(st.get("sel_val"), ref.get("sel_val"))
         for name in ("p", "q", "M", "V"):
             assert rel(st.get(name), ref.get(name)) < TOL_STATE, name
-        rounds.append((int(st.get("rounds")), int(st.get("fallback"))))
+        rounds.append((int(st.get("rounds")), int(st.get("fallback")), int(st.get("list_rounds"))))
         seen |= set(ref.get("sel_idx").tolist())
         targets = dict(M=ref.get("Mhat"), V=ref.get("Vhat"))
         rec = {}
@@ -150,7 +150,7 @@ def sgc():
 def test_config2_full_size(sgc):
     # 4096 x 4096, k = 2048, s = 64, seed 1: the benchmark's workload; exact-recovery regime
     rounds, status = run_config(sgc, 4096 * 4096, 2048, 64, 1, 2, steps=3, planted=True, full_oracle_picks=1)
-    assert all(fb == 0 for _, fb in rounds), rounds
+    assert all(fb == 0 for _, fb, _ in rounds), rounds
     assert rounds[-1][0] == 1, rounds            # warm candidate list: one screening pass per step
     assert not status & (sgc.STATUS_CANDIDATE_OVERFLOW | sgc.STATUS_SELECT_FALLBACK)
 
@@ -159,6 +159,14 @@ def test_config2_full_size(sgc):
 def test_config3_shapes_full_size(sgc, rows, cols):
     # one Llama-2-7B layer: k = 2048, s = 128 per matrix (recovery is inexact here: noise columns get picked)
     run_config(sgc, rows * cols, 2048, 128, 1, 3, steps=2, planted=False)
+
+
+def test_config3_two_level_screening_full_size(sgc):
+    # enough steps for the wide lists and the list passes to come into play (they start once a step needed three passes)
+    rounds, status = run_config(sgc, 4096 * 4096, 2048, 128, 1, 3, steps=5, planted=False)
+    assert all(fb == 0 for _, fb, _ in rounds), rounds
+    assert sum(lr for _, _, lr in rounds) > 0, rounds
+    assert not status & sgc.STATUS_CANDIDATE_OVERFLOW
 
 
 def test_config4_matrix_full_size(sgc):

@@ -105,7 +105,7 @@ def test_select_flags_non_finite_input(sgc):
 
 # ---- whole step, config-1 shape and relatives -------------------------------------------------------------
 def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_support=False, compare_every=1, mode=None,
-             stats=None):
+             stats=None, list_rounds=None):
     hp = inputs.ADAM
     st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha)
     if mode is not None:
@@ -126,6 +126,8 @@ def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_suppo
         assert st.get("t") == step == ref.get("t")
         if stats is not None:
             stats.append((int(st.get("rounds")), int(st.get("fallback")), int(st.get("n_cand"))))
+        if list_rounds is not None:
+            list_rounds.append(int(st.get("list_rounds")))
         assert np.array_equal(st.get("sel_idx"), ref.get("sel_idx"))
         assert np.array_equal(st.get("sel_val"), ref.get("sel_val"))
         for name in ("p", "q", "M", "V"):
@@ -186,6 +188,17 @@ def test_speculative_recovery_with_redrawn_supports_and_alpha(sgc):
     stats = []
     run_both(sgc, 150_000, 256, 8, 11, "student", 5, cfg_id=2, alpha=2.0, redraw_support=True, mode=2, stats=stats)
     assert all(fb == 0 for _, fb, _ in stats), stats
+
+
+@pytest.mark.parametrize("d,k,s,steps", [(400_000, 256, 48, 7), (1_000_000, 512, 100, 4)])
+def test_two_level_screening_matches_the_oracle(sgc, d, k, s, steps):
+    # inexact regime (supports redrawn every step, k small): steps need several passes over all columns, which switches
+    # on the wide lists and the list passes between full passes; the picks must not depend on any of that
+    stats, lists = [], []
+    run_both(sgc, d, k, s, 21, "student", steps, cfg_id=2, redraw_support=True, mode=2, stats=stats, list_rounds=lists)
+    assert all(fb == 0 for _, fb, _ in stats), stats
+    assert max(r for r, _, _ in stats) >= 3, stats               # the regime this test is about
+    assert sum(lists) > 0, (stats, lists)                        # list passes ran and were resolved
 
 
 def test_speculative_and_lockstep_agree_bit_for_bit_on_supports(sgc):
