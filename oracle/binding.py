@@ -58,6 +58,13 @@ def lib():
             L.orc_adam.argtypes = [f32p, f32p, f64p, f64p, C.c_int32, C.c_float, C.c_float, C.c_int64, f64p, f64p]
             L.orc_omp.restype = C.c_int32
             L.orc_omp.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32, f64p, u32p, f64p, f64p, f64p, f64p]
+            L.orc_omp_tol.restype = C.c_int32
+            L.orc_omp_tol.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32, f64p, C.c_double, u32p, f64p, f64p, f64p,
+                                      f64p]
+            L.orc_least_squares.restype = C.c_int32
+            L.orc_least_squares.argtypes = [C.c_uint64, C.c_int32, u32p, C.c_int32, f64p, f64p]
+            L.orc_set_recovery.restype = None
+            L.orc_set_recovery.argtypes = [C.c_void_p, C.c_int32, C.c_double]
             L.orc_combine_scatter.restype = C.c_int32
             L.orc_combine_scatter.argtypes = [u32p, f64p, C.c_int32, u32p, f64p, C.c_int32, C.c_float, C.c_float,
                                               C.c_float, f32p, u32p, f64p, i32p, i32p]
@@ -138,8 +145,11 @@ def adam(M, V, p, q, beta1, beta2, t):
     return Mh, Vh
 
 
-def omp(seed, d, k, s, y):
-    """Textbook OMP of y against A(seed, k x d).  Returns a dict of per-iteration records."""
+def omp(seed, d, k, s, y, residual_tol=0.0):
+    """Textbook OMP of y against A(seed, k x d).  Returns a dict of per-iteration records.
+
+    residual_tol > 0 ends the iterations once ||r|| <= residual_tol * ||y|| (an opt-in variant; 0 = Algorithm 3's s
+    iterations)."""
     y = np.ascontiguousarray(y, dtype=np.float64)
     assert y.size == k
     lam = np.empty(s, dtype=np.uint32)
@@ -147,9 +157,21 @@ def omp(seed, d, k, s, y):
     t1 = np.empty(s, dtype=np.float64)
     t2 = np.empty(s, dtype=np.float64)
     rn = np.empty(s, dtype=np.float64)
-    done = lib().orc_omp(C.c_uint64(seed), d, k, s, _p(y, C.c_double), _p(lam, C.c_uint32), _p(x, C.c_double),
-                         _p(t1, C.c_double), _p(t2, C.c_double), _p(rn, C.c_double))
+    done = lib().orc_omp_tol(C.c_uint64(seed), d, k, s, _p(y, C.c_double), float(residual_tol), _p(lam, C.c_uint32),
+                             _p(x, C.c_double), _p(t1, C.c_double), _p(t2, C.c_double), _p(rn, C.c_double))
     return dict(done=int(done), lam=lam, x=x, top1=t1, top2=t2, rnorm=rn)
+
+
+def least_squares(seed, k, lam, y):
+    """argmin_x ||y - A_lam x||_2 for the columns lam of A(seed, k x .): the last step of an OMP iteration on its own."""
+    lam = np.ascontiguousarray(lam, dtype=np.uint32)
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    assert y.size == k
+    x = np.zeros(lam.size, dtype=np.float64)
+    rc = lib().orc_least_squares(C.c_uint64(seed), k, _p(lam, C.c_uint32), lam.size, _p(y, C.c_double), _p(x, C.c_double))
+    if rc != 0:
+        raise ValueError("dependent columns")
+    return x
 
 
 def combine_scatter(lamM, xM, lamV, xV, alpha, eps, lr, W):
@@ -216,6 +238,10 @@ class Oracle:
     def step(self, grad, weight):
         self.step_compress(grad)
         self.step_recover(weight)
+
+    def set_recovery(self, shared_support, residual_tol=0.0):
+        """Opt-in variant: one support (that of OMP_A(M^)) for both moments, and / or an early stop on ||r||."""
+        lib().orc_set_recovery(self._h, 1 if shared_support else 0, float(residual_tol))
 
     def reproject(self, new_seed):
         """SGCA (Algorithm 4, lines 9-12): M <- A' OMP_A(M), V <- A' OMP_A(V), A <- A' with A' named by new_seed."""

@@ -263,9 +263,15 @@ void orc_adam(float* M, float* V, const double* p, const double* q, int32_t k,
 // x = least-squares coefficients aligned with lam (final support), top1/top2 = best and
 // second-best normalised correlation at each iteration, rnorm = ||r|| AFTER each iteration.
 // Returns the number of completed iterations (< s only on a dependent column).
-int32_t orc_omp(uint64_t seed, int64_t d, int32_t k, int32_t s, const double* y,
-                uint32_t* lam, double* x, double* top1, double* top2, double* rnorm) {
+//
+// orc_omp_tol is the same recovery with an optional early stop (not in Algorithm 3, which always runs s iterations):
+// with residual_tol > 0 the iterations end after the first one that leaves ||r|| <= residual_tol * ||y||.
+int32_t orc_omp_tol(uint64_t seed, int64_t d, int32_t k, int32_t s, const double* y, double residual_tol,
+                    uint32_t* lam, double* x, double* top1, double* top2, double* rnorm) {
     const double sigma = (double)sigma_of_k(k);
+    double ynorm = 0.0;
+    for (int32_t row = 0; row < k; ++row) ynorm += y[row] * y[row];
+    ynorm = std::sqrt(ynorm);
     std::vector<double> r(y, y + k);
     std::vector<double> cols;            // selected columns of A, column-major k x j
     std::vector<uint8_t> taken((size_t)d, 0);
@@ -342,9 +348,27 @@ int32_t orc_omp(uint64_t seed, int64_t d, int32_t k, int32_t s, const double* y,
         rnorm[it] = std::sqrt(rn);
         for (int32_t c = 0; c < j; ++c) x[c] = xs[c];
         done = j;
+        if (residual_tol > 0.0 && rnorm[it] <= residual_tol * ynorm) break;
     }
     for (int32_t c = done; c < s; ++c) { lam[c] = 0xFFFFFFFFu; x[c] = 0.0; top1[c] = top2[c] = rnorm[c] = 0.0; }
     return done;
+}
+
+int32_t orc_omp(uint64_t seed, int64_t d, int32_t k, int32_t s, const double* y,
+                uint32_t* lam, double* x, double* top1, double* top2, double* rnorm) {
+    return orc_omp_tol(seed, d, k, s, y, 0.0, lam, x, top1, top2, rnorm);
+}
+
+// Least squares of y on a given support: x = argmin ||y - A_Lambda x||_2 (the last step of every OMP iteration, on
+// its own).  The columns must be independent, as the picks of an OMP run are; returns 0, or -1 on an exactly zero pivot.
+int32_t orc_least_squares(uint64_t seed, int32_t k, const uint32_t* lam, int32_t n, const double* y, double* x) {
+    const double sigma = (double)sigma_of_k(k);
+    std::vector<double> cols((size_t)n * k);
+    for (int32_t c = 0; c < n; ++c) {
+        const uint32_t ck = column_key(seed, lam[c]);
+        for (int32_t row = 0; row < k; ++row) cols[(size_t)c * k + row] = a_entry(ck, (uint32_t)row, sigma);
+    }
+    return least_squares_qr(cols, std::vector<double>(y, y + k), k, n, x) ? 0 : -1;
 }
 
 // ---- a5: N = alpha x^M / (sqrt(x^V) + eps) on the common support; W <- W - eta N (Eq. 8, Eq. 3) ---
@@ -385,6 +409,8 @@ struct orc_state {
     std::vector<uint32_t> lamM, lamV; std::vector<double> xM, xV, top1M, top2M, top1V, top2V, rnM, rnV;
     int32_t doneM, doneV, n_upd, mismatch, negv;
     std::vector<uint32_t> upd_idx; std::vector<double> upd_val;
+    // opt-in variant of the recovery (orc_set_recovery)
+    int32_t shared_support; double residual_tol;
 };
 
 orc_state* orc_create(int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, float beta1, float beta2, float eps) {
@@ -399,10 +425,18 @@ orc_state* orc_create(int64_t d, int32_t k, int32_t s, uint64_t seed, float lr, 
     st->top1M.resize(s); st->top2M.resize(s); st->top1V.resize(s); st->top2V.resize(s);
     st->rnM.resize(s); st->rnV.resize(s); st->upd_idx.resize(s); st->upd_val.resize(s);
     st->doneM = st->doneV = st->n_upd = st->mismatch = st->negv = 0;
+    st->shared_support = 0; st->residual_tol = 0.0;
     return st;
 }
 void orc_destroy(orc_state* st) { delete st; }
 void orc_set_alpha(orc_state* st, float alpha) { st->alpha = alpha; }
+// Opt-in variant built on the remark after Eq. (8) that OMP_A(M) and OMP_A(V) have the same non-zero positions:
+// shared_support = 1: OMP_A(M^) alone selects the support; x^V is the least-squares fit of V^ on that support.
+// residual_tol > 0: a recovery ends early once ||r|| <= residual_tol * ||y|| (see orc_omp_tol).
+// The defaults (0, 0.0) are Algorithm 2 as printed.
+void orc_set_recovery(orc_state* st, int32_t shared_support, double residual_tol) {
+    st->shared_support = shared_support; st->residual_tol = residual_tol;
+}
 
 // Steps a1-a3 only (cheap); used when the recovery is sampled.
 void orc_step_compress(orc_state* st, const float* grad) {
@@ -414,10 +448,19 @@ void orc_step_compress(orc_state* st, const float* grad) {
 }
 // Steps a4-a5 on the state left by orc_step_compress.
 void orc_step_recover(orc_state* st, float* weight) {
-    st->doneM = orc_omp(st->seed, st->d, st->k, st->s, st->Mhat.data(), st->lamM.data(), st->xM.data(),
-                        st->top1M.data(), st->top2M.data(), st->rnM.data());
-    st->doneV = orc_omp(st->seed, st->d, st->k, st->s, st->Vhat.data(), st->lamV.data(), st->xV.data(),
-                        st->top1V.data(), st->top2V.data(), st->rnV.data());
+    st->doneM = orc_omp_tol(st->seed, st->d, st->k, st->s, st->Mhat.data(), st->residual_tol, st->lamM.data(),
+                            st->xM.data(), st->top1M.data(), st->top2M.data(), st->rnM.data());
+    if (st->shared_support) {
+        // one support for both moments: the columns OMP_A(M^) selected, in its order
+        for (int32_t c = 0; c < st->s; ++c) {
+            st->lamV[c] = st->lamM[c]; st->xV[c] = 0.0; st->top1V[c] = st->top2V[c] = st->rnV[c] = 0.0;
+        }
+        st->doneV = st->doneM;
+        if (st->doneM > 0) orc_least_squares(st->seed, st->k, st->lamM.data(), st->doneM, st->Vhat.data(), st->xV.data());
+    } else {
+        st->doneV = orc_omp_tol(st->seed, st->d, st->k, st->s, st->Vhat.data(), st->residual_tol, st->lamV.data(),
+                                st->xV.data(), st->top1V.data(), st->top2V.data(), st->rnV.data());
+    }
     st->n_upd = orc_combine_scatter(st->lamM.data(), st->xM.data(), st->doneM, st->lamV.data(), st->xV.data(),
                                     st->doneV, st->alpha, st->eps, st->lr, weight, st->upd_idx.data(),
                                     st->upd_val.data(), &st->mismatch, &st->negv);
@@ -436,10 +479,18 @@ void orc_reproject(orc_state* st, uint64_t new_seed) {
     std::vector<double> y((size_t)k), x((size_t)s), t1((size_t)s), t2((size_t)s), rn((size_t)s), out((size_t)k), unused((size_t)k);
     std::vector<uint32_t> lam((size_t)s);
     std::vector<float> val((size_t)s);
+    int32_t done = 0;
     for (int pass = 0; pass < 2; ++pass) {
         std::vector<float>& state = pass == 0 ? st->M : st->V;
         for (int32_t j = 0; j < k; ++j) y[j] = (double)state[j];
-        const int32_t done = orc_omp(st->seed, st->d, k, s, y.data(), lam.data(), x.data(), t1.data(), t2.data(), rn.data());
+        if (pass == 1 && st->shared_support) {
+            // the variant of orc_set_recovery: V is fitted on the support found for M
+            for (int32_t l = 0; l < s; ++l) x[l] = 0.0;
+            if (done > 0) orc_least_squares(st->seed, k, lam.data(), done, y.data(), x.data());
+        } else {
+            done = orc_omp_tol(st->seed, st->d, k, s, y.data(), st->residual_tol, lam.data(), x.data(), t1.data(), t2.data(),
+                               rn.data());
+        }
         // A' x with x supported on the recovered columns: sum in fp64 in the order of selection
         for (int32_t j = 0; j < k; ++j) out[j] = 0.0;
         const double sigma = (double)sigma_of_k(k);

@@ -161,3 +161,95 @@ def test_create_rejects_bad_arguments():
     for (d, k, s) in [(0, 4, 1), (10, 0, 1), (10, 4, 0), (10, 4, 5), (3, 8, 4), (1 << 32, 8, 4)]:
         with pytest.raises(ValueError):
             oracle.Oracle(d, k, s, 0, 1e-3, 0.9, 0.999, 1e-8)
+
+
+# ---- opt-in variant: shared support and early stop (remark after Eq. (8)) -----------------------------------
+def test_least_squares_on_a_support_is_numpy_lstsq():
+    seed, d, k = 3, 1000, 96
+    rng = np.random.default_rng(8)
+    lam = rng.choice(d, size=7, replace=False).astype(np.uint32)
+    y = rng.standard_normal(k)
+    A = dense_A(seed, k, d)
+    want, *_ = np.linalg.lstsq(A[:, lam.astype(np.int64)], y, rcond=None)
+    np.testing.assert_allclose(oracle.least_squares(seed, k, lam, y), want, rtol=1e-10, atol=1e-12)
+
+
+def test_early_stop_ends_at_the_sparsity_of_an_exactly_sparse_target():
+    # y has 5 non-zeros in the A-basis; with k this large OMP finds them in 5 picks and the residual drops to rounding
+    # noise, so a tolerance of 1e-9 stops there, while tolerance 0 runs all s iterations (Algorithm 3 as printed)
+    seed, d, k, s, s0 = 17, 3000, 400, 12, 5
+    rng = np.random.default_rng(3)
+    supp = rng.choice(d, size=s0, replace=False)
+    A = dense_A(seed, k, d)
+    y = A[:, supp] @ rng.uniform(1.0, 2.0, size=s0)
+    full = oracle.omp(seed, d, k, s, y)
+    early = oracle.omp(seed, d, k, s, y, residual_tol=1e-9)
+    assert full["done"] == s and early["done"] == s0
+    assert np.array_equal(early["lam"][:s0], full["lam"][:s0]) and sorted(early["lam"][:s0].tolist()) == sorted(supp.tolist())
+    assert np.all(early["lam"][s0:] == 0xFFFFFFFF) and np.all(early["x"][s0:] == 0.0)
+    # a tolerance the first residual already meets stops after one pick; the stop never changes the picks made before it
+    one = oracle.omp(seed, d, k, s, y, residual_tol=1.0)
+    assert one["done"] == 1 and one["lam"][0] == full["lam"][0]
+    # the coefficients at the stop are the least-squares fit on the picks made so far
+    np.testing.assert_allclose(early["x"][:s0], oracle.least_squares(seed, k, early["lam"][:s0], y), rtol=1e-9)
+
+
+def test_shared_support_step_against_its_definition():
+    # noisy gradients: the two printed recoveries pick different columns late on; the variant keeps OMP_A(M^)'s picks
+    # for both moments and fits V^ on them by least squares (numpy restatement), then applies Eq. (8) on that support
+    d, k, s, seed = 1500, 128, 10, 9
+    lr, eps, alpha = np.float32(1e-3), np.float32(1e-8), 2.0
+    rng = np.random.default_rng(31)
+    plain = oracle.Oracle(d, k, s, seed, lr, 0.9, 0.999, eps, alpha=alpha)
+    var = oracle.Oracle(d, k, s, seed, lr, 0.9, 0.999, eps, alpha=alpha)
+    var.set_recovery(True)
+    A = dense_A(seed, k, d)
+    Wp = rng.standard_normal(d).astype(np.float32)
+    Wv = Wp.copy()
+    differed = False
+    for _ in range(4):
+        g = (rng.standard_t(3.0, size=d) * 1e-2).astype(np.float32)
+        W_before = Wv.copy()
+        plain.step(g, Wp)
+        var.step(g, Wv)
+        # a1-a3 and the recovery of M^ do not depend on the variant
+        for name in ("sel_idx", "M", "V", "lamM", "xM", "Mhat", "Vhat"):
+            assert np.array_equal(plain.get(name), var.get(name)), name
+        lam = var.get("lamM").astype(np.int64)
+        assert np.array_equal(var.get("lamV"), var.get("lamM")) and var.get("doneV") == var.get("doneM") == s
+        want, *_ = np.linalg.lstsq(A[:, lam], var.get("Vhat"), rcond=None)
+        np.testing.assert_allclose(var.get("xV"), want, rtol=1e-8, atol=1e-14)
+        differed |= sorted(plain.get("lamV").tolist()) != sorted(lam.tolist())
+        # Eq. (8) on the one support, guarded where x^V <= 0
+        xM, xV = var.get("xM"), var.get("xV")
+        ok = xV > 0
+        assert var.get("mismatch") == 0 and var.get("negv") == int((~ok).sum()) and var.get("n_upd") == int(ok.sum())
+        expect = W_before.astype(np.float64)
+        expect[lam[ok]] -= np.float64(lr) * alpha * xM[ok] / (np.sqrt(xV[ok]) + np.float64(eps))
+        np.testing.assert_allclose(Wv, expect.astype(np.float32), rtol=0, atol=1e-7)
+    assert differed          # otherwise this test would not tell the variant from Algorithm 2 as printed
+    plain.close()
+    var.close()
+
+
+def test_shared_support_equals_the_printed_algorithm_when_the_supports_coincide():
+    # constant exactly sparse gradient: both printed recoveries return the planted support (the premise of the remark after
+    # Eq. (8)), so the variant must reproduce the printed step up to the order in which x^V is listed
+    d, k, s, seed = 2048, 256, 6, 21
+    rng = np.random.default_rng(4)
+    supp = np.sort(rng.choice(d, size=s, replace=False))
+    g = np.zeros(d, dtype=np.float32)
+    g[supp] = (rng.uniform(1.0, 2.0, size=s) * rng.choice([-1.0, 1.0], size=s)).astype(np.float32)
+    a = oracle.Oracle(d, k, s, seed, 1e-3, 0.9, 0.999, 1e-8)
+    b = oracle.Oracle(d, k, s, seed, 1e-3, 0.9, 0.999, 1e-8)
+    b.set_recovery(True, 0.0)
+    Wa = rng.standard_normal(d).astype(np.float32)
+    Wb = Wa.copy()
+    for _ in range(3):
+        a.step(g, Wa)
+        b.step(g, Wb)
+        assert np.array_equal(a.get("upd_idx"), b.get("upd_idx"))
+        np.testing.assert_allclose(b.get("upd_val"), a.get("upd_val"), rtol=1e-9)
+        np.testing.assert_allclose(Wb, Wa, rtol=0, atol=1e-9)
+    a.close()
+    b.close()
