@@ -158,6 +158,18 @@ SGC_API int sgc_reproject(sgc_state* st, uint64_t new_seed, void* stream);
  * SGC_ERR_DIM when SGC_MODE_SPECULATIVE is requested and k is not a multiple of 64. */
 SGC_API int sgc_set_mode(sgc_state* st, int32_t mode);
 
+/* Opt-in variant of the recovery, built on the remark after Eq. (8) that OMP_A(M_t) and OMP_A(V_t) have their
+ * non-zeros at the same positions.  The default (0, 0.0) is Algorithm 2 as printed: two independent recoveries of s
+ * iterations each.
+ *   shared_support  1: only OMP_A(M^) selects columns; x^V is the least-squares fit of V^ on those columns (same
+ *                   order), so both supports are equal by construction and Eq. (8) applies on all of it where
+ *                   x^V > 0.  The per-iteration residual norms of V^ (SGC_GET_RNORM_V) are not recorded (zeros).
+ *   residual_tol    > 0: a recovery ends after the first iteration that leaves ||r|| <= residual_tol * ||y||
+ *                   (fewer than s picks; SGC_GET_DONE_* tell how many).  The picks made before the stop are those of
+ *                   Algorithm 3; the coefficients are the least-squares fit on them.  Must be finite and >= 0.
+ * Takes effect from the next step; sgc_reproject reuses whatever the last step recovered. */
+SGC_API int sgc_set_recovery(sgc_state* st, int32_t shared_support, double residual_tol);
+
 /* Synchronises with the state's last step and copies one record to host memory (selectors above).
  *   dst    host pointer; bytes = its capacity, must cover the record */
 SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes);

@@ -14,7 +14,7 @@ _lib = None
 
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
            "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
-           "sgc_set_mode", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version"]
+           "sgc_set_mode", "sgc_set_recovery", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -82,6 +82,8 @@ def lib():
         L.sgc_z_block.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, vp, vp]
         L.sgc_set_mode.restype = C.c_int
         L.sgc_set_mode.argtypes = [vp, C.c_int32]
+        L.sgc_set_recovery.restype = C.c_int
+        L.sgc_set_recovery.argtypes = [vp, C.c_int32, C.c_double]
         L.sgc_reproject.restype = C.c_int
         L.sgc_reproject.argtypes = [vp, C.c_uint64, vp]
         L.sgc_screen.restype = C.c_int
@@ -182,6 +184,10 @@ class Sgc:
 
     def set_mode(self, mode):
         _check(lib().sgc_set_mode(self._h, int(mode)), "sgc_set_mode")
+
+    def set_recovery(self, shared_support, residual_tol=0.0):
+        """Opt-in variant: one support (that of OMP_A(M^)) for both moments, and / or an early stop on ||r||."""
+        _check(lib().sgc_set_recovery(self._h, 1 if shared_support else 0, float(residual_tol)), "sgc_set_recovery")
 
     def reproject(self, new_seed, stream=None):
         """SGCA: switch to the matrix named by new_seed and re-align M, V with it (after the step of an iteration t = 0 mod T)."""

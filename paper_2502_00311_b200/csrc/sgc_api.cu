@@ -213,6 +213,14 @@ SGC_API int sgc_set_mode(sgc_state* st, int32_t mode) {
     return SGC_OK;
 }
 
+SGC_API int sgc_set_recovery(sgc_state* st, int32_t shared_support, double residual_tol) {
+    if (!st) return SGC_ERR_NULL;
+    if ((shared_support != 0 && shared_support != 1) || !(residual_tol >= 0.0) || !isfinite(residual_tol)) return SGC_ERR_WHAT;
+    st->shared_support = shared_support;
+    st->residual_tol = residual_tol;
+    return SGC_OK;
+}
+
 SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
     if (!st || !dst) return SGC_ERR_NULL;
     const size_t k = (size_t)st->k, s = (size_t)st->s;

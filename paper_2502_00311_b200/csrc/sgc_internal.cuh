@@ -180,11 +180,15 @@ struct sgc_state {
     int32_t last_launches; bool stepped;
     int corr_grid, corr_smem;
     int mode;                   // 0 auto, 1 lock-step only, 2 speculative whenever k allows it
+    int shared_support;         // 1: OMP(M^) alone selects, V^ is fitted on its support (sgc_set_recovery)
+    double residual_tol;        // > 0: recoveries are cut at the first pick that leaves ||r|| <= residual_tol ||y||
     bool spec_ok;               // speculative recovery usable for this (d, k)
     int pass_n;                 // residuals per screening pass (multiple of 32, <= 256); pass_n / 2 per residual stream
     double z_harvest, z_floor;  // thresholds of the screening pass in units of ||r|| / sqrt(k)
     double z_wide;              // threshold of the wide lists, same units
     unsigned char tmap[8][128]; // CUtensorMaps of the residual matrix R^T, one per number of states batched into a pass
+    unsigned char tmap_half[128]; // the same for a pass over the first stream's residuals alone (shared-support variant)
+    int pass_n_half;            // its width: pass_n / 2 rounded up to a multiple of 32
     // optional per-kernel timing (sgc_set_profile)
     bool profile;
     std::vector<cudaEvent_t>* ev_pool; size_t ev_used;

@@ -1355,7 +1355,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
 }
 
 // start of the recovery of one step
-__global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau) {
+__global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau, int shared) {
     if (threadIdx.x == 0) {
         ctl->tv[0] = ctl->tv[1] = 0;
         ctl->tforced[0] = ctl->tforced[1] = kNoColumn;
@@ -1365,7 +1365,8 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau) {
         ctl->round_active = speculate; ctl->fallback = speculate ? 0 : 1;
         ctl->v[0] = ctl->v[1] = 0;
         ctl->forced[0] = ctl->forced[1] = kNoColumn;
-        ctl->finished[0] = ctl->finished[1] = 0;
+        ctl->finished[0] = 0;
+        ctl->finished[1] = shared ? 1 : 0;          // shared support: the second stream makes no picks of its own
         ctl->stop[0] = ctl->stop[1] = 0;
         ctl->rounds = 0; ctl->pass_error = 0;
         for (int r = 0; r < kMaxRounds; ++r) ctl->trace[r][0] = ctl->trace[r][1] = ctl->trace[r][2] = 0;
@@ -1427,6 +1428,78 @@ k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uin
         const int n_new = n_s < kCandCap ? n_s : kCandCap;
         if (n_new != ctl->n_cand || n == 0) ctl->list_version = ctl->list_version + 1;     // rebuilt or extended
         ctl->n_cand = n_new;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Opt-in variant of the recovery (remark after Eq. (8): both recoveries have their non-zeros at the same positions).
+// Runs after the recoveries of the step, one block.
+//   tol > 0: each recovery is cut after the first pick that left ||r|| <= tol ||y||.  OMP is greedy, so the picks before
+//            the cut are those an early-stopping run makes, and the leading block of the inverse Cholesky factor F with
+//            the leading coefficients a gives the least-squares fit on them: x = F_j a_j.
+//   shared:  the second stream made no picks; x^V = F F^T A_Lambda^T V^ is the least-squares fit of V^ on the support
+//            of the first stream (F F^T = (A_Lambda^T A_Lambda)^-1, Appendix B).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kOmpThreads, 1) k_variant_tail(OmpArgs a, int shared, double tol) {
+    __shared__ double red[32];
+    __shared__ double u[kMaxS], av[kMaxS];
+    __shared__ int cut;
+    const int k = a.k, s = a.s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (tol > 0.0) {
+        for (int m = 0; m < (shared ? 1 : 2); ++m) {
+            const double* y = a.y64 + (size_t)m * k;
+            double yn2 = 0.0;
+            for (int row = threadIdx.x; row < k; row += kOmpThreads) yn2 += y[row] * y[row];
+            yn2 = block_sum(yn2, red);
+            const int done = a.cnt->done[m];
+            if (threadIdx.x == 0) {
+                const double bound = tol * sqrt(yn2);
+                cut = done;
+                for (int j = 0; j < done; ++j) if (a.rnorm[(size_t)m * s + j] <= bound) { cut = j + 1; break; }
+            }
+            __syncthreads();
+            const int n = cut;
+            if (n < done) {
+                const double* F = a.F + (size_t)m * s * s;
+                const double* ac = a.acoef + (size_t)m * s;
+                for (int i = threadIdx.x; i < s; i += kOmpThreads) {
+                    double acc = 0.0;
+                    for (int l = i; l < n; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
+                    a.x[(size_t)m * s + i] = acc;                  // 0 for i >= n
+                    if (i >= n) a.rnorm[(size_t)m * s + i] = 0.0;
+                }
+                if (threadIdx.x == 0) a.cnt->done[m] = n;
+            }
+            __syncthreads();
+        }
+    }
+    if (shared) {
+        const int n = a.cnt->done[0];
+        const double* y = a.y64 + (size_t)k;                       // V^
+        const double* F = a.F;                                     // factor of the first stream's support
+        for (int l = warp; l < n; l += kOmpThreads / 32) {
+            const uint16_t* zl = a.zsel + (size_t)l * k;
+            double acc = 0.0;
+            for (int row = lane; row < k; row += 32) acc += (double)half_bits_to_float(zl[row]) * y[row];
+            acc = warp_sum(acc);
+            if (lane == 0) u[l] = a.sigma * acc;
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += kOmpThreads) {
+            double acc = 0.0;
+            for (int l = 0; l <= i; ++l) acc += F[(size_t)l * s + i] * u[l];
+            av[i] = acc;
+        }
+        __syncthreads();
+        for (int i = threadIdx.x; i < s; i += kOmpThreads) {
+            double acc = 0.0;
+            for (int l = i; l < n; ++l) acc += F[(size_t)i * s + l] * av[l];
+            a.x[(size_t)s + i] = acc;                              // 0 for i >= n
+            a.lam[(size_t)s + i] = i < n ? a.lam[i] : kNoColumn;
+            a.rnorm[(size_t)s + i] = 0.0;
+        }
+        if (threadIdx.x == 0) a.cnt->done[1] = n;
     }
 }
 
@@ -1565,6 +1638,10 @@ cudaError_t finish_recover_setup(sgc_state* st) {
     for (int g = 1; g <= kPassMaxN / st->pass_n && e == cudaSuccess; ++g)      // one map per number of states in a batch
         e = pass_encode_map(st->tmap[g - 1], st->rt, g * st->pass_n, st->k);
     if (e != cudaSuccess) return e;
+    // shared-support variant: only the first stream has residuals to screen, a pass half as wide does
+    st->pass_n_half = ((st->pass_n / 2 + 31) / 32) * 32;
+    e = pass_encode_map(st->tmap_half, st->rt, st->pass_n_half, st->k);
+    if (e != cudaSuccess) return e;
     e = launch_inv_norms(st->seed, (uint64_t)st->d, st->k, st->inv_norm, 0);     // column norms: a property of (seed, k)
     if (e != cudaSuccess) return e;
     return cudaDeviceSynchronize();
@@ -1595,7 +1672,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
         args[i] = a;
         {
             PhaseTimer timer(st, stream, kPhaseBook, 1);
-            k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0, st->wide_tau);
+            k_spec_init<<<1, 32, 0, stream>>>(st->ctl, speculate ? 1 : 0, st->wide_tau, st->shared_support);
             *launches += 1;
             if (speculate) {
                 k_cand_begin<<<1, kOmpThreads, 0, stream>>>(st->ctl, st->sel_idx, st->s, st->kept_ring, st->hist_slots,
@@ -1642,7 +1719,9 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     int* errors[kPassMaxBatch] = {&st->ctl->pass_error};
                     PassWide lp = wide;
                     lp.list_pass = true;
-                    e = launch_pass(st->tmap[0], st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale,
+                    const bool narrow = st->shared_support && st->pass_n_half < st->pass_n;
+                    e = launch_pass(narrow ? st->tmap_half : st->tmap[0], st->seed, (uint64_t)st->d, st->k,
+                                    narrow ? st->pass_n_half : st->pass_n, st->tau, st->inv_scale,
                                     st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp);
                     *launches += 1;
                 }
@@ -1679,7 +1758,9 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                         gates[q] = q < nb ? &sts[b0 + q]->ctl->round_active : nullptr;
                         errors[q] = q < nb ? &sts[b0 + q]->ctl->pass_error : nullptr;
                     }
-                    e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
+                    const bool narrow = nb == 1 && lead->shared_support && lead->pass_n_half < lead->pass_n;
+                    e = launch_pass(narrow ? lead->tmap_half : lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k,
+                                    narrow ? lead->pass_n_half : nb * lead->pass_n, lead->tau,
                                     lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
                                     lead->sm_count, stream, two_level ? &wide : nullptr);
                     *launches += 1;
@@ -1707,6 +1788,11 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
             *launches += 1;
         }
         if (e != cudaSuccess) return e;
+        if (st->shared_support || st->residual_tol > 0.0) {
+            PhaseTimer timer(st, stream, kPhaseBook, 1);
+            k_variant_tail<<<1, kOmpThreads, 0, stream>>>(args[i], st->shared_support, st->residual_tol);
+            *launches += 1;
+        }
         PhaseTimer timer(st, stream, kPhaseScatter, 1);
         k_scatter<<<1, kBookThreads, 0, stream>>>(st->s, st->lam, st->x, st->cnt, weights[i], st->upd_idx, st->upd_val,
                                                   (double)st->alpha, (double)st->eps, (double)st->lr);

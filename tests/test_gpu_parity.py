@@ -105,20 +105,23 @@ def test_select_flags_non_finite_input(sgc):
 
 # ---- whole step, config-1 shape and relatives -------------------------------------------------------------
 def run_both(sgc, d, k, s, seed, kind, steps, cfg_id=1, alpha=None, redraw_support=False, compare_every=1, mode=None,
-             stats=None, list_rounds=None):
+             stats=None, list_rounds=None, recovery=None, n_planted=None):
     hp = inputs.ADAM
     st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha)
     if mode is not None:
         st.set_mode(mode)
     ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=alpha or 1.0)
-    supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0))
+    if recovery is not None:                     # the opt-in variant, on both sides
+        st.set_recovery(*recovery)
+        ref.set_recovery(*recovery)
+    supp, sign = inputs.planted_support(d, n_planted or s, inputs.support_seed(cfg_id, 0))
     w0 = inputs.weights(d, 99)
     w_gpu = cuda(w0.copy())
     w_ref = w0.copy()
     worst = dict(p=0.0, q=0.0, M=0.0, V=0.0, upd=0.0, x=0.0)
     for step in range(1, steps + 1):
         if redraw_support:
-            supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, 0) + 7919 * step)
+            supp, sign = inputs.planted_support(d, n_planted or s, inputs.support_seed(cfg_id, 0) + 7919 * step)
         g = inputs.gradient(d, kind, supp, sign, inputs.step_seed(cfg_id, 0, step))
         w_before = w_ref.copy()
         st.step(cuda(g), w_gpu)
@@ -199,6 +202,48 @@ def test_two_level_screening_matches_the_oracle(sgc, d, k, s, steps):
     assert all(fb == 0 for _, fb, _ in stats), stats
     assert max(r for r, _, _ in stats) >= 3, stats               # the regime this test is about
     assert sum(lists) > 0, (stats, lists)                        # list passes ran and were resolved
+
+
+# ---- opt-in recovery variant: shared support, early stop (remark after Eq. (8)) ----------------------------------
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("d,k,s,kind,redraw", [(70_001, 320, 17, "student", True), (1 << 17, 512, 64, "student", False),
+                                               (4096, 256, 16, "gauss", False)])
+def test_shared_support_variant_matches_its_oracle(sgc, mode, d, k, s, kind, redraw):
+    # OMP(M^) alone selects; x^V is the least-squares fit of V^ on its support.  Redrawn supports make the two printed
+    # recoveries disagree, so this is not the printed algorithm in disguise.
+    if mode == 2 and k % 64:
+        pytest.skip("speculative recovery needs k to be a multiple of 64")
+    run_both(sgc, d, k, s, 5, kind, 4, cfg_id=2, mode=mode, redraw_support=redraw, recovery=(True, 0.0))
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("shared", [False, True])
+def test_early_stop_on_the_residual_matches_its_oracle(sgc, mode, shared):
+    # gradients with 10 non-zeros while s = 16: M^ and V^ are exactly 10-sparse in the A-basis, the residual falls to
+    # rounding noise after 10 picks, and a tolerance of 1e-6 ends both recoveries there on both sides (the later picks
+    # of an uncut run would be decided by that noise)
+    d, k, s = 50_000, 512, 16
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, 3, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    st.set_mode(mode)
+    st.set_recovery(shared, 1e-6)
+    run_both(sgc, d, k, s, 3, "zero", 3, cfg_id=2, mode=mode, recovery=(shared, 1e-6), n_planted=10)
+    # the cut is visible in the records
+    supp, sign = inputs.planted_support(d, 10, inputs.support_seed(2, 0))
+    w = cuda(inputs.weights(d, 99))
+    st.step(cuda(inputs.gradient(d, "zero", supp, sign, inputs.step_seed(2, 0, 1))), w)
+    assert st.get("doneM") == 10 == st.get("doneV")
+    assert sorted(st.get("lamM")[:10].tolist()) == sorted(supp.tolist()) and np.all(st.get("lamM")[10:] == 0xFFFFFFFF)
+    assert np.all(st.get("xM")[10:] == 0.0) and st.get("n_upd") == 10
+    st.close()
+
+
+def test_set_recovery_rejects_bad_arguments(sgc):
+    st = sgc.Sgc(4096, 64, 4, 1, 1e-3, 0.9, 0.999, 1e-8)
+    for args in [(2, 0.0), (0, -1.0), (1, float("nan")), (0, float("inf"))]:
+        assert sgc.lib().sgc_set_recovery(st._h, args[0], args[1]) != 0
+    assert sgc.lib().sgc_set_recovery(st._h, 1, 0.5) == 0
+    st.close()
 
 
 def test_speculative_and_lockstep_agree_bit_for_bit_on_supports(sgc):
