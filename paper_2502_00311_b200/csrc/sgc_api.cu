@@ -169,6 +169,28 @@ SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* g
     if (!states[0]) return SGC_ERR_NULL;
     const int64_t dc = states[0]->d;
     if ((dc * 4) % 16 != 0 && c > 1) return SGC_ERR_ALIGN;          // every chunk must start on a 16-byte boundary
+    if (((uintptr_t)grad & 15u) || ((uintptr_t)weight & 15u)) return SGC_ERR_ALIGN;
+    bool alike = true;
+    for (int32_t i = 0; i < c && alike; ++i) {
+        if (!states[i]) return SGC_ERR_NULL;
+        alike = states[i]->d == dc && states[i]->k == states[0]->k && states[i]->s == states[0]->s && states[i]->seed == states[0]->seed;
+    }
+    if (!alike) return SGC_ERR_GROUP;
+    if (sgc::chunked_batch_eligible(states, c)) {
+        // small per-chunk problems: all chunks in one set of launches (sgc_chunked.cu); a state listed twice is
+        // rejected there, when the table of the chunk list is built
+        cudaStream_t cs = static_cast<cudaStream_t>(stream);
+        for (int32_t i = 0; i < c; ++i) states[i]->t += 1;
+        int launches = 0;
+        const cudaError_t e = sgc::launch_chunked_batch(states, c, grad, weight, cs, &launches);
+        if (e == cudaErrorInvalidValue) { for (int32_t i = 0; i < c; ++i) states[i]->t -= 1; return SGC_ERR_GROUP; }
+        for (int32_t i = 0; i < c; ++i) {
+            sgc_state* st = states[i];
+            st->last_stream = cs; st->has_stream = true; st->stepped = true;
+            st->last_launches = i == 0 ? launches : 0;
+        }
+        return (int)e;
+    }
     std::vector<const float*> gs((size_t)c);
     std::vector<float*> ws((size_t)c);
     for (int32_t i = 0; i < c; ++i) { gs[i] = grad + (size_t)i * dc; ws[i] = weight + (size_t)i * dc; }
@@ -179,6 +201,7 @@ SGC_API int sgc_destroy(sgc_state* st) {
     if (!st) return SGC_OK;
     cudaError_t e = cudaSuccess;
     if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    sgc::free_chunk_ws(st);
     cudaError_t e2 = cudaFree(st->base);
     if (st->h_rounds) cudaFreeHost(st->h_rounds);
     for (cudaEvent_t ev : *st->ev_pool) cudaEventDestroy(ev);

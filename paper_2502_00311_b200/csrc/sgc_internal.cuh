@@ -170,6 +170,23 @@ struct Counters {
     int n_upd, mismatch, negv, pad;
 };
 
+// Batched chunk path (sgc_chunked.cu): the records of one chunk's state, as the batched kernels address them
+struct ChunkRef {
+    float* M; float* V; double* p; double* q; double* y64; double* r64;
+    uint32_t* sel_idx; float* sel_val;
+    uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
+    uint32_t* upd_idx; double* upd_val; Counters* cnt; SpecCtl* ctl;
+};
+// workspace of the batched chunk path, owned by the first state of the chunk list it was built for
+struct ChunkWs {
+    void* base;                 // one device allocation holding everything below
+    ChunkRef* table;            // [c]
+    float* r32;                 // [2c][kp] residuals of all streams (stream = 2 * chunk + moment), rows padded to kp
+    Cand* cand;                 // [2c][splits][2] best two columns of every column split, per stream
+    int c, kp, splits;
+    unsigned long long key;     // names the chunk list (its state pointers) the table was built from
+};
+
 }  // namespace sgc
 
 // the state behind the opaque handle
@@ -225,6 +242,7 @@ struct sgc_state {
     int* pick_li;               // [2][s] list position of every pick (Gram path)
     uint32_t* kept_ring;         // [hist_slots][s] kept indices of the last steps (all of them are columns M^ and V^ are made of)
     int hist_slots;
+    sgc::ChunkWs* chunk_ws;     // batched chunk path: workspace built for the chunk list that starts with this state
     bool two_level;             // host: wide lists and list passes are in use (steps that need several full passes)
     float* wide_tau;            // [kPassMaxN / 8] thresholds of the wide lists, one per 8th screened residual
     uint32_t* wide_list;        // [2][kWideCap]
@@ -267,6 +285,11 @@ cudaError_t launch_reproject(sgc_state* st, uint64_t new_seed, cudaStream_t stre
 cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches);
 cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
                            cudaStream_t stream);
+// MESGC with small per-chunk problems (s <= 16, k <= 128): the whole step of all chunks in 2 + 2s launches
+bool chunked_batch_eligible(sgc_state* const* sts, int c);
+cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad, float* weight, cudaStream_t stream,
+                                 int* launches);
+void free_chunk_ws(sgc_state* st);
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
 cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T
 

@@ -415,6 +415,59 @@ def test_mesgc_chunks_share_one_matrix_and_match_independent_oracles(sgc):
         r.close()
 
 
+@pytest.mark.parametrize("c,dc,k,sc,kind", [(6, 70_000, 56, 4, "student"), (40, 4096, 8, 1, "student"), (9, 65_536, 112, 16, "student"),
+                                             (300, 2048, 14, 2, "gauss"), (5, 10_000, 128, 16, "student"), (3, 5_000, 33, 7, "student")])
+def test_mesgc_small_chunks_batched_path_matches_independent_oracles(sgc, c, dc, k, sc, kind):
+    # the regime the paper runs MESGC in (s_c of 1 to 16, k_c = 7 or 8 times s_c): all chunks go through one set of
+    # launches; every chunk must still equal an SGC problem of its own, record by record
+    d = c * dc
+    hp = inputs.ADAM
+    m = sgc.Mesgc(d, c, k, sc, 8, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0)
+    refs = [oracle.Oracle(dc, k, sc, 8, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0) for _ in range(c)]
+    w0 = inputs.weights(d, 2)
+    w_gpu, w_ref = cuda(w0.copy()), w0.copy()
+    check = sorted(set(range(0, c, max(1, c // 12))) | {c - 1})          # chunks compared record by record
+    for step in range(1, 4):
+        supp, sign = inputs.planted_support(d, c * sc, 17 + step)          # redrawn: M^ and V^ have more than s_c columns
+        g = inputs.gradient(d, kind, supp, sign, 40 + step)
+        w_before = w_ref.copy()
+        m.step(cuda(g), w_gpu)
+        assert m.chunks[0].last_launches() == 2 + 2 * sc                  # the batched path ran
+        for i in range(c):
+            refs[i].step(g[i * dc:(i + 1) * dc], w_ref[i * dc:(i + 1) * dc])
+        for i in check:
+            st, ref = m.chunks[i], refs[i]
+            assert st.get("t") == step
+            for name in ("sel_idx", "sel_val", "lamM", "lamV", "upd_idx"):
+                assert np.array_equal(st.get(name), ref.get(name)), (name, i, step)
+            for name in ("p", "q", "M", "V"):
+                assert rel(st.get(name), ref.get(name)) < TOL_STATE, (name, i, step)
+            for name in ("doneM", "doneV", "n_upd", "mismatch", "negv"):
+                assert st.get(name) == ref.get(name), (name, i, step)
+            assert rel(st.get("xM"), ref.get("xM")) < TOL_UPDATE and rel(st.get("xV"), ref.get("xV")) < TOL_UPDATE
+            assert rel(st.get("rnormM"), ref.get("rnormM")) < 1e-6
+        wg = w_gpu.cpu().numpy()
+        changed = w_ref != w_before
+        assert np.array_equal(wg[~changed], w_before[~changed])           # nothing else is written
+        if changed.any():
+            dw_g = wg[changed].astype(np.float64) - w_before[changed]
+            dw_r = w_ref[changed].astype(np.float64) - w_before[changed]
+            assert np.abs(dw_g - dw_r).max() <= TOL_UPDATE * np.abs(dw_r).max() + 1.2e-7 * np.abs(w_before[changed]).max()
+    m.close()
+    for r in refs:
+        r.close()
+
+
+def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
+    import torch
+    m = sgc.Mesgc(4 * 4096, 4, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
+    hs = (sgc.C.c_void_p * 4)(m.chunks[0]._h, m.chunks[1]._h, m.chunks[1]._h, m.chunks[3]._h)
+    g, w = torch.zeros(4 * 4096, device="cuda"), torch.zeros(4 * 4096, device="cuda")
+    assert sgc.lib().sgc_step_chunked(hs, 4, g.data_ptr(), w.data_ptr(), None) != 0
+    assert m.chunks[0].get("t") == 0
+    m.close()
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 def test_sgca_reprojection_matches_the_oracle(sgc, mode):
     # Algorithm 4: every T = 2 steps the matrix is replaced and M, V are re-aligned; the steps after that run under the
