@@ -1,0 +1,65 @@
+"""Step time of memory-efficient SGC (Section 4.4) on one flat gradient, timed on the device.
+
+    python -m paper_2502_00311_b200.mesgc_timing [--d 16777216] [--steps 20] [--warmup 3] [--configs c:k:s,c:k:s,...]
+
+One JSON line per configuration (c chunks, k_c rows of A and s_c kept entries per chunk).  Gradients are synthetic
+(Student-t noise plus c * s_c planted entries), four buffers used in rotation so that no step finds its input in L2;
+CUDA events on the launching stream bracket the timed steps.  "launches" is what one step enqueued.
+"""
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import binding, inputs
+
+# the paper's settings: c = 256, s_c = 1, kappa = 8 (its reported runs) and the corners of its chunk-count study
+# (s = 4096 entries in all, kappa = 7)
+DEFAULT = "256:8:1,256:112:16,1024:28:4,4096:7:1"
+
+
+def time_config(d, c, k, s_c, steps, warmup):
+    hp = inputs.ADAM
+    m = binding.Mesgc(d, c, k, s_c, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0)
+    grads = []
+    for i in range(4):
+        supp, sign = inputs.planted_support(d, c * s_c, 100 + i)
+        grads.append(torch.from_numpy(inputs.gradient(d, "student", supp, sign, 200 + i)).cuda())
+    w = torch.from_numpy(inputs.weights(d, 5)).cuda()
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        m.step(grads[i % 4], w)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    for i in range(steps):
+        m.step(grads[(warmup + i) % 4], w)
+    stop.record(stream)
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(stop) / steps
+    out = dict(metric="mesgc_step_ms", d=d, c=c, k_c=k, s_c=s_c, value=ms, unit="ms", steps=steps, warmup=warmup,
+               launches=m.chunks[0].last_launches(),
+               status=int(np.bitwise_or.reduce([int(st.get("status")) for st in m.chunks[:: max(1, c // 16)]])),
+               gradient_GBps=4.0 * d / ms / 1e6, data="synthetic", l2="4 rotating gradients of %d MiB" % (4 * d >> 20))
+    m.close()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--d", type=int, default=4096 * 4096)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--configs", default=DEFAULT)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("a CUDA device is required")
+    binding.lib()
+    for item in args.configs.split(","):
+        c, k, s_c = (int(v) for v in item.split(":"))
+        print(json.dumps(time_config(args.d, c, k, s_c, args.steps, max(args.warmup, 3))), flush=True)
+
+
+if __name__ == "__main__":
+    main()
