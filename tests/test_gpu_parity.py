@@ -458,6 +458,44 @@ def test_mesgc_small_chunks_batched_path_matches_independent_oracles(sgc, c, dc,
         r.close()
 
 
+def test_mesgc_batched_path_edge_cases(sgc):
+    import torch
+    hp = inputs.ADAM
+    # tiny chunks: as many kept entries as a chunk can give (s_c = d/c), k_c barely above s_c
+    c, dc, k, sc = 5, 8, 12, 8
+    m = sgc.Mesgc(c * dc, c, k, sc, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    refs = [oracle.Oracle(dc, k, sc, 4, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]) for _ in range(c)]
+    rng = np.random.default_rng(0)
+    w0 = rng.standard_normal(c * dc).astype(np.float32)
+    w_gpu, w_ref = cuda(w0.copy()), w0.copy()
+    for step in range(2):
+        g = rng.standard_normal(c * dc).astype(np.float32)
+        m.step(cuda(g), w_gpu)
+        assert m.chunks[0].last_launches() == 2 + 2 * sc
+        for i in range(c):
+            refs[i].step(g[i * dc:(i + 1) * dc], w_ref[i * dc:(i + 1) * dc])
+            assert np.array_equal(m.chunks[i].get("sel_idx"), np.arange(dc, dtype=np.uint32))
+            for name in ("lamM", "lamV", "upd_idx"):
+                assert np.array_equal(m.chunks[i].get(name), refs[i].get(name)), (name, i)
+            assert m.chunks[i].get("doneM") == refs[i].get("doneM") and m.chunks[i].get("doneV") == refs[i].get("doneV")
+        assert rel(w_gpu.cpu().numpy(), w_ref) < 1e-5
+    m.close()
+    for r in refs:
+        r.close()
+    # a NaN is flagged in the chunk that holds it and nowhere else; equal magnitudes go to the lower index
+    c, dc = 4, 4096
+    m = sgc.Mesgc(c * dc, c, 16, 2, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    g = np.full(c * dc, 0.25, dtype=np.float32)
+    g[1::2] *= -1
+    g[2 * dc + 77] = np.nan
+    m.step(cuda(g), cuda(np.zeros(c * dc, dtype=np.float32)))
+    flags = [int(st.get("status")) & sgc.STATUS_NONFINITE_INPUT for st in m.chunks]
+    assert flags[2] and not (flags[0] or flags[1] or flags[3])
+    for i in (0, 1, 3):
+        assert np.array_equal(m.chunks[i].get("sel_idx"), np.array([0, 1], dtype=np.uint32))
+    m.close()
+
+
 def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
     import torch
     m = sgc.Mesgc(4 * 4096, 4, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
