@@ -34,6 +34,11 @@ struct ChunkArgs {
     float* r32;                          // [2c][kp]
     Cand* cand;                          // [2c][splits][2]
     int splits, cols_per_split;
+    // tensor-core route (see ChunkWs)
+    int kp64;
+    uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; uint2* rep;
+    double* rnv; unsigned char* unresolved; int* flags;
+    double z_rep;
 };
 
 __device__ __forceinline__ double warp_sum_d(double v) {
@@ -145,8 +150,10 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 // recovery in registers, scores all columns of the tile in ascending order (a strict ">" keeps the lowest index).
 // Only the best two columns per recovery leave the block; columns already in the support are skipped when they show up
 // as a new best.
+// gate != nullptr: the launch is a fallback of the tensor-core route and returns at once when *gate == 0.
 template <int KP>
-__global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter) {
+__global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter, const int* gate) {
+    if (gate != nullptr && *gate == 0) return;
     constexpr int TC = KP <= 64 ? 256 : 128;                         // columns per tile
     constexpr int ZS = KP + 4;                                       // row stride of a tile column (16-byte multiple)
     extern __shared__ float smem[];
@@ -234,35 +241,17 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
 // <Z_i, r>^2 / ||Z_i||^2 with the lowest index winning ties; then Algorithm 3 (Appendix B) for the new column:
 // g = A_Lambda^T a_new, c = F^T g, gamma = 1 / sqrt(g_ll - c^T c) (a pivot below 1e-10 g_ll ends this recovery),
 // new column [-gamma F c; gamma] of F, a_j = gamma <a_new, r>, x = F a, r = y - A_Lambda x.
-__global__ void __launch_bounds__(32) k_chunk_pick(ChunkArgs a, int iter) {
-    __shared__ double gv[kChunkMaxS], cv[kChunkMaxS], xs[kChunkMaxS];
-    __shared__ uint32_t cidx[kRescoreCap];
-    __shared__ int n_c;
-    const int res = blockIdx.x, m = res & 1, lane = threadIdx.x;
-    const ChunkRef ref = a.table[res >> 1];
-    if (ref.cnt->stopped[m]) return;
-    const int k = a.k, s = a.s, j = iter;
-    const Cand* cc = a.cand + (size_t)res * a.splits * 2;
-    const int n_entries = a.splits * 2;
-    float mx = -1.0f;
-    for (int e = lane; e < n_entries; e += 32) if (cc[e].idx != kNoColumn) mx = fmaxf(mx, cc[e].score);
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) n_c = 0;
-    __syncwarp();
-    const float thr = mx - 2e-3f * fabsf(mx);
-    for (int e = lane; e < n_entries; e += 32) {
-        const Cand c = cc[e];
-        if (c.idx != kNoColumn && c.score >= 0.0f && c.score >= thr) {
-            const int slot = atomicAdd(&n_c, 1);
-            if (slot < kRescoreCap) cidx[slot] = c.idx;
-        }
-    }
-    __syncwarp();
-    int nc = n_c;
-    if (nc > kRescoreCap) {
-        if (lane == 0) atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
-        nc = kRescoreCap;
-    }
+struct PickSmem {
+    double gv[kChunkMaxS], cv[kChunkMaxS], xs[kChunkMaxS];
+    uint32_t cidx[kRescoreCap];
+    int n_c;
+};
+
+// the decision among the nc candidates in sh.cidx and the update of the recovery `res` with the winner as pick j
+__device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& sh, int res, int j, int nc) {
+    double* gv = sh.gv; double* cv = sh.cv; double* xs = sh.xs;
+    const uint32_t* cidx = sh.cidx;
+    const int m = res & 1, lane = threadIdx.x, k = a.k, s = a.s;
     double* r = ref.r64 + (size_t)m * k;
     const double* y = ref.y64 + (size_t)m * k;
     if (nc == 0) {                                                   // no column left to pick (d/c = iterations made)
@@ -362,6 +351,133 @@ __global__ void __launch_bounds__(32) k_chunk_pick(ChunkArgs a, int iter) {
     }
 }
 
+// SIMT route: the candidates are the columns that phase A left within 2e-3 (relative) of the best fp32 score.
+// only != nullptr: a second chance for the recoveries that the tensor-core route marked unresolved; *gate == 0 skips it.
+__global__ void __launch_bounds__(32) k_chunk_pick(ChunkArgs a, int iter, const int* gate, const unsigned char* only) {
+    __shared__ PickSmem sh;
+    if (gate != nullptr && *gate == 0) return;
+    const int res = blockIdx.x, m = res & 1, lane = threadIdx.x;
+    if (only != nullptr && !only[res]) return;
+    const ChunkRef ref = a.table[res >> 1];
+    if (ref.cnt->stopped[m]) return;
+    const int j = iter;
+    uint32_t* cidx = sh.cidx;
+    int& n_c = sh.n_c;
+    const Cand* cc = a.cand + (size_t)res * a.splits * 2;
+    const int n_entries = a.splits * 2;
+    float mx = -1.0f;
+    for (int e = lane; e < n_entries; e += 32) if (cc[e].idx != kNoColumn) mx = fmaxf(mx, cc[e].score);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) n_c = 0;
+    __syncwarp();
+    const float thr = mx - 2e-3f * fabsf(mx);
+    for (int e = lane; e < n_entries; e += 32) {
+        const Cand c = cc[e];
+        if (c.idx != kNoColumn && c.score >= 0.0f && c.score >= thr) {
+            const int slot = atomicAdd(&n_c, 1);
+            if (slot < kRescoreCap) cidx[slot] = c.idx;
+        }
+    }
+    __syncwarp();
+    int nc = n_c;
+    if (nc > kRescoreCap) {
+        if (lane == 0) atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
+        nc = kRescoreCap;
+    }
+    pick_finish(a, ref, sh, res, j, nc);
+}
+
+// ---- tensor-core route of phase A (k_c > 32) --------------------------------------------------------------------
+// The contraction Z^T R of an iteration (all columns of A against the residuals of all recoveries) is what the screening
+// pass of sgc_pass.cu computes on the tensor cores: k_chunk_rt lays the residuals out as its binary16 rows (each scaled
+// by a power of two, rows k_c.. of the padded height zero) with a report threshold of z_rep noise deviations, the pass
+// reports every (column, recovery) pair above it, and k_chunk_pick_rep takes the candidates from the reports: every
+// column within twice the pass's error bound of the best report.  Whatever that cannot settle (no report, too many, a
+// window that reaches below the threshold, a zero residual) is marked unresolved and goes through the fp32 route.
+__global__ void __launch_bounds__(64) k_chunk_rt(ChunkArgs a, int n_rows) {
+    __shared__ double red[2];
+    const int row = blockIdx.x, t = threadIdx.x;
+    if (row == 0 && t == 0) a.flags[0] = 0;
+    const float inf = __int_as_float(0x7f800000);
+    bool live = row < 2 * a.c;
+    const ChunkRef* ref = live ? &a.table[row >> 1] : nullptr;
+    if (live && ref->cnt->stopped[row & 1]) live = false;
+    if (!live) {
+        if (t == 0) { a.tau[row] = inf; a.rep_count[row] = 0u; if (row < 2 * a.c) a.unresolved[row] = 0; }
+        return;
+    }
+    const double* r = ref->r64 + (size_t)(row & 1) * a.k;
+    double rn2 = 0.0;
+    for (int q = t; q < a.k; q += 64) rn2 += r[q] * r[q];
+    rn2 = warp_sum_d(rn2);
+    if ((t & 31) == 0) red[t >> 5] = rn2;
+    __syncthreads();
+    const double rn = sqrt(red[0] + red[1]);
+    if (!(rn > 0.0) || !isfinite(rn)) {                               // nothing to screen: the fp32 route decides
+        if (t == 0) { a.tau[row] = inf; a.rep_count[row] = 0u; a.unresolved[row] = 1; a.flags[0] = 1; }
+        return;
+    }
+    const double sc = residual_scale(rn);
+    uint16_t* dst = a.rt + (size_t)row * a.kp64;
+    for (int q = t; q < a.kp64; q += 64) dst[q] = q < a.k ? half_rn_bits(r[q] * sc) : (uint16_t)0;
+    if (t == 0) {
+        a.tau[row] = (float)(a.z_rep * rn / sqrt((double)a.k) * sc);
+        a.inv_scale[row] = (float)(1.0 / sc);
+        a.rep_count[row] = 0u;
+        a.rnv[row] = rn;
+        a.unresolved[row] = 0;
+    }
+}
+
+__global__ void __launch_bounds__(32) k_chunk_pick_rep(ChunkArgs a, int iter) {
+    __shared__ PickSmem sh;
+    const int res = blockIdx.x, m = res & 1, lane = threadIdx.x, j = iter;
+    const ChunkRef ref = a.table[res >> 1];
+    if (ref.cnt->stopped[m] || a.unresolved[res]) return;
+    const unsigned int count = a.rep_count[res];
+    bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;
+    const uint2* rp = a.rep + (size_t)res * kChunkRepCap;
+    const uint32_t* sup = ref.lam + (size_t)m * a.s;
+    float smax = -1.0f;
+    if (!give_up) {
+        for (unsigned int e = lane; e < count; e += 32) {
+            const uint2 v = rp[e];
+            bool taken = false;
+            for (int q = 0; q < j; ++q) taken |= (sup[q] == v.x);
+            if (!taken) smax = fmaxf(smax, __uint_as_float(v.y));
+        }
+        for (int o = 16; o > 0; o >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+        if (smax < 0.0f) give_up = true;
+    }
+    float lo = 0.0f;
+    if (!give_up) {
+        const double rn = a.rnv[res];
+        lo = (float)((double)smax - 2.0 * screen_margin(rn, (double)smax));
+        // the window must stay above the report threshold, or a column inside it may not have been reported
+        if (!((double)lo > a.z_rep * rn / sqrt((double)a.k) * 1.001)) give_up = true;
+    }
+    if (!give_up) {
+        if (lane == 0) sh.n_c = 0;
+        __syncwarp();
+        for (unsigned int e = lane; e < count; e += 32) {
+            const uint2 v = rp[e];
+            if (__uint_as_float(v.y) < lo) continue;
+            bool taken = false;
+            for (int q = 0; q < j; ++q) taken |= (sup[q] == v.x);
+            if (taken) continue;
+            const int slot = atomicAdd(&sh.n_c, 1);
+            if (slot < kRescoreCap) sh.cidx[slot] = v.x;
+        }
+        __syncwarp();
+        if (sh.n_c > kRescoreCap) give_up = true;
+    }
+    if (give_up) {
+        if (lane == 0) { a.unresolved[res] = 1; a.flags[0] = 1; }
+        return;
+    }
+    pick_finish(a, ref, sh, res, j, sh.n_c);
+}
+
 // ---- a5: Eq. (8) on the common support of the two recoveries of a chunk, one warp per chunk -------------------
 __global__ void __launch_bounds__(32) k_chunk_scatter(ChunkArgs a, float* __restrict__ weight, double alpha, double eps, double lr) {
     __shared__ uint32_t vidx[kChunkMaxS];
@@ -427,6 +543,7 @@ unsigned long long list_key(sgc_state* const* sts, int c) {
         h ^= (unsigned long long)(uintptr_t)sts[i]; h *= 1099511628211ull;
         h ^= (unsigned long long)(uintptr_t)sts[i]->base; h *= 1099511628211ull;
     }
+    h ^= sts[0]->seed; h *= 1099511628211ull;                        // the norm table belongs to one matrix
     return h ^ (unsigned long long)c;
 }
 
@@ -439,9 +556,9 @@ cudaError_t corr_setup(size_t* smem_out) {
 }
 
 template <int KP>
-void corr_launch(const ChunkArgs& a, int iter, size_t smem, cudaStream_t stream) {
+void corr_launch(const ChunkArgs& a, int iter, size_t smem, cudaStream_t stream, const int* gate) {
     dim3 grid((unsigned int)a.splits, (unsigned int)((2 * a.c + kCorrBlock - 1) / kCorrBlock));
-    k_chunk_corr<KP><<<grid, kCorrBlock, smem, stream>>>(a, iter);
+    k_chunk_corr<KP><<<grid, kCorrBlock, smem, stream>>>(a, iter, gate);
 }
 
 // builds (or reuses) the workspace for this chunk list; the first build synchronises (one allocation, one copy)
@@ -469,15 +586,55 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     per = (per + tile - 1) / tile * tile;
     splits = (int)((st0->d + per - 1) / per);
     ws->splits = splits;
-    const size_t b_table = ((size_t)c * sizeof(ChunkRef) + 255) / 256 * 256;
-    const size_t b_r32 = ((size_t)2 * c * ws->kp * sizeof(float) + 255) / 256 * 256;
-    const size_t b_cand = (size_t)2 * c * splits * 2 * sizeof(Cand);
-    cudaError_t e = cudaMalloc(&ws->base, b_table + b_r32 + b_cand);
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    const size_t b_table = up((size_t)c * sizeof(ChunkRef));
+    const size_t b_r32 = up((size_t)2 * c * ws->kp * sizeof(float));
+    const size_t b_cand = up((size_t)2 * c * splits * 2 * sizeof(Cand));
+    // tensor-core route: worth it from k_c = 33 on; bounded by its report lists (n_rows * 16 KB)
+    ws->tensor = ws->kp >= 64 && 2 * c <= 2048 && st0->d >= 1024;
+    ws->kp64 = (st0->k + 63) / 64 * 64;
+    ws->n_rows = (2 * c + 31) / 32 * 32;
+    ws->passes = (ws->n_rows + kPassMaxN - 1) / kPassMaxN;
+    size_t b_rt = 0, b_row = 0, b_rep = 0, b_norm = 0, b_rn = 0, b_un = 0, b_flags = 0;
+    if (ws->tensor) {
+        b_rt = up((size_t)ws->n_rows * ws->kp64 * sizeof(uint16_t));
+        b_row = up((size_t)ws->n_rows * sizeof(float));
+        b_rep = up((size_t)ws->n_rows * kChunkRepCap * sizeof(uint2));
+        b_norm = up((size_t)st0->d * sizeof(uint16_t));
+        b_rn = up((size_t)2 * c * sizeof(double));
+        b_un = up((size_t)2 * c);
+        b_flags = 256;
+    }
+    cudaError_t e = cudaMalloc(&ws->base, b_table + b_r32 + b_cand + b_rt + 3 * b_row + b_rep + b_norm + b_rn + b_un + b_flags);
     if (e != cudaSuccess) { delete ws; return e; }
     unsigned char* base = static_cast<unsigned char*>(ws->base);
-    ws->table = reinterpret_cast<ChunkRef*>(base);
-    ws->r32 = reinterpret_cast<float*>(base + b_table);
-    ws->cand = reinterpret_cast<Cand*>(base + b_table + b_r32);
+    size_t off = 0;
+    ws->table = reinterpret_cast<ChunkRef*>(base + off); off += b_table;
+    ws->r32 = reinterpret_cast<float*>(base + off); off += b_r32;
+    ws->cand = reinterpret_cast<Cand*>(base + off); off += b_cand;
+    if (ws->tensor) {
+        ws->rt = reinterpret_cast<uint16_t*>(base + off); off += b_rt;
+        ws->tau = reinterpret_cast<float*>(base + off); off += b_row;
+        ws->inv_scale = reinterpret_cast<float*>(base + off); off += b_row;
+        ws->rep_count = reinterpret_cast<unsigned int*>(base + off); off += b_row;
+        ws->rep = reinterpret_cast<uint2*>(base + off); off += b_rep;
+        ws->inv_norm = reinterpret_cast<uint16_t*>(base + off); off += b_norm;
+        ws->rnv = reinterpret_cast<double*>(base + off); off += b_rn;
+        ws->unresolved = base + off; off += b_un;
+        ws->flags = reinterpret_cast<int*>(base + off); off += b_flags;
+        ws->z_rep = normal_tail_threshold((double)st0->d, 32.0);    // ~32 noise columns per recovery above the threshold
+        const int h_flags[3] = {0, 0, 1};
+        e = pass_configure(kPassMaxN);
+        if (e == cudaSuccess) e = cudaMemset(ws->rt, 0, b_rt);
+        if (e == cudaSuccess) e = cudaMemset(ws->unresolved, 0, b_un);
+        if (e == cudaSuccess) e = cudaMemcpy(ws->flags, h_flags, sizeof(h_flags), cudaMemcpyHostToDevice);
+        for (int p = 0; p < ws->passes && e == cudaSuccess; ++p) {
+            const int n_p = ws->n_rows - p * kPassMaxN < kPassMaxN ? ws->n_rows - p * kPassMaxN : kPassMaxN;
+            e = pass_encode_map(ws->tmap[p], ws->rt + (size_t)p * kPassMaxN * ws->kp64, n_p, ws->kp64);
+        }
+        if (e == cudaSuccess) e = launch_inv_norms(st0->seed, (uint64_t)st0->d, st0->k, ws->inv_norm, 0);
+        if (e != cudaSuccess) { cudaFree(ws->base); delete ws; return e; }
+    }
     std::vector<ChunkRef> host((size_t)c);
     for (int i = 0; i < c; ++i) {
         sgc_state* st = sts[i];
@@ -533,6 +690,8 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     a.cols_per_split = (int)((st0->d + ws->splits - 1) / ws->splits);
     const int tile = ws->kp <= 64 ? 256 : 128;
     a.cols_per_split = (a.cols_per_split + tile - 1) / tile * tile;
+    a.kp64 = ws->kp64; a.rt = ws->rt; a.tau = ws->tau; a.inv_scale = ws->inv_scale; a.rep_count = ws->rep_count; a.rep = ws->rep;
+    a.rnv = ws->rnv; a.unresolved = ws->unresolved; a.flags = ws->flags; a.z_rep = ws->z_rep;
     const double b1 = (double)st0->beta1, b2 = (double)st0->beta2;
     const double c1 = 1.0 - pow(b1, (double)st0->t), c2 = 1.0 - pow(b2, (double)st0->t);
     const int s = st0->s;
@@ -552,14 +711,32 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     }
     if (e != cudaSuccess) return e;
     for (int iter = 0; iter < s; ++iter) {
-        switch (ws->kp) {
-            case 8: corr_launch<8>(a, iter, smem, stream); break;
-            case 16: corr_launch<16>(a, iter, smem, stream); break;
-            case 32: corr_launch<32>(a, iter, smem, stream); break;
-            case 64: corr_launch<64>(a, iter, smem, stream); break;
-            default: corr_launch<128>(a, iter, smem, stream); break;
+        const int* gate = nullptr;
+        if (ws->tensor) {
+            // phase A on the tensor cores; the fp32 kernels below then only run for what the reports left open
+            k_chunk_rt<<<ws->n_rows, 64, 0, stream>>>(a, ws->n_rows);
+            const int* gates[kPassMaxBatch] = {ws->flags + 2};
+            int* errors[kPassMaxBatch] = {ws->flags + 1};
+            for (int p = 0; p < ws->passes && e == cudaSuccess; ++p) {
+                const int n_p = ws->n_rows - p * kPassMaxN < kPassMaxN ? ws->n_rows - p * kPassMaxN : kPassMaxN;
+                const size_t r0 = (size_t)p * kPassMaxN;
+                e = launch_pass(ws->tmap[p], st0->seed, (uint64_t)st0->d, ws->kp64, n_p, ws->tau + r0, ws->inv_scale + r0,
+                                ws->inv_norm, ws->rep_count + r0, ws->rep + r0 * kChunkRepCap, kChunkRepCap, gates, errors,
+                                st0->sm_count, stream);
+            }
+            if (e != cudaSuccess) return e;
+            k_chunk_pick_rep<<<2 * c, 32, 0, stream>>>(a, iter);
+            *launches += 2 + ws->passes;
+            gate = ws->flags;
         }
-        k_chunk_pick<<<2 * c, 32, 0, stream>>>(a, iter);
+        switch (ws->kp) {
+            case 8: corr_launch<8>(a, iter, smem, stream, gate); break;
+            case 16: corr_launch<16>(a, iter, smem, stream, gate); break;
+            case 32: corr_launch<32>(a, iter, smem, stream, gate); break;
+            case 64: corr_launch<64>(a, iter, smem, stream, gate); break;
+            default: corr_launch<128>(a, iter, smem, stream, gate); break;
+        }
+        k_chunk_pick<<<2 * c, 32, 0, stream>>>(a, iter, gate, gate ? ws->unresolved : nullptr);
         *launches += 2;
     }
     k_chunk_scatter<<<c, 32, 0, stream>>>(a, weight, (double)st0->alpha, (double)st0->eps, (double)st0->lr);

@@ -1,6 +1,7 @@
 // Internal declarations of the SGC CUDA library (sm_100a).  Not part of the public C ABI.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
@@ -124,6 +125,22 @@ constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
 // Cauchy-Schwarz), and the pass accumulates the column norm in short binary16 partial sums (error ~1e-4 relative)
 constexpr double kScreenMargin = 5.5e-4;
 constexpr double kScreenNormMargin = 1.0e-3;
+
+// binary16 residual rows of the screening pass
+__device__ __forceinline__ uint16_t half_rn_bits(double v) { return __half_as_ushort(__double2half(v)); }   // nearest even
+
+// bound on |score seen by the screening pass - exact score| for a residual of norm rn and a score near ps
+__device__ __forceinline__ double screen_margin(double rn, double ps) { return kScreenMargin * rn + kScreenNormMargin * ps; }
+
+// power-of-two scale that brings a residual of norm rn into [2^12, 2^13): no binary16 overflow, and entries
+// down to 2^-26 of the norm stay normal numbers
+__device__ __forceinline__ double residual_scale(double rn) {
+    if (!(rn > 0.0) || !isfinite(rn)) return 1.0;
+    int e;
+    frexp(rn, &e);
+    return ldexp(1.0, 13 - e);
+}
+
 constexpr uint32_t kNoColumn = 0xFFFFFFFFu;
 
 struct Cand { float score; uint32_t idx; };
@@ -185,7 +202,20 @@ struct ChunkWs {
     Cand* cand;                 // [2c][splits][2] best two columns of every column split, per stream
     int c, kp, splits;
     unsigned long long key;     // names the chunk list (its state pointers) the table was built from
+    // tensor-core route of the correlation (k_c > 32): the residuals of all recoveries go through the screening pass
+    bool tensor;
+    int kp64, n_rows, passes;   // rows of A per column padded to a multiple of 64; residual rows (multiple of 32); passes of <= 256 rows
+    uint16_t* rt;               // [n_rows][kp64] binary16 residuals, each scaled by a power of two
+    float* tau; float* inv_scale; unsigned int* rep_count;   // [n_rows]
+    uint2* rep;                 // [n_rows][kChunkRepCap] (column, score)
+    uint16_t* inv_norm;         // [d/c] 1 / ||Z_i|| over the k_c rows, binary16
+    double* rnv;                // [2c] ||r|| of every recovery at the start of the iteration
+    unsigned char* unresolved;  // [2c] 1: the reports did not settle this recovery's pick; the fp32 route decides it
+    int* flags;                 // [0] some recovery is unresolved, [1] a wait inside a pass expired, [2] constant 1 (gate)
+    double z_rep;               // report threshold in units of ||r|| / sqrt(k_c)
+    unsigned char tmap[8][128]; // tensor maps of the row blocks of rt, one per pass
 };
+constexpr int kChunkRepCap = 2048;      // report slots per residual row of the chunk path
 
 }  // namespace sgc
 
@@ -290,6 +320,7 @@ bool chunked_batch_eligible(sgc_state* const* sts, int c);
 cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad, float* weight, cudaStream_t stream,
                                  int* launches);
 void free_chunk_ws(sgc_state* st);
+double normal_tail_threshold(double d, double target);   // z with d * P(|N(0,1)| > z) = target
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
 cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T
 

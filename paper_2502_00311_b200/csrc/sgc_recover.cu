@@ -104,20 +104,6 @@ __device__ double block_sum(double v, double* red) {
     return t;
 }
 
-__device__ __forceinline__ uint16_t half_rn_bits(double v) { return __half_as_ushort(__double2half(v)); }   // nearest even
-
-// bound on |score seen by the screening pass - exact score| for a residual of norm rn and a score near ps
-__device__ __forceinline__ double screen_margin(double rn, double ps) { return kScreenMargin * rn + kScreenNormMargin * ps; }
-
-// power-of-two scale that brings a residual of norm rn into [2^12, 2^13): no binary16 overflow, and entries
-// down to 2^-26 of the norm stay normal numbers
-__device__ __forceinline__ double residual_scale(double rn) {
-    if (!(rn > 0.0) || !isfinite(rn)) return 1.0;
-    int e;
-    frexp(rn, &e);
-    return ldexp(1.0, 13 - e);
-}
-
 // threshold of a wide list: every column scoring at least z_wide noise deviations against a screened residual (norm rn)
 // whose row index is a multiple of 8, in the scaled units of that row
 __device__ __forceinline__ float wide_threshold(const OmpArgs& a, double rn) {
@@ -1557,7 +1543,7 @@ k_scatter(int s, uint32_t* lam, double* x, Counters* __restrict__ cnt, float* __
 }
 
 // z with d * P(|N(0,1)| > z) = target (bisection on erfc)
-double normal_tail_threshold(double d, double target) {
+double normal_tail_threshold_impl(double d, double target) {
     double p = target / d;
     if (p > 0.5) p = 0.5;
     double lo = 0.0, hi = 12.0;
@@ -1598,6 +1584,8 @@ cudaError_t launch_omp(sgc_state* st, const OmpArgs& a, int mode, cudaStream_t s
 
 }  // namespace
 
+double normal_tail_threshold(double d, double target) { return normal_tail_threshold_impl(d, target); }
+
 cudaError_t configure_recover(sgc_state* st) {
     const size_t smem = ((size_t)st->k + 1) * sizeof(float2);
     cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -1622,9 +1610,9 @@ cudaError_t configure_recover(sgc_state* st) {
     int half = st->s < 128 ? st->s : 128;
     half = (half + 15) / 16 * 16;
     st->pass_n = 2 * half;
-    st->z_harvest = normal_tail_threshold((double)st->d, 3072.0);
-    st->z_floor = normal_tail_threshold((double)st->d, 6144.0);
-    st->z_wide = normal_tail_threshold((double)st->d, 100000.0);
+    st->z_harvest = normal_tail_threshold_impl((double)st->d, 3072.0);
+    st->z_floor = normal_tail_threshold_impl((double)st->d, 6144.0);
+    st->z_wide = normal_tail_threshold_impl((double)st->d, 100000.0);
     if (st->spec_ok) {
         e = pass_configure(kPassMaxN);
         if (e != cudaSuccess) return e;

@@ -432,7 +432,9 @@ def test_mesgc_small_chunks_batched_path_matches_independent_oracles(sgc, c, dc,
         g = inputs.gradient(d, kind, supp, sign, 40 + step)
         w_before = w_ref.copy()
         m.step(cuda(g), w_gpu)
-        assert m.chunks[0].last_launches() == 2 + 2 * sc                  # the batched path ran
+        # the batched path ran: 2 + 2 s_c launches, or, with phase A on the tensor cores (k_c > 32), 4 + passes per pick
+        passes = -(-(-(-2 * c // 32) * 32) // 256)
+        assert m.chunks[0].last_launches() == (2 + sc * (4 + passes) if k > 32 else 2 + 2 * sc)
         for i in range(c):
             refs[i].step(g[i * dc:(i + 1) * dc], w_ref[i * dc:(i + 1) * dc])
         for i in check:
