@@ -163,7 +163,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // dynamic shared memory (after alignment to 1024 bytes):
 //   stages x { A tile 0 (16 KB) | A tile 1 (16 KB) | R^T chunk (n x 128 B) }
 //   norms  float[kNormRing][256][2]      partial ||Z_i||^2 of the two generator threads of each column
-//   tau    float[256]
+//   tau    float[256], 1 / tau float[256]
 //   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
 // WIDE: the two-level screening code (wide-list harvest, list passes) is compiled in
 template <bool TABLE, bool WIDE>
@@ -194,7 +194,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     const uint32_t norms_off = (uint32_t)a.stages * stage_bytes;
     float* norms = reinterpret_cast<float*>(gen_base + norms_off);
     float* tau_s = norms + kNormRing * kSuperCols * 2;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tau_s + 256);
+    float* itau_s = tau_s + 256;                                     // 1 / tau: a group of 16 residuals is skipped on one compare
+    uint64_t* bars = reinterpret_cast<uint64_t*>(itau_s + 256);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * a.stages;
     const uint32_t bar_accf = bar_empty + 8u * a.stages, bar_acce = bar_accf + 16u;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 4);
@@ -216,7 +217,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    for (int i = threadIdx.x; i < 256; i += kPassThreads) tau_s[i] = i < a.n ? a.tau[i] : __int_as_float(0x7f800000);
+    for (int i = threadIdx.x; i < 256; i += kPassThreads) {
+        const float tv = i < a.n ? a.tau[i] : __int_as_float(0x7f800000);
+        tau_s[i] = tv;
+        itau_s[i] = tv > 0.0f ? 1.0f / tv : 3.0e38f;                 // tau = +inf (unused residual) -> 0
+    }
     if (warp == 1) {           // tensor memory: all 512 columns (the only CTA on this SM)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
                      : "memory");
@@ -316,6 +321,21 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                             }
                         }
                     }
+                    // one compare settles the usual case that none of the 16 residuals reaches its threshold
+                    // (|v| inv >= tau  <=>  |v| / tau >= 1 / inv, with a little slack for the rounding of 1 / tau)
+                    float peak = 0.0f;
+                    {
+                        const float4* it4 = reinterpret_cast<const float4*>(itau_s + c0);
+#pragma unroll
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const float4 w = it4[i4];
+                            peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4])) * w.x);
+                            peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 1])) * w.y);
+                            peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 2])) * w.z);
+                            peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 3])) * w.w);
+                        }
+                    }
+                    if (!(peak * inv >= 0.999f)) continue;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float sc = fabsf(__uint_as_float(v[i])) * inv;
@@ -441,7 +461,7 @@ cudaError_t get_encoder(EncodeTiledFn* out) {
 }
 
 size_t pass_smem_bytes(int n, int stages) {
-    return 1024 + (size_t)stages * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 256) +
+    return 1024 + (size_t)stages * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 512) +
            8 * (2 * (size_t)stages + 4) + 16;
 }
 
