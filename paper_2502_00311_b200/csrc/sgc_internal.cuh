@@ -168,6 +168,7 @@ struct SpecCtl {
     int gram_ok;            // 0: the Gram path gave up in this step (a pick is missing from the list)
     int tv[2];              // tentative picks: confirmed against the wide lists only (tv >= v)
     uint32_t tforced[2];    // column imposed as pick tv[m] by a list pass, or kNoColumn
+    int narrow;             // 1: only the first stream still has residuals to screen: the half-width pass serves the round
     int mini_done;          // 1: list passes rest until the next full pass
     int list_rounds;        // list passes of the last step that were resolved
     int list_refuted;       // picks that those list passes refuted
@@ -340,6 +341,7 @@ cudaError_t pass_configure(int n);
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
-                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide = nullptr);
+                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide = nullptr,
+                        const int* sel = nullptr, int sel_value = 0);
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream);
 }  // namespace sgc

@@ -59,6 +59,7 @@ struct PassArgs {
     unsigned int* big_bits;      // bitmap over [0, d)
     int big_cap, big_half;
     const SpecCtl* list_ctl;     // list pass: gate and list lengths come from the control block
+    const int* sel; int sel_value;    // optional: the kernel returns at once unless *sel == sel_value (which of two widths runs)
     const int* gate[kPassMaxBatch];   // optional: the kernel returns at once when every *gate is 0 (one per batched state)
     int* error[kPassMaxBatch];        // set to 1 when a wait expired (one per batched state)
 };
@@ -174,6 +175,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         for (int q = 0; q < kPassMaxBatch; ++q) any = any || (a.gate[q] != nullptr && *a.gate[q] != 0);
         if (!any) return;
     }
+    if (a.sel != nullptr && *a.sel != a.sel_value) return;
     // list pass: the columns are the concatenation of the two wide lists (every block reads the same lengths: nothing
     // writes them while a list pass runs)
     unsigned int list_n0 = 0, list_n = 0, num_super = a.num_super;
@@ -504,8 +506,10 @@ cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cu
 
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
-                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide) {
+                        int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide, const int* sel,
+                        int sel_value) {
     PassArgs a;
+    a.sel = sel; a.sel_value = sel_value;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
     a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;

@@ -1335,6 +1335,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         } else if (ctl->finished[0] && ctl->finished[1]) {
             ctl->round_active = 0;
         }
+        ctl->narrow = (ctl->finished[1] && !ctl->finished[0]) ? 1 : 0;     // the rows of a pass start with the first stream's
         const int r = ctl->rounds - 1;
         if (r >= 0 && r < kMaxRounds) { ctl->trace[r][0] = ctl->v[0]; ctl->trace[r][1] = ctl->v[1]; ctl->trace[r][2] = ctl->n_cand; }
     }
@@ -1353,6 +1354,7 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau, int sh
         ctl->forced[0] = ctl->forced[1] = kNoColumn;
         ctl->finished[0] = 0;
         ctl->finished[1] = shared ? 1 : 0;          // shared support: the second stream makes no picks of its own
+        ctl->narrow = shared ? 1 : 0;
         ctl->stop[0] = ctl->stop[1] = 0;
         ctl->rounds = 0; ctl->pass_error = 0;
         for (int r = 0; r < kMaxRounds; ++r) ctl->trace[r][0] = ctl->trace[r][1] = ctl->trace[r][2] = 0;
@@ -1707,10 +1709,16 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     int* errors[kPassMaxBatch] = {&st->ctl->pass_error};
                     PassWide lp = wide;
                     lp.list_pass = true;
-                    const bool narrow = st->shared_support && st->pass_n_half < st->pass_n;
-                    e = launch_pass(narrow ? st->tmap_half : st->tmap[0], st->seed, (uint64_t)st->d, st->k,
-                                    narrow ? st->pass_n_half : st->pass_n, st->tau, st->inv_scale,
-                                    st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp);
+                    const bool two_widths = st->pass_n_half < st->pass_n;       // the width that ctl->narrow names runs
+                    e = launch_pass(st->tmap[0], st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale,
+                                    st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp,
+                                    two_widths ? &st->ctl->narrow : nullptr, 0);
+                    if (two_widths && e == cudaSuccess) {
+                        e = launch_pass(st->tmap_half, st->seed, (uint64_t)st->d, st->k, st->pass_n_half, st->tau,
+                                        st->inv_scale, st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors,
+                                        st->sm_count, stream, &lp, &st->ctl->narrow, 1);
+                        *launches += 1;
+                    }
                     *launches += 1;
                 }
                 if (e != cudaSuccess) break;
@@ -1746,11 +1754,19 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                         gates[q] = q < nb ? &sts[b0 + q]->ctl->round_active : nullptr;
                         errors[q] = q < nb ? &sts[b0 + q]->ctl->pass_error : nullptr;
                     }
-                    const bool narrow = nb == 1 && lead->shared_support && lead->pass_n_half < lead->pass_n;
-                    e = launch_pass(narrow ? lead->tmap_half : lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k,
-                                    narrow ? lead->pass_n_half : nb * lead->pass_n, lead->tau,
+                    // a state on its own: once only its first stream has residuals left (the second recovery is complete, or
+                    // the shared-support variant is on), the pass half as wide serves the round; ctl->narrow names the width
+                    const bool two_widths = n == 1 && lead->pass_n_half < lead->pass_n;
+                    e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
                                     lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
-                                    lead->sm_count, stream, two_level ? &wide : nullptr);
+                                    lead->sm_count, stream, two_level ? &wide : nullptr,
+                                    two_widths ? &lead->ctl->narrow : nullptr, 0);
+                    if (two_widths && e == cudaSuccess) {
+                        e = launch_pass(lead->tmap_half, lead->seed, (uint64_t)lead->d, lead->k, lead->pass_n_half, lead->tau,
+                                        lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
+                                        lead->sm_count, stream, two_level ? &wide : nullptr, &lead->ctl->narrow, 1);
+                        *launches += 1;
+                    }
                     *launches += 1;
                 }
                 for (int i = b0; i < b0 + nb && e == cudaSuccess; ++i) {
