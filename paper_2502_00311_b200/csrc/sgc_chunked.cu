@@ -633,6 +633,7 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
             e = pass_encode_map(ws->tmap[p], ws->rt + (size_t)p * kPassMaxN * ws->kp64, n_p, ws->kp64);
         }
         if (e == cudaSuccess) e = launch_inv_norms(st0->seed, (uint64_t)st0->d, st0->k, ws->inv_norm, 0);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();           // the table is ready before any stream uses it
         if (e != cudaSuccess) { cudaFree(ws->base); delete ws; return e; }
     }
     std::vector<ChunkRef> host((size_t)c);
@@ -646,6 +647,7 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     }
     e = cudaMemcpy(ws->table, host.data(), (size_t)c * sizeof(ChunkRef), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ws->r32, 0, b_r32);         // rows k..kp of every residual stay zero
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();               // set-up done before the caller's stream runs on it
     if (e != cudaSuccess) { cudaFree(ws->base); delete ws; return e; }
     st0->chunk_ws = ws;
     return cudaSuccess;
