@@ -498,6 +498,34 @@ def test_mesgc_batched_path_edge_cases(sgc):
     m.close()
 
 
+def test_mesgc_batched_path_on_a_side_stream(sgc):
+    # the first call builds the chunk table and the norm table; a stream that does not synchronise with the default
+    # stream must still find them complete
+    import torch
+    hp = inputs.ADAM
+    c, dc, k, sc = 8, 16_384, 56, 4
+    d = c * dc
+    supp, sign = inputs.planted_support(d, c * sc, 5)
+    g = cuda(inputs.gradient(d, "student", supp, sign, 6))
+    outs = []
+    for side in (False, True):
+        m = sgc.Mesgc(d, c, k, sc, 2, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+        w = cuda(inputs.weights(d, 1))
+        if side:
+            stream = torch.cuda.Stream()
+            stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(stream):
+                m.step(g, w, stream=stream)
+            stream.synchronize()
+        else:
+            m.step(g, w)
+        outs.append(([st.get("lamM").copy() for st in m.chunks], [st.get("lamV").copy() for st in m.chunks], w.cpu().numpy()))
+        m.close()
+    for a, b in zip(outs[0][0] + outs[0][1], outs[1][0] + outs[1][1]):
+        assert np.array_equal(a, b)
+    assert np.array_equal(outs[0][2], outs[1][2])
+
+
 def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
     import torch
     m = sgc.Mesgc(4 * 4096, 4, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
