@@ -255,10 +255,10 @@ class Mesgc:
             raise ValueError("d must be a multiple of the number of chunks")
         self.d, self.c = int(d), int(c)
         self.chunks = [Sgc(d // c, k, s_c, seed, lr, beta1, beta2, eps, alpha=alpha) for _ in range(c)]
+        self._hs = (C.c_void_p * self.c)(*[st._h for st in self.chunks])       # the handle array of every call
 
     def step(self, grad, weight, stream=None):
-        hs = (C.c_void_p * self.c)(*[st._h for st in self.chunks])
-        _check(lib().sgc_step_chunked(hs, self.c, _dev_ptr(grad, self.d, "grad"), _dev_ptr(weight, self.d, "weight"),
+        _check(lib().sgc_step_chunked(self._hs, self.c, _dev_ptr(grad, self.d, "grad"), _dev_ptr(weight, self.d, "weight"),
                                       _stream_ptr(stream)), "sgc_step_chunked")
 
     def close(self):
