@@ -136,7 +136,7 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
  * states with sgc_create(d / c, k, s_c, seed, ...) -- the same seed, hence the same A -- and passes the whole vectors:
  *   grad, weight   device pointers, c * (d / c) floats; chunk i occupies [i * d/c, (i + 1) * d/c)
  * d / c must be a multiple of 4 (16-byte aligned chunks).  The result is that of sgc_step_group on the c chunk
- * pointers.  Chunk lists with small problems (s_c <= 16, k <= 128, all chunks at the same step with the same
+ * pointers.  Chunk lists with small problems (s_c <= 32, k <= 256, all chunks at the same step with the same
  * hyper-parameters, no sgc_set_recovery variant, no forced speculative mode, profiling off) are served by batched
  * kernels, 2 + 2 s_c launches for all chunks together; the first such call for a given list of states allocates a
  * table of their buffers (one cudaMalloc and one synchronous copy; freed by sgc_destroy of states[0]), so it should

@@ -1,5 +1,5 @@
 // MESGC (Section 4.4) with small per-chunk problems: c chunks of one flat vector, each an SGC problem of its own
-// (own M, V; s_c <= 16 kept entries, k_c <= 128 rows), all sharing the matrix A (k_c x d/c) named by one seed.
+// (own M, V; s_c <= 32 kept entries, k_c <= 256 rows), all sharing the matrix A (k_c x d/c) named by one seed.
 // Run chunk by chunk this costs ~25 launches per chunk; here the whole step of all chunks takes 2 + 2 s_c launches:
 //   k_chunk_front    block = chunk: exact top-s_c of the chunk (a1), p = A g~, q = A g~^2 and the k-space Adam moments
 //                    (a2 + a3), residuals r = y for both moments
@@ -22,12 +22,12 @@ namespace {
 
 constexpr int kFrontThreads = 512;
 constexpr int kCorrBlock = 256;          // residuals per block of k_chunk_corr
-constexpr int kChunkMaxS = 16;
-constexpr int kChunkMaxK = 128;
+constexpr int kChunkMaxS = 32;
+constexpr int kChunkMaxK = 256;
 
 struct ChunkArgs {
     const ChunkRef* table;
-    int c, k, s, kp;                     // kp: k rounded up to 8, 16, 32, 64 or 128 (row stride of r32)
+    int c, k, s, kp;                     // kp: k rounded up to 8, 16, 32, 64, 128 or 256 (row stride of r32)
     long long dc;                        // columns per chunk
     uint32_t seed_lo, seed_hi;
     double sigma;
@@ -150,29 +150,34 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 // recovery in registers, scores all columns of the tile in ascending order (a strict ">" keeps the lowest index).
 // Only the best two columns per recovery leave the block; columns already in the support are skipped when they show up
 // as a new best.
+__host__ __device__ constexpr int corr_ks(int kp) { return kp > 128 ? 2 : 1; }        // threads that share the rows of a residual
+__host__ __device__ constexpr int corr_group(int kp) { return kCorrBlock / corr_ks(kp); }   // recoveries per block
+
 // gate != nullptr: the launch is a fallback of the tensor-core route and returns at once when *gate == 0.
 template <int KP>
 __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter, const int* gate) {
     if (gate != nullptr && *gate == 0) return;
-    constexpr int TC = KP <= 64 ? 256 : 128;                         // columns per tile
+    constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 64);      // columns per tile
     constexpr int ZS = KP + 4;                                       // row stride of a tile column (16-byte multiple)
+    constexpr int KS = corr_ks(KP), KL = KP / KS;                    // at the largest k two threads hold half the rows each
     extern __shared__ float smem[];
     float* zt = smem;                                                // [TC][ZS]
     float* inv = smem + TC * ZS;                                     // [TC]
-    const int res = blockIdx.y * kCorrBlock + threadIdx.x;           // recovery = 2 * chunk + moment
+    const int h = threadIdx.x % KS;
+    const int res = blockIdx.y * (kCorrBlock / KS) + threadIdx.x / KS;     // recovery = 2 * chunk + moment
     const bool have = res < 2 * a.c;
     bool active = false;
     const uint32_t* sup = nullptr;
-    float rr[KP];
+    float rr[KL];
 #pragma unroll
-    for (int q = 0; q < KP; ++q) rr[q] = 0.0f;
+    for (int q = 0; q < KL; ++q) rr[q] = 0.0f;
     if (have) {
         const ChunkRef& ref = a.table[res >> 1];
         active = ref.cnt->stopped[res & 1] == 0;
         sup = ref.lam + (size_t)(res & 1) * a.s;
-        const float4* src = reinterpret_cast<const float4*>(a.r32 + (size_t)res * KP);
+        const float4* src = reinterpret_cast<const float4*>(a.r32 + (size_t)res * KP + h * KL);
 #pragma unroll
-        for (int q = 0; q < KP / 4; ++q) { const float4 f = src[q]; rr[4 * q] = f.x; rr[4 * q + 1] = f.y; rr[4 * q + 2] = f.z; rr[4 * q + 3] = f.w; }
+        for (int q = 0; q < KL / 4; ++q) { const float4 f = src[q]; rr[4 * q] = f.x; rr[4 * q + 1] = f.y; rr[4 * q + 2] = f.z; rr[4 * q + 3] = f.w; }
     }
     float s1 = -1.0f, s2 = -1.0f;
     uint32_t i1 = kNoColumn, i2 = kNoColumn;
@@ -187,11 +192,11 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             float* dst = zt + t * ZS;
             if (col < col1) {
                 const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)col);
-                uint32_t h = key.ck;
+                uint32_t hw = key.ck;
 #pragma unroll 4
                 for (int row = 0; row < KP; row += 2) {
-                    float2 z = half2_bits_to_float2(z_pair_from_word(h));
-                    h += key.mk;
+                    float2 z = half2_bits_to_float2(z_pair_from_word(hw));
+                    hw += key.mk;
                     if (row >= a.k) z.x = 0.0f;
                     if (row + 1 >= a.k) z.y = 0.0f;
                     dst[row] = z.x; dst[row + 1] = z.y;
@@ -204,21 +209,23 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             inv[t] = n2 > 0.0f ? 1.0f / sqrtf(n2) : 0.0f;
         }
         __syncthreads();
-        if (!active) continue;
+        if (KS == 1 && !active) continue;                            // (with KS = 2 the shuffle below needs every lane)
         const int n_here = (int)((col1 - tile) < TC ? (col1 - tile) : TC);
         for (int t = 0; t < n_here; ++t) {
-            const float4* zc = reinterpret_cast<const float4*>(zt + t * ZS);
+            const float4* zc = reinterpret_cast<const float4*>(zt + t * ZS + h * KL);
             float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
-            for (int q = 0; q < KP / 4; ++q) {
-                const float4 z = zc[q];                              // same address in every thread: a broadcast
+            for (int q = 0; q < KL / 4; ++q) {
+                const float4 z = zc[q];                              // one address per row part: a broadcast
                 acc0 = __fmaf_rn(z.x, rr[4 * q], acc0);
                 acc1 = __fmaf_rn(z.y, rr[4 * q + 1], acc1);
                 acc0 = __fmaf_rn(z.z, rr[4 * q + 2], acc0);
                 acc1 = __fmaf_rn(z.w, rr[4 * q + 3], acc1);
             }
-            const float sc = fabsf(acc0 + acc1) * inv[t];
-            if (sc > s2) {
+            float dot = acc0 + acc1;
+            if (KS == 2) dot += __shfl_xor_sync(0xffffffffu, dot, 1);        // the other half of the rows
+            const float sc = fabsf(dot) * inv[t];
+            if (active && sc > s2) {
                 const uint32_t col = (uint32_t)(tile + t);
                 bool taken = false;
                 for (int q = 0; q < iter; ++q) taken |= (sup[q] == col);
@@ -229,7 +236,7 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             }
         }
     }
-    if (have) {
+    if (have && h == 0) {
         Cand* out = a.cand + ((size_t)res * a.splits + blockIdx.x) * 2;
         out[0].score = s1; out[0].idx = i1;
         out[1].score = s2; out[1].idx = i2;
@@ -535,7 +542,7 @@ __global__ void __launch_bounds__(32) k_chunk_scatter(ChunkArgs a, float* __rest
 // ---- host side ----------------------------------------------------------------------------------------------
 namespace {
 
-int padded_k(int k) { return k <= 8 ? 8 : k <= 16 ? 16 : k <= 32 ? 32 : k <= 64 ? 64 : 128; }
+int padded_k(int k) { return k <= 8 ? 8 : k <= 16 ? 16 : k <= 32 ? 32 : k <= 64 ? 64 : k <= 128 ? 128 : 256; }
 
 unsigned long long list_key(sgc_state* const* sts, int c) {
     unsigned long long h = 1469598103934665603ull;                   // FNV-1a
@@ -549,7 +556,7 @@ unsigned long long list_key(sgc_state* const* sts, int c) {
 
 template <int KP>
 cudaError_t corr_setup(size_t* smem_out) {
-    constexpr int TC = KP <= 64 ? 256 : 128;
+    constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 64);
     const size_t smem = (size_t)(TC * (KP + 4) + TC) * sizeof(float);
     *smem_out = smem;
     return cudaFuncSetAttribute(k_chunk_corr<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -557,7 +564,7 @@ cudaError_t corr_setup(size_t* smem_out) {
 
 template <int KP>
 void corr_launch(const ChunkArgs& a, int iter, size_t smem, cudaStream_t stream, const int* gate) {
-    dim3 grid((unsigned int)a.splits, (unsigned int)((2 * a.c + kCorrBlock - 1) / kCorrBlock));
+    dim3 grid((unsigned int)a.splits, (unsigned int)((2 * a.c + corr_group(KP) - 1) / corr_group(KP)));
     k_chunk_corr<KP><<<grid, kCorrBlock, smem, stream>>>(a, iter, gate);
 }
 
@@ -576,8 +583,8 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     if (!ws) return cudaErrorMemoryAllocation;
     ws->c = c; ws->key = key; ws->kp = padded_k(st0->k);
     // column splits: enough blocks for every SM twice over, at least one tile per split
-    const int groups = (2 * c + kCorrBlock - 1) / kCorrBlock;
-    const int tile = ws->kp <= 64 ? 256 : 128;
+    const int groups = (2 * c + corr_group(ws->kp) - 1) / corr_group(ws->kp);
+    const int tile = ws->kp <= 64 ? 256 : (ws->kp <= 128 ? 128 : 64);
     int splits = (2 * st0->sm_count + groups - 1) / groups;
     const long long max_splits = (st0->d + tile - 1) / tile;
     if (splits > max_splits) splits = (int)max_splits;
@@ -690,7 +697,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     a.sigma = (double)(float)(1.0 / sqrt((double)st0->k));
     a.r32 = ws->r32; a.cand = ws->cand; a.splits = ws->splits;
     a.cols_per_split = (int)((st0->d + ws->splits - 1) / ws->splits);
-    const int tile = ws->kp <= 64 ? 256 : 128;
+    const int tile = ws->kp <= 64 ? 256 : (ws->kp <= 128 ? 128 : 64);
     a.cols_per_split = (a.cols_per_split + tile - 1) / tile * tile;
     a.kp64 = ws->kp64; a.rt = ws->rt; a.tau = ws->tau; a.inv_scale = ws->inv_scale; a.rep_count = ws->rep_count; a.rep = ws->rep;
     a.rnv = ws->rnv; a.unresolved = ws->unresolved; a.flags = ws->flags; a.z_rep = ws->z_rep;
@@ -701,7 +708,8 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     else if (s <= 2) k_chunk_front<2><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
     else if (s <= 4) k_chunk_front<4><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
     else if (s <= 8) k_chunk_front<8><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else k_chunk_front<16><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 16) k_chunk_front<16><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else k_chunk_front<32><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
     *launches += 1;
     size_t smem = 0;
     switch (ws->kp) {
@@ -709,7 +717,8 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
         case 16: e = corr_setup<16>(&smem); break;
         case 32: e = corr_setup<32>(&smem); break;
         case 64: e = corr_setup<64>(&smem); break;
-        default: e = corr_setup<128>(&smem); break;
+        case 128: e = corr_setup<128>(&smem); break;
+        default: e = corr_setup<256>(&smem); break;
     }
     if (e != cudaSuccess) return e;
     for (int iter = 0; iter < s; ++iter) {
@@ -736,7 +745,8 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
             case 16: corr_launch<16>(a, iter, smem, stream, gate); break;
             case 32: corr_launch<32>(a, iter, smem, stream, gate); break;
             case 64: corr_launch<64>(a, iter, smem, stream, gate); break;
-            default: corr_launch<128>(a, iter, smem, stream, gate); break;
+            case 128: corr_launch<128>(a, iter, smem, stream, gate); break;
+            default: corr_launch<256>(a, iter, smem, stream, gate); break;
         }
         k_chunk_pick<<<2 * c, 32, 0, stream>>>(a, iter, gate, gate ? ws->unresolved : nullptr);
         *launches += 2;

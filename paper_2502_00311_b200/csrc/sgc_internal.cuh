@@ -316,7 +316,7 @@ cudaError_t launch_reproject(sgc_state* st, uint64_t new_seed, cudaStream_t stre
 cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches);
 cudaError_t launch_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, float* out,
                            cudaStream_t stream);
-// MESGC with small per-chunk problems (s <= 16, k <= 128): the whole step of all chunks in 2 + 2s launches
+// MESGC with small per-chunk problems (s <= 32, k <= 256): the whole step of all chunks in 2 + 2s launches
 bool chunked_batch_eligible(sgc_state* const* sts, int c);
 cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad, float* weight, cudaStream_t stream,
                                  int* launches);
