@@ -255,3 +255,24 @@ class Oracle:
         if rc != 0:
             raise RuntimeError("orc_get(%s) failed: %d" % (name, rc))
         return out[0] if dim is None else out
+
+
+def cesgc_step(chunks, B, G, W):
+    """One CESGC step (Section 4.4, "Compute Efficient SGC") written out from its definition, W <- W - eta B^T SGC(B G).
+
+    chunks: the c chunk oracles (Oracle objects of length r * n / c each, same seed: MESGC on the projected gradient);
+    B: float32 [r, m]; G: float32 [m, n]; W: float32 [m, n], updated in place.  P = B G is formed in fp64 and rounded
+    to float32 (the gradient the SGC core is given); every chunk steps on its slice of P with zero "weights", which
+    leaves -eta N there; the result goes back through B^T in fp64.  Returns (P, U) with U = -eta N as float32 [r, n]."""
+    r, m = B.shape
+    n = G.shape[1]
+    assert G.shape == (m, n) and W.shape == (m, n) and W.dtype == np.float32
+    P = (B.astype(np.float64) @ G.astype(np.float64)).astype(np.float32)
+    U = np.zeros(r * n, dtype=np.float32)
+    dc = r * n // len(chunks)
+    flat = P.reshape(-1)
+    for i, ch in enumerate(chunks):
+        ch.step(np.ascontiguousarray(flat[i * dc:(i + 1) * dc]), U[i * dc:(i + 1) * dc])
+    U2 = U.reshape(r, n)
+    W[...] = (W.astype(np.float64) + B.astype(np.float64).T @ U2.astype(np.float64)).astype(np.float32)
+    return P, U2

@@ -155,3 +155,52 @@ def test_reprojection_moves_an_exactly_sparse_state_to_the_new_matrix():
     assert sorted(o.get("lamM").tolist()) == supp.tolist() == sorted(o.get("lamV").tolist())
     np.testing.assert_allclose(w2[supp], -1e-3 * np.sign(g[supp]), rtol=0, atol=2e-8)
     o.close()
+
+
+# ---- CESGC (Section 4.4): SGC on the projected gradient, update back through B^T --------------------------------
+def test_cesgc_with_an_identity_projection_is_the_chunked_step_itself():
+    # r = m and B = I: B G = G and B^T N = N, so the step must equal the chunk oracles run on G directly
+    m, n, c, k, sc, seed = 8, 64, 4, 24, 2, 3
+    rng = np.random.default_rng(1)
+    G = (rng.standard_t(3.0, size=(m, n)) * 1e-2).astype(np.float32)
+    W0 = rng.standard_normal((m, n)).astype(np.float32)
+    a = [oracle.Oracle(m * n // c, k, sc, seed, 1e-3, 0.9, 0.999, 1e-8) for _ in range(c)]
+    b = [oracle.Oracle(m * n // c, k, sc, seed, 1e-3, 0.9, 0.999, 1e-8) for _ in range(c)]
+    Wa, Wb = W0.copy(), W0.copy()
+    for _ in range(2):
+        oracle.cesgc_step(a, np.eye(m, dtype=np.float32), G, Wa)
+        flat = Wb.reshape(-1)
+        dc = m * n // c
+        for i, ch in enumerate(b):
+            ch.step(np.ascontiguousarray(G.reshape(-1)[i * dc:(i + 1) * dc]), flat[i * dc:(i + 1) * dc])
+        for x, y in zip(a, b):
+            assert np.array_equal(x.get("lamM"), y.get("lamM")) and np.array_equal(x.get("M"), y.get("M"))
+        np.testing.assert_allclose(Wa, Wb, rtol=0, atol=2e-7)
+    for ch in a + b:
+        ch.close()
+
+
+def test_cesgc_update_lives_in_the_row_space_of_the_projection_and_matches_its_formula():
+    # orthonormal B (first r left-singular vectors of G): the weight change is B^T U with U = -eta N at most s-sparse,
+    # so it is orthogonal to every direction outside the span of B's rows, and B (W1 - W0) returns U itself
+    m, n, r, c, k, sc, seed = 48, 40, 6, 3, 32, 3, 5
+    rng = np.random.default_rng(2)
+    G = (rng.standard_normal((m, 4)) @ rng.standard_normal((4, n)) + 0.05 * rng.standard_normal((m, n))).astype(np.float32)
+    Um, _, _ = np.linalg.svd(G.astype(np.float64), full_matrices=True)
+    B = np.ascontiguousarray(Um[:, :r].T).astype(np.float32)
+    chunks = [oracle.Oracle(r * n // c, k, sc, seed, 1e-3, 0.9, 0.999, 1e-8) for _ in range(c)]
+    W0 = rng.standard_normal((m, n)).astype(np.float32)
+    W1 = W0.copy()
+    P, U = oracle.cesgc_step(chunks, B, G, W1)
+    np.testing.assert_allclose(P, B.astype(np.float64) @ G, rtol=1e-6, atol=1e-7)
+    assert 0 < np.count_nonzero(U) <= c * sc
+    dW = W1.astype(np.float64) - W0
+    np.testing.assert_allclose(Um[:, r:].T @ dW, 0.0, atol=2e-6)                  # nothing outside the row space of B
+    np.testing.assert_allclose(B.astype(np.float64) @ dW, U, rtol=0, atol=2e-6)   # B B^T = I on that space
+    # the non-zeros of U are each chunk's update record
+    dc = r * n // c
+    for i, ch in enumerate(chunks):
+        nz = np.nonzero(U.reshape(-1)[i * dc:(i + 1) * dc])[0]
+        assert np.array_equal(nz, np.sort(ch.get("upd_idx")[:ch.get("n_upd")]))
+    for ch in chunks:
+        ch.close()
