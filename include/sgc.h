@@ -143,6 +143,22 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
  * not happen inside a stream capture.  SGC_ERR_GROUP when the states differ in (d, k, s, seed) or one appears twice. */
 SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* grad, float* weight, void* stream);
 
+/* Compute-efficient SGC (CESGC, Section 4.4 "Efficient SGC"): the gradient of an m x n weight matrix is first
+ * compressed with a projection B (r x m, rows orthonormal; the paper takes the first r left-singular vectors of a
+ * gradient and renews them every fixed number of iterations -- computing B is the caller's business), SGC runs on the
+ * r x n matrix B G, chunked as in sgc_step_chunked, and the update returns through B^T:
+ *     W <- W - eta B^T SGC(B G).
+ *   states       c states created with sgc_create(r * n / c, k, s_c, seed, ...); chunk i covers the flat range
+ *                [i * r n / c, (i + 1) * r n / c) of the row-major r x n matrix (r * n / c a multiple of 4)
+ *   B            device, r x m row-major floats, read-only; r <= 64
+ *   grad         device, m x n row-major floats, read-only
+ *   weight       device, m x n row-major floats; column j changes where SGC's update has a non-zero in column j
+ *   scratch      device, 2 * r * n floats, 16-byte aligned, owned by the caller, overwritten: B G, then -eta N
+ * B G is rounded once, from fp64 sums, so the kept entries are those of the exactly projected gradient.
+ * Enqueued on stream.  Errors: as sgc_step_chunked; SGC_ERR_DIM for r < 1, r > 64, m < 1, n < 1 or c not dividing r * n. */
+SGC_API int sgc_cesgc_step(sgc_state* const* states, int32_t c, const float* B, int32_t r, int32_t m, int32_t n,
+                           const float* grad, float* weight, float* scratch, void* stream);
+
 /* Waits for the state's last enqueued work, then frees everything.  NULL is accepted. */
 SGC_API int sgc_destroy(sgc_state* st);
 

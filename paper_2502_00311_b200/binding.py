@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libsgc_b200.so")
 _lib = None
 
-EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
+EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_cesgc_step", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
            "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
            "sgc_set_mode", "sgc_set_recovery", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version"]
 
@@ -60,6 +60,8 @@ def lib():
         L.sgc_step_group.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.c_int32, vp]
         L.sgc_step_chunked.restype = C.c_int
         L.sgc_step_chunked.argtypes = [C.POINTER(vp), C.c_int32, vp, vp, vp]
+        L.sgc_cesgc_step.restype = C.c_int
+        L.sgc_cesgc_step.argtypes = [C.POINTER(vp), C.c_int32, vp, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp]
         L.sgc_destroy.restype = C.c_int
         L.sgc_destroy.argtypes = [vp]
         L.sgc_set_alpha.restype = C.c_int
@@ -264,6 +266,36 @@ class Mesgc:
     def close(self):
         for st in self.chunks:
             st.close()
+
+
+class Cesgc:
+    """Compute-efficient SGC (Section 4.4): SGC, chunked, on the projected gradient B G of an m x n matrix; the update
+    returns through B^T (sgc_cesgc_step).  B (r x m, float32, CUDA) is the caller's: set_projection() stores it."""
+
+    def __init__(self, m, n, r, c, k, s_c, seed, lr, beta1, beta2, eps, alpha=None):
+        import torch
+        if (r * n) % c:
+            raise ValueError("r * n must be a multiple of the number of chunks")
+        self.m, self.n, self.r, self.c = int(m), int(n), int(r), int(c)
+        self.core = Mesgc(r * n, c, k, s_c, seed, lr, beta1, beta2, eps, alpha=alpha)
+        self.scratch = torch.empty(2 * r * n, dtype=torch.float32, device="cuda")
+        self.B = None
+
+    def set_projection(self, B):
+        if B.shape != (self.r, self.m) or not B.is_cuda or not B.is_contiguous() or B.element_size() != 4:
+            raise TypeError("B must be a contiguous float32 CUDA tensor of shape (r, m)")
+        self.B = B
+
+    def step(self, grad, weight, stream=None):
+        if self.B is None:
+            raise ValueError("set_projection() first")
+        d = self.m * self.n
+        _check(lib().sgc_cesgc_step(self.core._hs, self.c, C.c_void_p(self.B.data_ptr()), self.r, self.m, self.n,
+                                    _dev_ptr(grad, d, "grad"), _dev_ptr(weight, d, "weight"),
+                                    C.c_void_p(self.scratch.data_ptr()), _stream_ptr(stream)), "sgc_cesgc_step")
+
+    def close(self):
+        self.core.close()
 
 
 def step_group(states, grads, weights, stream=None):

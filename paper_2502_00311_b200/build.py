@@ -6,7 +6,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libsgc_b200.so")
-SOURCES = ["sgc_api.cu", "sgc_select.cu", "sgc_project.cu", "sgc_recover.cu", "sgc_pass.cu", "sgc_chunked.cu"]
+SOURCES = ["sgc_api.cu", "sgc_select.cu", "sgc_project.cu", "sgc_recover.cu", "sgc_pass.cu", "sgc_chunked.cu", "sgc_cesgc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -197,6 +197,25 @@ SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* g
     return sgc_step_group(states, gs.data(), ws.data(), c, stream);
 }
 
+SGC_API int sgc_cesgc_step(sgc_state* const* states, int32_t c, const float* B, int32_t r, int32_t m, int32_t n,
+                           const float* grad, float* weight, float* scratch, void* stream) {
+    if (!states || !B || !grad || !weight || !scratch) return SGC_ERR_NULL;
+    if (c < 1 || !sgc::cesgc_shape_ok(r, m, n)) return SGC_ERR_DIM;
+    if (!states[0]) return SGC_ERR_NULL;
+    const int64_t dp = (int64_t)r * n;
+    if (dp % c != 0 || states[0]->d != dp / c) return SGC_ERR_DIM;
+    if ((uintptr_t)scratch & 15u) return SGC_ERR_ALIGN;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    float* P = scratch;                  // B G
+    float* U = scratch + dp;             // the compressed problem's "weights": start at zero, end as -eta N
+    cudaError_t e = sgc::launch_cesgc_project(B, grad, P, r, m, n, cs);
+    if (e == cudaSuccess) e = cudaMemsetAsync(U, 0, (size_t)dp * sizeof(float), cs);
+    if (e != cudaSuccess) return (int)e;
+    const int rc = sgc_step_chunked(states, c, P, U, stream);
+    if (rc != SGC_OK) return rc;
+    return (int)sgc::launch_cesgc_back(B, U, weight, r, m, n, cs);
+}
+
 SGC_API int sgc_destroy(sgc_state* st) {
     if (!st) return SGC_OK;
     cudaError_t e = cudaSuccess;

@@ -1,0 +1,103 @@
+// CESGC (Section 4.4, "Compute Efficient SGC"): SGC runs on the projected gradient B G (r x n) instead of G (m x n), and
+// its update goes back through B^T:  W <- W - eta B^T SGC(B G).  B (r x m, the first r left-singular vectors of a
+// gradient, refreshed by the caller every few hundred steps) is an input here; the two projections around the SGC core
+// are the kernels of this file.
+//   k_cesgc_project   P = B G.  Thread = one column j of G and eight rows of B; G is read row by row (coalesced over j),
+//                     the rows of B come from shared memory as broadcasts.  Sums are carried in fp64, so that P is the
+//                     correctly rounded fp32 value of the exact product: the top-s selection that follows decides on
+//                     those values, and a reference computing B G in fp64 decides on the same ones.
+//   k_cesgc_back      W += B^T U for the r x n matrix U that the SGC core left (U = -eta N has at most s non-zeros):
+//                     block = one column of U; columns without a non-zero cost one read of r values.
+#include "sgc_internal.cuh"
+
+namespace sgc {
+namespace {
+
+constexpr int kProjCols = 64;            // columns of G per block
+constexpr int kProjRows = 8;             // rows of B per thread
+constexpr int kProjChunk = 64;           // rows of G per staged slab of B
+constexpr int kCesgcMaxR = 64;
+
+__global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows))
+k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float* __restrict__ P, int r, int m, int n) {
+    __shared__ float bs[kCesgcMaxR][kProjChunk];                      // B[:, row0 .. row0 + 64)
+    const int groups = (r + kProjRows - 1) / kProjRows;
+    const int jl = threadIdx.x % kProjCols, ig = threadIdx.x / kProjCols;
+    const int j = blockIdx.x * kProjCols + jl;
+    const bool work = ig < groups && j < n;
+    double acc[kProjRows];
+#pragma unroll
+    for (int u = 0; u < kProjRows; ++u) acc[u] = 0.0;
+    for (int row0 = 0; row0 < m; row0 += kProjChunk) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < r * kProjChunk; e += blockDim.x) {
+            const int i = e / kProjChunk, q = e % kProjChunk;
+            bs[i][q] = row0 + q < m ? B[(size_t)i * m + row0 + q] : 0.0f;
+        }
+        __syncthreads();
+        if (!work) continue;
+        const int rows = m - row0 < kProjChunk ? m - row0 : kProjChunk;
+        for (int q = 0; q < rows; ++q) {
+            const double g = (double)G[(size_t)(row0 + q) * n + j];
+#pragma unroll
+            for (int u = 0; u < kProjRows; ++u) acc[u] = acc[u] + (double)bs[ig * kProjRows + u][q] * g;
+        }
+    }
+    if (work) {
+#pragma unroll
+        for (int u = 0; u < kProjRows; ++u) {
+            const int i = ig * kProjRows + u;
+            if (i < r) P[(size_t)i * n + j] = (float)acc[u];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_cesgc_back(const float* __restrict__ B, const float* __restrict__ U, float* __restrict__ W, int r, int m, int n) {
+    __shared__ float us[kCesgcMaxR];
+    __shared__ int idx[kCesgcMaxR];
+    __shared__ int n_nz;
+    const int j = blockIdx.x;
+    if (threadIdx.x == 0) n_nz = 0;
+    __syncthreads();
+    if ((int)threadIdx.x < r) {
+        const float u = U[(size_t)threadIdx.x * n + j];
+        if (u != 0.0f) { const int slot = atomicAdd(&n_nz, 1); us[slot] = u; idx[slot] = threadIdx.x; }
+    }
+    __syncthreads();
+    const int nz = n_nz;
+    if (nz == 0) return;
+    // ascending row order of B, whatever order the atomics gave: the sum below does not depend on the schedule
+    if (threadIdx.x == 0) {
+        for (int a = 1; a < nz; ++a) {
+            const int ia = idx[a]; const float ua = us[a];
+            int b = a - 1;
+            while (b >= 0 && idx[b] > ia) { idx[b + 1] = idx[b]; us[b + 1] = us[b]; --b; }
+            idx[b + 1] = ia; us[b + 1] = ua;
+        }
+    }
+    __syncthreads();
+    for (int row = threadIdx.x; row < m; row += 256) {
+        double acc = 0.0;
+        for (int a = 0; a < nz; ++a) acc += (double)B[(size_t)idx[a] * m + row] * (double)us[a];
+        float* w = W + (size_t)row * n + j;
+        *w = (float)((double)*w + acc);
+    }
+}
+
+}  // namespace
+
+bool cesgc_shape_ok(int r, int m, int n) { return r >= 1 && r <= kCesgcMaxR && m >= 1 && n >= 1; }
+
+cudaError_t launch_cesgc_project(const float* B, const float* G, float* P, int r, int m, int n, cudaStream_t stream) {
+    const int groups = (r + kProjRows - 1) / kProjRows;
+    k_cesgc_project<<<(n + kProjCols - 1) / kProjCols, kProjCols * groups, 0, stream>>>(B, G, P, r, m, n);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_cesgc_back(const float* B, const float* U, float* W, int r, int m, int n, cudaStream_t stream) {
+    k_cesgc_back<<<n, 256, 0, stream>>>(B, U, W, r, m, n);
+    return cudaGetLastError();
+}
+
+}  // namespace sgc

@@ -321,6 +321,10 @@ bool chunked_batch_eligible(sgc_state* const* sts, int c);
 cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad, float* weight, cudaStream_t stream,
                                  int* launches);
 void free_chunk_ws(sgc_state* st);
+// CESGC projections (sgc_cesgc.cu): P = B G and W += B^T U
+bool cesgc_shape_ok(int r, int m, int n);
+cudaError_t launch_cesgc_project(const float* B, const float* G, float* P, int r, int m, int n, cudaStream_t stream);
+cudaError_t launch_cesgc_back(const float* B, const float* U, float* W, int r, int m, int n, cudaStream_t stream);
 double normal_tail_threshold(double d, double target);   // z with d * P(|N(0,1)| > z) = target
 cudaError_t configure_recover(sgc_state* st);   // occupancy / shared-memory set-up at create time
 cudaError_t finish_recover_setup(sgc_state* st); // after the workspace exists: tensor map of R^T

@@ -538,6 +538,61 @@ def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
     m.close()
 
 
+@pytest.mark.parametrize("m,n,r,c,k,sc", [(512, 256, 8, 4, 28, 4), (1000, 384, 32, 16, 56, 8), (4096, 512, 32, 8, 217, 31)])
+def test_cesgc_step_matches_its_oracle(sgc, m, n, r, c, k, sc):
+    # Section 4.4: SGC (chunked) on B G, update back through B^T; B = first r left-singular vectors of the first gradient
+    hp = inputs.ADAM
+    rng = np.random.default_rng(m + r)
+    low = rng.standard_normal((m, 6)) @ rng.standard_normal((6, n))
+    ce = sgc.Cesgc(m, n, r, c, k, sc, 9, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0)
+    refs = [oracle.Oracle(r * n // c, k, sc, 9, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0) for _ in range(c)]
+    W_ref = (rng.standard_normal((m, n)) * 0.02).astype(np.float32)
+    w_gpu = cuda(W_ref.copy())
+    B = None
+    for step in range(1, 4):
+        G = (low * (1.0 + 0.1 * step) + 0.3 * rng.standard_t(3.0, size=(m, n))).astype(np.float32)
+        if B is None:
+            U, _, _ = np.linalg.svd(G.astype(np.float64), full_matrices=False)
+            B = np.ascontiguousarray(U[:, :r].T).astype(np.float32)
+            ce.set_projection(cuda(B))
+        W_before = W_ref.copy()
+        P, Uref = oracle.cesgc_step(refs, B, G, W_ref)
+        ce.step(cuda(G), w_gpu)
+        import torch
+        torch.cuda.synchronize()
+        got_P = ce.scratch[: r * n].cpu().numpy().reshape(r, n)
+        assert np.array_equal(got_P, P), "B G is not the correctly rounded product"
+        for i in range(c):
+            st = ce.core.chunks[i]
+            for name in ("sel_idx", "lamM", "lamV", "upd_idx"):
+                assert np.array_equal(st.get(name), refs[i].get(name)), (name, i, step)
+        got_U = ce.scratch[r * n:].cpu().numpy().reshape(r, n)
+        assert np.array_equal(got_U != 0, Uref != 0)
+        assert rel(got_U, Uref) < TOL_UPDATE
+        wg = w_gpu.cpu().numpy()
+        dw_g = wg.astype(np.float64) - W_before
+        dw_r = W_ref.astype(np.float64) - W_before
+        cols = np.nonzero(np.any(Uref != 0, axis=0))[0]
+        other = np.setdiff1d(np.arange(n), cols)
+        assert np.array_equal(wg[:, other], W_before[:, other])          # columns without an update are not written
+        assert np.abs(dw_g - dw_r).max() <= TOL_UPDATE * np.abs(dw_r).max() + 1.2e-7 * np.abs(W_before).max()
+    ce.close()
+    for rf in refs:
+        rf.close()
+
+
+def test_cesgc_step_rejects_bad_shapes(sgc):
+    import torch
+    ce = sgc.Cesgc(64, 32, 4, 2, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
+    g, w = torch.zeros(64, 32, device="cuda"), torch.zeros(64, 32, device="cuda")
+    B = torch.zeros(4, 64, device="cuda")
+    call = lambda r, m, n: sgc.lib().sgc_cesgc_step(ce.core._hs, 2, B.data_ptr(), r, m, n, g.data_ptr(), w.data_ptr(),
+                                                      ce.scratch.data_ptr(), None)
+    assert call(0, 64, 32) != 0 and call(65, 64, 32) != 0 and call(4, 64, 31) != 0 and call(4, 0, 32) != 0
+    assert ce.core.chunks[0].get("t") == 0
+    ce.close()
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 def test_sgca_reprojection_matches_the_oracle(sgc, mode):
     # Algorithm 4: every T = 2 steps the matrix is replaced and M, V are re-aligned; the steps after that run under the
