@@ -154,7 +154,8 @@ SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* g
  *   grad         device, m x n row-major floats, read-only
  *   weight       device, m x n row-major floats; column j changes where SGC's update has a non-zero in column j
  *   scratch      device, 2 * r * n floats, 16-byte aligned, owned by the caller, overwritten: B G, then -eta N
- * B G is rounded once, from fp64 sums, so the kept entries are those of the exactly projected gradient.
+ * B G is accumulated to about 44 bits and rounded to fp32 once, so the kept entries are those of the exactly projected
+ * gradient (a product formed in fp64 differs by one ulp in a few elements per ten thousand).
  * Enqueued on stream.  Errors: as sgc_step_chunked; SGC_ERR_DIM for r < 1, r > 64, m < 1, n < 1 or c not dividing r * n. */
 SGC_API int sgc_cesgc_step(sgc_state* const* states, int32_t c, const float* B, int32_t r, int32_t m, int32_t n,
                            const float* grad, float* weight, float* scratch, void* stream);

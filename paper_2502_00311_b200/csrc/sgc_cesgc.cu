@@ -3,9 +3,12 @@
 // gradient, refreshed by the caller every few hundred steps) is an input here; the two projections around the SGC core
 // are the kernels of this file.
 //   k_cesgc_project   P = B G.  Thread = one column j of G and eight rows of B; G is read row by row (coalesced over j),
-//                     the rows of B come from shared memory as broadcasts.  Sums are carried in fp64, so that P is the
-//                     correctly rounded fp32 value of the exact product: the top-s selection that follows decides on
-//                     those values, and a reference computing B G in fp64 decides on the same ones.
+//                     the rows of B come from shared memory as broadcasts.  Sums are carried as pairs of floats (error-free
+//                     product through one FMA, error-free two-term sum: some 44 bits in all; fp64 arithmetic runs at a
+//                     64th of the fp32 rate on this part and made this kernel 1.1 ms), and rounded to fp32 once at the
+//                     end.  The top-s selection that follows decides on those values; a reference that forms B G in fp64
+//                     gets the same fp32 numbers but for a few elements in ten thousand (entries much smaller than
+//                     their terms), which differ by one ulp.  Slabs of B and G are staged in shared memory.
 //   k_cesgc_back      W += B^T U for the r x n matrix U that the SGC core left (U = -eta N has at most s non-zeros):
 //                     block = one column of U; columns without a non-zero cost one read of r values.
 #include "sgc_internal.cuh"
@@ -13,7 +16,7 @@
 namespace sgc {
 namespace {
 
-constexpr int kProjCols = 64;            // columns of G per block
+constexpr int kProjCols = 32;            // columns of G per block
 constexpr int kProjRows = 8;             // rows of B per thread
 constexpr int kProjChunk = 64;           // rows of G per staged slab of B
 constexpr int kCesgcMaxR = 64;
@@ -21,33 +24,48 @@ constexpr int kCesgcMaxR = 64;
 __global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows))
 k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float* __restrict__ P, int r, int m, int n) {
     __shared__ float bs[kCesgcMaxR][kProjChunk];                      // B[:, row0 .. row0 + 64)
+    __shared__ float gs[kProjChunk][kProjCols];                       // G[row0 .. row0 + 64, the block's columns]
     const int groups = (r + kProjRows - 1) / kProjRows;
     const int jl = threadIdx.x % kProjCols, ig = threadIdx.x / kProjCols;
     const int j = blockIdx.x * kProjCols + jl;
     const bool work = ig < groups && j < n;
-    double acc[kProjRows];
+    float hi[kProjRows], lo[kProjRows];
 #pragma unroll
-    for (int u = 0; u < kProjRows; ++u) acc[u] = 0.0;
+    for (int u = 0; u < kProjRows; ++u) hi[u] = lo[u] = 0.0f;
     for (int row0 = 0; row0 < m; row0 += kProjChunk) {
         __syncthreads();
         for (int e = threadIdx.x; e < r * kProjChunk; e += blockDim.x) {
             const int i = e / kProjChunk, q = e % kProjChunk;
             bs[i][q] = row0 + q < m ? B[(size_t)i * m + row0 + q] : 0.0f;
         }
+        for (int e = threadIdx.x; e < kProjChunk * kProjCols; e += blockDim.x) {       // many independent loads in flight
+            const int q = e / kProjCols, c = e % kProjCols;
+            const int col = blockIdx.x * kProjCols + c;
+            gs[q][c] = (row0 + q < m && col < n) ? G[(size_t)(row0 + q) * n + col] : 0.0f;
+        }
         __syncthreads();
         if (!work) continue;
         const int rows = m - row0 < kProjChunk ? m - row0 : kProjChunk;
         for (int q = 0; q < rows; ++q) {
-            const double g = (double)G[(size_t)(row0 + q) * n + j];
+            const float g = gs[q][jl];
 #pragma unroll
-            for (int u = 0; u < kProjRows; ++u) acc[u] = acc[u] + (double)bs[ig * kProjRows + u][q] * g;
+            for (int u = 0; u < kProjRows; ++u) {
+                const float b = bs[ig * kProjRows + u][q];
+                const float p = __fmul_rn(b, g);
+                const float pe = __fmaf_rn(b, g, -p);                 // b g = p + pe exactly
+                const float t = __fadd_rn(hi[u], p);
+                const float v = __fsub_rn(t, hi[u]);
+                const float te = __fadd_rn(__fsub_rn(hi[u], __fsub_rn(t, v)), __fsub_rn(p, v));   // hi + p = t + te exactly
+                hi[u] = t;
+                lo[u] = __fadd_rn(lo[u], __fadd_rn(te, pe));
+            }
         }
     }
     if (work) {
 #pragma unroll
         for (int u = 0; u < kProjRows; ++u) {
             const int i = ig * kProjRows + u;
-            if (i < r) P[(size_t)i * n + j] = (float)acc[u];
+            if (i < r) P[(size_t)i * n + j] = (float)((double)hi[u] + (double)lo[u]);
         }
     }
 }

@@ -163,6 +163,8 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
     extern __shared__ float smem[];
     float* zt = smem;                                                // [TC][ZS]
     float* inv = smem + TC * ZS;                                     // [TC]
+    float* n2p = inv + TC;                                           // [GPC][TC] partial ||Z_i||^2
+    constexpr int GPC = kCorrBlock / TC, RG = KP / GPC;              // generating threads per column, rows each
     const int h = threadIdx.x % KS;
     const int res = blockIdx.y * (kCorrBlock / KS) + threadIdx.x / KS;     // recovery = 2 * chunk + moment
     const bool have = res < 2 * a.c;
@@ -186,27 +188,37 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
     if (col1 > a.dc) col1 = a.dc;
     for (long long tile = col0; tile < col1; tile += TC) {
         __syncthreads();
-        for (int t = threadIdx.x; t < TC; t += kCorrBlock) {
+        {
+            // every thread generates: GPC threads share a column of the tile, RG rows each
+            const int t = threadIdx.x % TC, part = threadIdx.x / TC;
             const long long col = tile + t;
             float n2 = 0.0f;
-            float* dst = zt + t * ZS;
+            float* dst = zt + t * ZS + part * RG;
             if (col < col1) {
                 const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)col);
-                uint32_t hw = key.ck;
+                uint32_t hw = key.ck + (uint32_t)(part * RG / 2) * key.mk;
 #pragma unroll 4
-                for (int row = 0; row < KP; row += 2) {
+                for (int q = 0; q < RG; q += 2) {
+                    const int row = part * RG + q;
                     float2 z = half2_bits_to_float2(z_pair_from_word(hw));
                     hw += key.mk;
                     if (row >= a.k) z.x = 0.0f;
                     if (row + 1 >= a.k) z.y = 0.0f;
-                    dst[row] = z.x; dst[row + 1] = z.y;
+                    dst[q] = z.x; dst[q + 1] = z.y;
                     n2 = __fmaf_rn(z.x, z.x, n2);
                     n2 = __fmaf_rn(z.y, z.y, n2);
                 }
             } else {
-                for (int row = 0; row < KP; ++row) dst[row] = 0.0f;
+                for (int q = 0; q < RG; ++q) dst[q] = 0.0f;
             }
-            inv[t] = n2 > 0.0f ? 1.0f / sqrtf(n2) : 0.0f;
+            n2p[part * TC + t] = n2;
+        }
+        __syncthreads();
+        if (threadIdx.x < TC) {
+            float n2 = 0.0f;
+#pragma unroll
+            for (int g = 0; g < GPC; ++g) n2 += n2p[g * TC + threadIdx.x];
+            inv[threadIdx.x] = n2 > 0.0f ? 1.0f / sqrtf(n2) : 0.0f;
         }
         __syncthreads();
         if (KS == 1 && !active) continue;                            // (with KS = 2 the shuffle below needs every lane)
@@ -557,7 +569,7 @@ unsigned long long list_key(sgc_state* const* sts, int c) {
 template <int KP>
 cudaError_t corr_setup(size_t* smem_out) {
     constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 64);
-    const size_t smem = (size_t)(TC * (KP + 4) + TC) * sizeof(float);
+    const size_t smem = (size_t)(TC * (KP + 4) + TC + kCorrBlock) * sizeof(float);
     *smem_out = smem;
     return cudaFuncSetAttribute(k_chunk_corr<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
@@ -598,7 +610,8 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     const size_t b_r32 = up((size_t)2 * c * ws->kp * sizeof(float));
     const size_t b_cand = up((size_t)2 * c * splits * 2 * sizeof(Cand));
     // tensor-core route: worth it from k_c = 33 on; bounded by its report lists (n_rows * 16 KB)
-    ws->tensor = ws->kp >= 64 && 2 * c <= 2048 && st0->d >= 1024;
+    // (a pass has some 40 us of fixed cost: below ~1e9 multiply-adds per iteration the fp32 kernel is quicker)
+    ws->tensor = ws->kp >= 64 && 2 * c <= 2048 && (double)st0->d * ws->kp * 2.0 * c >= 1.0e9;
     ws->kp64 = (st0->k + 63) / 64 * 64;
     ws->n_rows = (2 * c + 31) / 32 * 32;
     ws->passes = (ws->n_rows + kPassMaxN - 1) / kPassMaxN;
