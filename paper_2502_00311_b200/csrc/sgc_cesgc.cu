@@ -2,7 +2,7 @@
 // its update goes back through B^T:  W <- W - eta B^T SGC(B G).  B (r x m, the first r left-singular vectors of a
 // gradient, refreshed by the caller every few hundred steps) is an input here; the two projections around the SGC core
 // are the kernels of this file.
-//   k_cesgc_project   P = B G.  Thread = one column j of G and eight rows of B; G is read row by row (coalesced over j),
+//   k_cesgc_project   P = B G.  Thread = one column j of G and four rows of B; G is read row by row (coalesced over j),
 //                     the rows of B come from shared memory as broadcasts.  Sums are carried as pairs of floats (error-free
 //                     product through one FMA, error-free two-term sum: some 44 bits in all; fp64 arithmetic runs at a
 //                     64th of the fp32 rate on this part and made this kernel 1.1 ms), and rounded to fp32 once at the
@@ -17,7 +17,7 @@ namespace sgc {
 namespace {
 
 constexpr int kProjCols = 32;            // columns of G per block
-constexpr int kProjRows = 8;             // rows of B per thread
+constexpr int kProjRows = 4;             // rows of B per thread
 constexpr int kProjChunk = 64;           // rows of G per staged slab of B
 constexpr int kCesgcMaxR = 64;
 
