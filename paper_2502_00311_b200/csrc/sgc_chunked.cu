@@ -7,7 +7,7 @@
 //   generated once and meets the residuals of every chunk):
 //     k_chunk_corr   thread = one residual, block = 256 residuals x a range of columns: fp32 scores |<A_i,r>| / ||A_i||,
 //                    best two columns of the range per residual
-//     k_chunk_pick   warp = one recovery: fp64 rescoring of the columns within 2e-3 of the best fp32 score, lowest
+//     k_chunk_pick   block of 128 threads = one recovery: fp64 rescoring of the columns within 2e-3 of the best fp32 score, lowest
 //                    index on ties, then the inverse-Cholesky recurrences of Algorithm 3, x, r
 //   k_chunk_scatter  warp = chunk: Eq. (8) on the common support, weight update (a5)
 // Every record lands in the chunk's own state, so sgc_get works per chunk exactly as after sgc_step.
@@ -255,26 +255,55 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
     }
 }
 
-// ---- phase B of one OMP iteration: one warp per recovery ---------------------------------------------------
+// ---- phase B of one OMP iteration: one block of kPickThreads threads per recovery ---------------------------------------------------
 // Argmax among the columns that phase A left within 2e-3 (relative) of the best fp32 score, decided on fp64 scores
 // <Z_i, r>^2 / ||Z_i||^2 with the lowest index winning ties; then Algorithm 3 (Appendix B) for the new column:
 // g = A_Lambda^T a_new, c = F^T g, gamma = 1 / sqrt(g_ll - c^T c) (a pivot below 1e-10 g_ll ends this recovery),
 // new column [-gamma F c; gamma] of F, a_j = gamma <a_new, r>, x = F a, r = y - A_Lambda x.
+constexpr int kPickThreads = 128;        // one block per recovery
+
 struct PickSmem {
     double gv[kChunkMaxS], cv[kChunkMaxS], xs[kChunkMaxS];
+    double red[2][kPickThreads / 32];
+    double csq;
     uint32_t cidx[kRescoreCap];
     int n_c;
+    float fred[kPickThreads / 32];
 };
 
+// sums of two values over the block; every thread receives both
+__device__ __forceinline__ void pick_sum2(PickSmem& sh, double& a, double& b) {
+    a = warp_sum_d(a); b = warp_sum_d(b);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) { sh.red[0][threadIdx.x >> 5] = a; sh.red[1][threadIdx.x >> 5] = b; }
+    __syncthreads();
+    a = 0.0; b = 0.0;
+#pragma unroll
+    for (int w = 0; w < kPickThreads / 32; ++w) { a += sh.red[0][w]; b += sh.red[1][w]; }
+}
+
+// largest value over the block; every thread receives it
+__device__ __forceinline__ float pick_max(PickSmem& sh, float v) {
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh.fred[threadIdx.x >> 5] = v;
+    __syncthreads();
+    v = sh.fred[0];
+#pragma unroll
+    for (int w = 1; w < kPickThreads / 32; ++w) v = fmaxf(v, sh.fred[w]);
+    return v;
+}
+
 // the decision among the nc candidates in sh.cidx and the update of the recovery `res` with the winner as pick j
+// (all kPickThreads threads of the block; nc is the same in every thread)
 __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& sh, int res, int j, int nc) {
     double* gv = sh.gv; double* cv = sh.cv; double* xs = sh.xs;
     const uint32_t* cidx = sh.cidx;
-    const int m = res & 1, lane = threadIdx.x, k = a.k, s = a.s;
+    const int m = res & 1, t = threadIdx.x, lane = t & 31, warp = t >> 5, k = a.k, s = a.s;
     double* r = ref.r64 + (size_t)m * k;
     const double* y = ref.y64 + (size_t)m * k;
     if (nc == 0) {                                                   // no column left to pick (d/c = iterations made)
-        if (lane == 0) { ref.cnt->stopped[m] = 1; ref.cnt->done[m] = j; }
+        if (t == 0) { ref.cnt->stopped[m] = 1; ref.cnt->done[m] = j; }
         return;
     }
     // fp64 scores of the candidates
@@ -284,13 +313,13 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         const uint32_t idx = cidx[c];
         const ColKey key = column_key(a.seed_lo, a.seed_hi, idx);
         double dot = 0.0, n2 = 0.0;
-        for (int row = 2 * lane; row < k; row += 64) {
+        for (int row = 2 * t; row < k; row += 2 * kPickThreads) {
             const float2 zz = half2_bits_to_float2(z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk));
             dot += (double)zz.x * r[row];
             n2 += (double)zz.x * (double)zz.x;
             if (row + 1 < k) { dot += (double)zz.y * r[row + 1]; n2 += (double)zz.y * (double)zz.y; }
         }
-        dot = warp_sum_d(dot); n2 = warp_sum_d(n2);
+        pick_sum2(sh, dot, n2);
         const double sc = n2 > 0.0 ? dot * dot / n2 : 0.0;
         if (sc > best_sc || (sc == best_sc && idx < best_idx)) { best_sc = sc; best_idx = idx; best_dot = dot; best_n2 = n2; }
     }
@@ -301,61 +330,68 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
     {
         const ColKey key = column_key(a.seed_lo, a.seed_hi, best_idx);
         uint16_t* znew = zs + (size_t)j * k;
-        for (int row = 2 * lane; row < k; row += 64) {
+        for (int row = 2 * t; row < k; row += 2 * kPickThreads) {
             const uint32_t z2 = z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk);
             znew[row] = (uint16_t)(z2 & 0xFFFFu);
             if (row + 1 < k) znew[row + 1] = (uint16_t)(z2 >> 16);
         }
     }
-    __syncwarp();
+    __syncthreads();
     const double sig2 = a.sigma * a.sigma;
     const uint16_t* znew = zs + (size_t)j * k;
-    for (int l = 0; l < j; ++l) {                                    // g = A_Lambda^T a_new
+    for (int l = warp; l < j; l += kPickThreads / 32) {              // g = A_Lambda^T a_new, one earlier column per warp
         const uint16_t* zl = zs + (size_t)l * k;
         double acc = 0.0;
         for (int row = lane; row < k; row += 32) acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));
         acc = warp_sum_d(acc);
         if (lane == 0) gv[l] = sig2 * acc;
     }
-    __syncwarp();
-    double csq = 0.0;
-    if (lane < j) {                                                  // c = F^T g (F upper triangular, F(l, i) at F[l*s + i])
-        double acc = 0.0;
-        for (int l = 0; l <= lane; ++l) acc += F[(size_t)l * s + lane] * gv[l];
-        cv[lane] = acc;
-        csq = acc * acc;
+    __syncthreads();
+    if (warp == 0) {
+        double csq = 0.0;
+        if (lane < j) {                                              // c = F^T g (F upper triangular, F(l, i) at F[l*s + i])
+            double acc = 0.0;
+            for (int l = 0; l <= lane; ++l) acc += F[(size_t)l * s + lane] * gv[l];
+            cv[lane] = acc;
+            csq = acc * acc;
+        }
+        csq = warp_sum_d(csq);
+        if (lane == 0) sh.csq = csq;
     }
-    csq = warp_sum_d(csq);
+    __syncthreads();
     const double gnn = sig2 * best_n2;
-    const double piv = gnn - csq;
+    const double piv = gnn - sh.csq;
     if (!(piv > 1e-10 * gnn)) {                                      // dependent column: this recovery ends with j picks
-        if (lane == 0) {
+        if (t == 0) {
             ref.cnt->stopped[m] = 1; ref.cnt->done[m] = j;
             atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_DEPENDENT_COLUMN);
         }
         return;
     }
     const double gamma = 1.0 / sqrt(piv);
-    __syncwarp();
-    if (lane < j) {
-        double acc = 0.0;
-        for (int l = lane; l < j; ++l) acc += F[(size_t)lane * s + l] * cv[l];
-        F[(size_t)lane * s + j] = -gamma * acc;
-    } else if (lane == j) {
-        F[(size_t)j * s + j] = gamma;
-    }
     const double aj = gamma * a.sigma * best_dot;
-    __syncwarp();
-    if (lane <= j) {
-        const double xo = lane < j ? xg[lane] : 0.0;
-        const double xn = xo + aj * F[(size_t)lane * s + j];
-        xg[lane] = xn;
-        xs[lane] = xn;
+    if (warp == 0) {
+        double fj = 0.0;                                             // this lane's entry of the new column of F
+        if (lane < j) {
+            double acc = 0.0;
+            for (int l = lane; l < j; ++l) acc += F[(size_t)lane * s + l] * cv[l];
+            fj = -gamma * acc;
+            F[(size_t)lane * s + j] = fj;
+        } else if (lane == j) {
+            fj = gamma;
+            F[(size_t)j * s + j] = fj;
+        }
+        if (lane <= j) {
+            const double xo = lane < j ? xg[lane] : 0.0;
+            const double xn = xo + aj * fj;
+            xg[lane] = xn;
+            xs[lane] = xn;
+        }
+        if (lane == 0) { ref.acoef[(size_t)m * s + j] = aj; ref.lam[(size_t)m * s + j] = best_idx; }
     }
-    if (lane == 0) { ref.acoef[(size_t)m * s + j] = aj; ref.lam[(size_t)m * s + j] = best_idx; }
-    __syncwarp();
-    double rn2 = 0.0;
-    for (int row = lane; row < k; row += 32) {                       // r = y - A_Lambda x
+    __syncthreads();
+    double rn2 = 0.0, unused = 0.0;
+    for (int row = t; row < k; row += kPickThreads) {                // r = y - A_Lambda x
         double acc = 0.0;
         for (int l = 0; l <= j; ++l) acc += xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
         const double rv = y[row] - a.sigma * acc;
@@ -363,8 +399,8 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         a.r32[(size_t)res * a.kp + row] = (float)rv;
         rn2 += rv * rv;
     }
-    rn2 = warp_sum_d(rn2);
-    if (lane == 0) {
+    pick_sum2(sh, rn2, unused);
+    if (t == 0) {
         ref.rnorm[(size_t)m * s + j] = sqrt(rn2);
         ref.cnt->done[m] = j + 1;
     }
@@ -372,35 +408,32 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
 
 // SIMT route: the candidates are the columns that phase A left within 2e-3 (relative) of the best fp32 score.
 // only != nullptr: a second chance for the recoveries that the tensor-core route marked unresolved; *gate == 0 skips it.
-__global__ void __launch_bounds__(32) k_chunk_pick(ChunkArgs a, int iter, const int* gate, const unsigned char* only) {
+__global__ void __launch_bounds__(kPickThreads) k_chunk_pick(ChunkArgs a, int iter, const int* gate, const unsigned char* only) {
     __shared__ PickSmem sh;
     if (gate != nullptr && *gate == 0) return;
-    const int res = blockIdx.x, m = res & 1, lane = threadIdx.x;
+    const int res = blockIdx.x, m = res & 1, t = threadIdx.x;
     if (only != nullptr && !only[res]) return;
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m]) return;
     const int j = iter;
-    uint32_t* cidx = sh.cidx;
-    int& n_c = sh.n_c;
     const Cand* cc = a.cand + (size_t)res * a.splits * 2;
     const int n_entries = a.splits * 2;
     float mx = -1.0f;
-    for (int e = lane; e < n_entries; e += 32) if (cc[e].idx != kNoColumn) mx = fmaxf(mx, cc[e].score);
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) n_c = 0;
-    __syncwarp();
+    for (int e = t; e < n_entries; e += kPickThreads) if (cc[e].idx != kNoColumn) mx = fmaxf(mx, cc[e].score);
+    if (t == 0) sh.n_c = 0;
+    mx = pick_max(sh, mx);                                          // (its barriers also publish n_c = 0)
     const float thr = mx - 2e-3f * fabsf(mx);
-    for (int e = lane; e < n_entries; e += 32) {
+    for (int e = t; e < n_entries; e += kPickThreads) {
         const Cand c = cc[e];
         if (c.idx != kNoColumn && c.score >= 0.0f && c.score >= thr) {
-            const int slot = atomicAdd(&n_c, 1);
-            if (slot < kRescoreCap) cidx[slot] = c.idx;
+            const int slot = atomicAdd(&sh.n_c, 1);
+            if (slot < kRescoreCap) sh.cidx[slot] = c.idx;
         }
     }
-    __syncwarp();
-    int nc = n_c;
+    __syncthreads();
+    int nc = sh.n_c;
     if (nc > kRescoreCap) {
-        if (lane == 0) atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
+        if (t == 0) atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
         nc = kRescoreCap;
     }
     pick_finish(a, ref, sh, res, j, nc);
@@ -448,24 +481,24 @@ __global__ void __launch_bounds__(64) k_chunk_rt(ChunkArgs a, int n_rows) {
     }
 }
 
-__global__ void __launch_bounds__(32) k_chunk_pick_rep(ChunkArgs a, int iter) {
+__global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, int iter) {
     __shared__ PickSmem sh;
-    const int res = blockIdx.x, m = res & 1, lane = threadIdx.x, j = iter;
+    const int res = blockIdx.x, m = res & 1, t = threadIdx.x, j = iter;
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m] || a.unresolved[res]) return;
     const unsigned int count = a.rep_count[res];
-    bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;
+    bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;      // the same in every thread
     const uint2* rp = a.rep + (size_t)res * kChunkRepCap;
     const uint32_t* sup = ref.lam + (size_t)m * a.s;
     float smax = -1.0f;
     if (!give_up) {
-        for (unsigned int e = lane; e < count; e += 32) {
+        for (unsigned int e = t; e < count; e += kPickThreads) {
             const uint2 v = rp[e];
             bool taken = false;
             for (int q = 0; q < j; ++q) taken |= (sup[q] == v.x);
             if (!taken) smax = fmaxf(smax, __uint_as_float(v.y));
         }
-        for (int o = 16; o > 0; o >>= 1) smax = fmaxf(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+        smax = pick_max(sh, smax);
         if (smax < 0.0f) give_up = true;
     }
     float lo = 0.0f;
@@ -476,9 +509,9 @@ __global__ void __launch_bounds__(32) k_chunk_pick_rep(ChunkArgs a, int iter) {
         if (!((double)lo > a.z_rep * rn / sqrt((double)a.k) * 1.001)) give_up = true;
     }
     if (!give_up) {
-        if (lane == 0) sh.n_c = 0;
-        __syncwarp();
-        for (unsigned int e = lane; e < count; e += 32) {
+        if (t == 0) sh.n_c = 0;
+        __syncthreads();
+        for (unsigned int e = t; e < count; e += kPickThreads) {
             const uint2 v = rp[e];
             if (__uint_as_float(v.y) < lo) continue;
             bool taken = false;
@@ -487,11 +520,11 @@ __global__ void __launch_bounds__(32) k_chunk_pick_rep(ChunkArgs a, int iter) {
             const int slot = atomicAdd(&sh.n_c, 1);
             if (slot < kRescoreCap) sh.cidx[slot] = v.x;
         }
-        __syncwarp();
+        __syncthreads();
         if (sh.n_c > kRescoreCap) give_up = true;
     }
     if (give_up) {
-        if (lane == 0) { a.unresolved[res] = 1; a.flags[0] = 1; }
+        if (t == 0) { a.unresolved[res] = 1; a.flags[0] = 1; }
         return;
     }
     pick_finish(a, ref, sh, res, j, sh.n_c);
@@ -749,7 +782,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
                                 st0->sm_count, stream);
             }
             if (e != cudaSuccess) return e;
-            k_chunk_pick_rep<<<2 * c, 32, 0, stream>>>(a, iter);
+            k_chunk_pick_rep<<<2 * c, kPickThreads, 0, stream>>>(a, iter);
             *launches += 2 + ws->passes;
             gate = ws->flags;
         }
@@ -761,7 +794,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
             case 128: corr_launch<128>(a, iter, smem, stream, gate); break;
             default: corr_launch<256>(a, iter, smem, stream, gate); break;
         }
-        k_chunk_pick<<<2 * c, 32, 0, stream>>>(a, iter, gate, gate ? ws->unresolved : nullptr);
+        k_chunk_pick<<<2 * c, kPickThreads, 0, stream>>>(a, iter, gate, gate ? ws->unresolved : nullptr);
         *launches += 2;
     }
     k_chunk_scatter<<<c, 32, 0, stream>>>(a, weight, (double)st0->alpha, (double)st0->eps, (double)st0->lr);
