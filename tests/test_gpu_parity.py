@@ -539,7 +539,8 @@ def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
     m.close()
 
 
-@pytest.mark.parametrize("m,n,r,c,k,sc", [(512, 256, 8, 4, 28, 4), (1000, 384, 32, 16, 56, 8), (4096, 512, 32, 8, 217, 31)])
+@pytest.mark.parametrize("m,n,r,c,k,sc", [(512, 256, 8, 4, 28, 4), (1000, 384, 32, 16, 56, 8), (4096, 512, 32, 8, 217, 31),
+                                          (300, 128, 8, 1, 320, 8)])          # the last one: a core too large for the batched chunk path
 def test_cesgc_step_matches_its_oracle(sgc, m, n, r, c, k, sc):
     # Section 4.4: SGC (chunked) on B G, update back through B^T; B = first r left-singular vectors of the first gradient
     hp = inputs.ADAM
