@@ -8,7 +8,8 @@
 //                     64th of the fp32 rate on this part and made this kernel 1.1 ms), and rounded to fp32 once at the
 //                     end.  The top-s selection that follows decides on those values; a reference that forms B G in fp64
 //                     gets the same fp32 numbers but for a few elements in ten thousand (entries much smaller than
-//                     their terms), which differ by one ulp.  Slabs of B and G are staged in shared memory.
+//                     their terms), which differ by one ulp.  Slabs of B and G are staged in shared memory; the next ones travel
+//                     through registers while the current ones are worked on.
 //   k_cesgc_back      W += B^T U for the r x n matrix U that the SGC core left (U = -eta N has at most s non-zeros):
 //                     block = one column of U; columns without a non-zero cost one read of r values.
 #include "sgc_internal.cuh"
@@ -21,6 +22,8 @@ constexpr int kProjRows = 4;             // rows of B per thread
 constexpr int kProjChunk = 64;           // rows of G per staged slab of B
 constexpr int kCesgcMaxR = 64;
 
+constexpr int kProjStage = 8;            // floats of each slab that one thread moves (at 256 threads: 64 x 32 floats)
+
 __global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows))
 k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float* __restrict__ P, int r, int m, int n) {
     __shared__ float bs[kCesgcMaxR][kProjChunk];                      // B[:, row0 .. row0 + 64)
@@ -29,21 +32,39 @@ k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float*
     const int jl = threadIdx.x % kProjCols, ig = threadIdx.x / kProjCols;
     const int j = blockIdx.x * kProjCols + jl;
     const bool work = ig < groups && j < n;
+    const int nb = r * kProjChunk, ng = kProjChunk * kProjCols;       // slab sizes
+    const int per_b = (nb + blockDim.x - 1) / blockDim.x, per_g = (ng + blockDim.x - 1) / blockDim.x;   // <= kProjStage
+    float pb[kProjStage], pg[kProjStage];                             // the next slabs, on their way through registers
+    auto fetch = [&](int row0) {
+#pragma unroll
+        for (int u = 0; u < kProjStage; ++u) {
+            const int eb = threadIdx.x + u * blockDim.x, eg = eb;
+            pb[u] = 0.0f; pg[u] = 0.0f;
+            if (u < per_b && eb < nb) {
+                const int i = eb / kProjChunk, q = eb % kProjChunk;
+                if (row0 + q < m) pb[u] = B[(size_t)i * m + row0 + q];
+            }
+            if (u < per_g && eg < ng) {
+                const int q = eg / kProjCols, c = eg % kProjCols;
+                const int col = blockIdx.x * kProjCols + c;
+                if (row0 + q < m && col < n) pg[u] = G[(size_t)(row0 + q) * n + col];
+            }
+        }
+    };
     float hi[kProjRows], lo[kProjRows];
 #pragma unroll
     for (int u = 0; u < kProjRows; ++u) hi[u] = lo[u] = 0.0f;
+    fetch(0);
     for (int row0 = 0; row0 < m; row0 += kProjChunk) {
-        __syncthreads();
-        for (int e = threadIdx.x; e < r * kProjChunk; e += blockDim.x) {
-            const int i = e / kProjChunk, q = e % kProjChunk;
-            bs[i][q] = row0 + q < m ? B[(size_t)i * m + row0 + q] : 0.0f;
-        }
-        for (int e = threadIdx.x; e < kProjChunk * kProjCols; e += blockDim.x) {       // many independent loads in flight
-            const int q = e / kProjCols, c = e % kProjCols;
-            const int col = blockIdx.x * kProjCols + c;
-            gs[q][c] = (row0 + q < m && col < n) ? G[(size_t)(row0 + q) * n + col] : 0.0f;
+        __syncthreads();                                              // the previous slabs have been used up
+#pragma unroll
+        for (int u = 0; u < kProjStage; ++u) {
+            const int e = threadIdx.x + u * blockDim.x;
+            if (u < per_b && e < nb) bs[e / kProjChunk][e % kProjChunk] = pb[u];
+            if (u < per_g && e < ng) gs[e / kProjCols][e % kProjCols] = pg[u];
         }
         __syncthreads();
+        if (row0 + kProjChunk < m) fetch(row0 + kProjChunk);          // in flight while this slab is worked on
         if (!work) continue;
         const int rows = m - row0 < kProjChunk ? m - row0 : kProjChunk;
         for (int q = 0; q < rows; ++q) {
@@ -109,7 +130,8 @@ bool cesgc_shape_ok(int r, int m, int n) { return r >= 1 && r <= kCesgcMaxR && m
 
 cudaError_t launch_cesgc_project(const float* B, const float* G, float* P, int r, int m, int n, cudaStream_t stream) {
     const int groups = (r + kProjRows - 1) / kProjRows;
-    k_cesgc_project<<<(n + kProjCols - 1) / kProjCols, kProjCols * groups, 0, stream>>>(B, G, P, r, m, n);
+    const int threads = kProjCols * groups < 256 ? 256 : kProjCols * groups;      // at least 256: the slabs are staged 8 floats per thread
+    k_cesgc_project<<<(n + kProjCols - 1) / kProjCols, threads, 0, stream>>>(B, G, P, r, m, n);
     return cudaGetLastError();
 }
 
