@@ -286,6 +286,14 @@ class Cesgc:
             raise TypeError("B must be a contiguous float32 CUDA tensor of shape (r, m)")
         self.B = B
 
+    def refresh_projection(self, grad):
+        """B <- the first r left-singular vectors of grad (m x n), transposed: what the paper renews every fixed number
+        of iterations.  The SVD is torch's (a library routine outside the per-step path)."""
+        import torch
+        U, _, _ = torch.linalg.svd(grad.reshape(self.m, self.n).float(), full_matrices=False)
+        Q, _ = torch.linalg.qr(U[:, :self.r].double())          # fp32 singular vectors are orthonormal to ~1e-4 only
+        self.set_projection(Q.t().float().contiguous())
+
     def step(self, grad, weight, stream=None):
         if self.B is None:
             raise ValueError("set_projection() first")
