@@ -64,7 +64,7 @@ size_t layout(sgc_state* st, unsigned char* base) {
         st->wide_tau = carve<float>(base, off, sgc::kPassMaxN / 8);
         st->wide_list = carve<uint32_t>(base, off, 2 * (size_t)sgc::kWideCap);
         st->wide_count = carve<unsigned int>(base, off, 2);
-        st->wide_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
+        st->wide_bits = carve<unsigned int>(base, off, 2 * (((size_t)st->d + 31) / 32));
     }
     return off;
 }

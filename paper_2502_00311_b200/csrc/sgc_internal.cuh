@@ -278,7 +278,7 @@ struct sgc_state {
     float* wide_tau;            // [kPassMaxN / 8] thresholds of the wide lists, one per 8th screened residual
     uint32_t* wide_list;        // [2][kWideCap]
     unsigned int* wide_count;   // [2]
-    unsigned int* wide_bits;    // bitmap over [0, d): the column is in one of the wide lists
+    unsigned int* wide_bits;    // [2] bitmaps over [0, d): the column is in the stream's wide list
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };
@@ -334,7 +334,7 @@ struct PassWide {
     const float* tau;            // [n / 8] thresholds of the wide lists (scaled units of rows 0, 8, 16, ...)
     uint32_t* list;              // [2][cap]
     unsigned int* count;         // [2]
-    unsigned int* bits;          // bitmap over [0, d): a column enters the lists once
+    unsigned int* bits;          // [2] bitmaps over [0, d), one per stream: a column enters a list once
     int cap, half_n;
     const SpecCtl* ctl;
     bool list_pass;              // true: screen the lists' columns; false: full pass that feeds the lists

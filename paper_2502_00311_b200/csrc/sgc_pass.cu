@@ -56,7 +56,7 @@ struct PassArgs {
     const float* big_tau;        // [n / 8] or nullptr
     uint32_t* big_list;          // [2][big_cap]
     unsigned int* big_count;     // [2]
-    unsigned int* big_bits;      // bitmap over [0, d)
+    unsigned int* big_bits;      // [2] bitmaps over [0, d), one per stream
     int big_cap, big_half;
     const SpecCtl* list_ctl;     // list pass: gate and list lengths come from the control block
     const int* sel; int sel_value;    // optional: the kernel returns at once unless *sel == sel_value (which of two widths runs)
@@ -183,7 +183,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         const volatile SpecCtl* lc = a.list_ctl;
         if (!lc->round_active || lc->fallback || lc->mini_done || lc->n_cand <= kSmallList) return;
         list_n0 = min(a.big_count[0], (unsigned int)a.big_cap);
-        list_n = list_n0 + min(a.big_count[1], (unsigned int)a.big_cap);
+        // the half-width pass serves the first stream alone: its own list is all it needs
+        list_n = list_n0 + ((a.sel != nullptr && a.sel_value == 1) ? 0u : min(a.big_count[1], (unsigned int)a.big_cap));
         if (list_n == 0) return;
         num_super = (list_n + kSuperCols - 1) / kSuperCols;
         if (blockIdx.x >= num_super) return;
@@ -316,8 +317,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                         const bool w8 = fabsf(__uint_as_float(v[8])) * inv >= a.big_tau[(c0 >> 3) + 1];
                         if (w0 || w8) {
                             const unsigned int bit = 1u << ((unsigned int)col & 31u);
-                            if (!(atomicOr(&a.big_bits[col >> 5], bit) & bit)) {
-                                const int m = c0 >= a.big_half ? 1 : 0;
+                            const int m = c0 >= a.big_half ? 1 : 0;
+                            if (!(atomicOr(&a.big_bits[(size_t)m * ((a.d + 31) >> 5) + (col >> 5)], bit) & bit)) {
                                 const unsigned int slot = atomicAdd(&a.big_count[m], 1u);
                                 if (slot < (unsigned int)a.big_cap) a.big_list[(size_t)m * a.big_cap + slot] = (uint32_t)col;
                             }

@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
     // cover the whole path of this step, which is where the next step's path runs, too)
     if (mode == 0 && !a.mini && a.wide_count != nullptr && ctl->rounds == 0) {
         if (mb == 0 && threadIdx.x == 0) a.wide_count[0] = a.wide_count[1] = 0u;
-        const size_t words = ((size_t)a.d + 31) / 32;
+        const size_t words = 2 * (((size_t)a.d + 31) / 32);          // both streams' bitmaps
         for (size_t w = (size_t)blockIdx.x * kOmpThreads + threadIdx.x; w < words; w += (size_t)gridDim.x * kOmpThreads)
             a.wide_bits[w] = 0u;
     }
