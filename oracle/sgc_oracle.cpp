@@ -23,6 +23,13 @@
 //   * Ties in |g| and in the OMP argmax go to the lower index; selected columns are not re-selected.
 //   * Exactly s OMP iterations unless the new column is numerically dependent on the support.
 //   * Eq. (8) is applied on the intersection of the two supports where x^V > 0; elsewhere N = 0.
+//   Parity unpinned by the paper (readings of ours, nothing printed fixes them): the stop on a numerically dependent
+//   column, the treatment of Eq. (8) where the two supports differ or x^V <= 0, and the opt-in variant of
+//   orc_set_recovery (one shared support, early stop on the residual).
+//
+// Beyond the step itself: orc_reproject (SGCA, Appendix C, Algorithm 4 lines 9-12), orc_omp_tol / orc_least_squares /
+// orc_set_recovery (the variant built on the remark after Eq. (8)); the chunked (MESGC) and projected (CESGC) forms of
+// Section 4.4 are compositions of these states written out in oracle/binding.py (cesgc_step) and in the tests.
 //
 // Arithmetic: inputs and stored state are fp32; every sum is accumulated in fp64.
 // Pins: see tests/test_oracle_*.py (dense-matrix definitions, brute-force supports, closed-form
