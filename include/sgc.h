@@ -177,7 +177,9 @@ SGC_API int sgc_reproject(sgc_state* st, uint64_t new_seed, void* stream);
  * the speculative one runs OMP on a short candidate list and then proves, with one tensor-core pass over all
  * d columns against the residuals of all iterations at once, that no other column would have been picked; a
  * refuted pick is replaced by the true argmax and the round repeats from there.
- * SGC_ERR_DIM when SGC_MODE_SPECULATIVE is requested and k is not a multiple of 64. */
+ * SGC_ERR_DIM when SGC_MODE_SPECULATIVE is requested and k is not a multiple of 64.  States with d < 65536 never
+ * speculate on their own accord and are created without the buffers of that strategy (some 50 MB plus 6.5 bytes per
+ * column); asking for SGC_MODE_SPECULATIVE allocates them here (one cudaMalloc, synchronises; a CUDA error code if it fails). */
 SGC_API int sgc_set_mode(sgc_state* st, int32_t mode);
 
 /* Opt-in variant of the recovery, built on the remark after Eq. (8) that OMP_A(M_t) and OMP_A(V_t) have their

@@ -42,7 +42,16 @@ size_t layout(sgc_state* st, unsigned char* base) {
     st->upd_val = carve<double>(base, off, s);
     st->cnt = carve<sgc::Counters>(base, off, 1);
     st->ctl = carve<sgc::SpecCtl>(base, off, 1);
-    if (st->spec_ok) {
+    return off;
+}
+
+// lays out (base == nullptr: only measures) the buffers of the speculative recovery: a second allocation, made at
+// creation for states that will use it on their own accord (d >= 65536) and at sgc_set_mode(SGC_MODE_SPECULATIVE)
+// for the others, so that thousands of small chunk states do not carry 50 MB each that they never touch
+size_t layout_spec(sgc_state* st, unsigned char* base) {
+    size_t off = 0;
+    const size_t k = (size_t)st->k, s = (size_t)st->s;
+    {
         const size_t n = (size_t)sgc::kPassMaxN;          // room for a whole batch of same-A states (sgc_step_group)
         st->rt = carve<uint16_t>(base, off, n * k);
         st->tau = carve<float>(base, off, n);
@@ -70,6 +79,22 @@ size_t layout(sgc_state* st, unsigned char* base) {
 }
 
 bool finite_f(float v) { return isfinite(v); }
+
+cudaError_t ensure_spec(sgc_state* st) {
+    if (!st->spec_ok || st->spec_ready) return cudaSuccess;
+    {
+        sgc_state probe = *st;                                       // measuring must not leave pointers behind
+        st->spec_bytes = layout_spec(&probe, nullptr);
+    }
+    cudaError_t e = cudaMalloc(&st->spec_base, st->spec_bytes);
+    if (e != cudaSuccess) { st->spec_base = nullptr; return e; }
+    layout_spec(st, static_cast<unsigned char*>(st->spec_base));
+    e = cudaMemset(st->spec_base, 0, st->spec_bytes);             // empty candidate list, bitmaps, wide lists
+    if (e == cudaSuccess) e = sgc::finish_recover_setup(st);      // tensor maps of R^T, column norms (synchronises)
+    if (e != cudaSuccess) { cudaFree(st->spec_base); st->spec_base = nullptr; return e; }
+    st->spec_ready = true;
+    return cudaSuccess;
+}
 
 }  // namespace
 
@@ -104,13 +129,14 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
         layout(st, static_cast<unsigned char*>(st->base));
         e = cudaMemset(st->base, 0, st->bytes);        // M_0 = V_0 = 0, counters, histogram, empty candidate list
     }
-    if (e == cudaSuccess) e = sgc::finish_recover_setup(st);
+    if (e == cudaSuccess && st->d >= ((int64_t)1 << 16)) e = ensure_spec(st);      // SGC_MODE_AUTO speculates from this size on
     if (e == cudaSuccess) {
         e = cudaHostAlloc(reinterpret_cast<void**>(&st->h_rounds), sizeof(int), cudaHostAllocMapped);
         if (e == cudaSuccess) { st->h_rounds[0] = 0; e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&st->d_rounds), st->h_rounds, 0); }
     }
     if (e != cudaSuccess) {
         if (st->base) cudaFree(st->base);
+        if (st->spec_base) cudaFree(st->spec_base);
         if (st->h_rounds) cudaFreeHost(st->h_rounds);
         delete st->ev_pool; delete st->ev_phase;
         delete st;
@@ -221,6 +247,7 @@ SGC_API int sgc_destroy(sgc_state* st) {
     cudaError_t e = cudaSuccess;
     if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
     sgc::free_chunk_ws(st);
+    if (st->spec_base) cudaFree(st->spec_base);
     cudaError_t e2 = cudaFree(st->base);
     if (st->h_rounds) cudaFreeHost(st->h_rounds);
     for (cudaEvent_t ev : *st->ev_pool) cudaEventDestroy(ev);
@@ -242,7 +269,7 @@ SGC_API int sgc_reproject(sgc_state* st, uint64_t new_seed, void* stream) {
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     cudaError_t e = sgc::launch_reproject(st, new_seed, cs);
     st->seed = new_seed;
-    if (e == cudaSuccess && st->spec_ok) e = sgc::launch_inv_norms(new_seed, (uint64_t)st->d, st->k, st->inv_norm, cs);
+    if (e == cudaSuccess && st->spec_ready) e = sgc::launch_inv_norms(new_seed, (uint64_t)st->d, st->k, st->inv_norm, cs);
     st->last_stream = cs; st->has_stream = true;
     return (int)e;
 }
@@ -251,6 +278,10 @@ SGC_API int sgc_set_mode(sgc_state* st, int32_t mode) {
     if (!st) return SGC_ERR_NULL;
     if (mode < SGC_MODE_AUTO || mode > SGC_MODE_SPECULATIVE) return SGC_ERR_WHAT;
     if (mode == SGC_MODE_SPECULATIVE && !st->spec_ok) return SGC_ERR_DIM;
+    if (mode == SGC_MODE_SPECULATIVE) {
+        const cudaError_t e = ensure_spec(st);                       // small states get their speculative buffers here
+        if (e != cudaSuccess) return (int)e;
+    }
     st->mode = mode;
     return SGC_OK;
 }

@@ -231,6 +231,8 @@ struct sgc_state {
     int shared_support;         // 1: OMP(M^) alone selects, V^ is fitted on its support (sgc_set_recovery)
     double residual_tol;        // > 0: recoveries are cut at the first pick that leaves ||r|| <= residual_tol ||y||
     bool spec_ok;               // speculative recovery usable for this (d, k)
+    bool spec_ready;            // its buffers exist (second allocation: at creation for d >= 65536, else at sgc_set_mode)
+    void* spec_base; size_t spec_bytes;
     int pass_n;                 // residuals per screening pass (multiple of 32, <= 256); pass_n / 2 per residual stream
     double z_harvest, z_floor;  // thresholds of the screening pass in units of ||r|| / sqrt(k)
     double z_wide;              // threshold of the wide lists, same units

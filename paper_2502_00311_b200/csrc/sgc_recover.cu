@@ -1644,7 +1644,8 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
     sgc_state* st0 = sts[0];
     bool speculate = true;
     for (int i = 0; i < n; ++i)
-        speculate = speculate && sts[i]->spec_ok && (sts[i]->mode == 2 || (sts[i]->mode == 0 && sts[i]->d >= (1ll << 16)));
+        speculate = speculate && sts[i]->spec_ok && sts[i]->spec_ready &&
+                    (sts[i]->mode == 2 || (sts[i]->mode == 0 && sts[i]->d >= (1ll << 16)));
     const int per_batch = speculate ? kPassMaxN / st0->pass_n : 1;
     std::vector<OmpArgs> args((size_t)n);
     cudaError_t e = cudaSuccess;

@@ -529,6 +529,26 @@ def test_mesgc_batched_path_on_a_side_stream(sgc):
     assert np.array_equal(outs[0][2], outs[1][2])
 
 
+def test_small_states_are_created_without_speculative_buffers(sgc):
+    import torch
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    states = [sgc.Sgc(4096, 64, 8, 1, 1e-3, 0.9, 0.999, 1e-8) for _ in range(64)]      # k a multiple of 64: could speculate
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < 64 * (4 << 20), (free0 - free1) / 64                     # a few MB each at most, not 50
+    states[0].set_mode(sgc.MODE_SPECULATIVE)                                        # this one gets them now
+    free2, _ = torch.cuda.mem_get_info()
+    assert free1 - free2 > (30 << 20)
+    g = cuda((np.random.default_rng(0).standard_normal(4096) * 0.1).astype(np.float32))
+    wa, wb = cuda(np.zeros(4096, dtype=np.float32)), cuda(np.zeros(4096, dtype=np.float32))
+    states[0].step(g, wa)
+    states[1].step(g, wb)
+    assert states[0].get("fallback") == 0 and states[1].get("fallback") == 1
+    assert np.array_equal(states[0].get("lamM"), states[1].get("lamM")) and np.array_equal(wa.cpu().numpy(), wb.cpu().numpy())
+    for st in states:
+        st.close()
+
+
 def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
     import torch
     m = sgc.Mesgc(4 * 4096, 4, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
