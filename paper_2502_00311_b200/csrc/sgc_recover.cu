@@ -1164,7 +1164,7 @@ __device__ void harvest(const ResolveArgs& ra, BookSmem& sh, const uint2* rep, u
 // Full mode (reports of a pass over all d columns): confirms the speculated picks in order; the first refuted pick of a
 // stream gets its true winner, which becomes final.  Mini mode (reports of a list pass over the wide lists): the same
 // walk, but what it establishes is tentative -- tv / tforced tell the next speculation where to resume, while v, forced,
-// the round count and everything a finished recovery records are left alone; the next full pass judges all of it.
+// the round count and everything a finished recovery records are left alone; the next full pass decides on all of it.
 __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
     const OmpArgs& a = ra.o;
     __shared__ BookSmem sh;
