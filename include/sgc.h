@@ -5,11 +5,11 @@
  * index of the measurement matrix A in R^{k x d}):
  *
  *   a1  G~ = Sparsify_s(G)                      keep the s largest |g_i|                (Section 3.2)
- *   a2  p = A G~ ,  q = A G~^2                  Eq. (4) and the equation after it; Algorithm 2 line 1
+ *   a2  p = A G~ ,  q = A G~^2                  Eq. (4) and the equation after it; Algorithm 2
  *   a3  M <- b1 M + (1-b1) p ; V <- b2 V + (1-b2) q ; M^ = M/(1-b1^t) ; V^ = V/(1-b2^t)
- *                                                Algorithm 2 lines 2-5
+ *                                                Algorithm 2
  *   a4  x^M = OMP_A(M^) , x^V = OMP_A(V^)       Eq. (7); Appendix B Algorithm 3
- *   a5  N = alpha x^M / (sqrt(x^V) + eps) ; W <- W - lr N          Eq. (8), Eq. (3); Algorithm 2 line 6
+ *   a5  N = alpha x^M / (sqrt(x^V) + eps) ; W <- W - lr N          Eq. (8), Eq. (3); Algorithm 2
  *
  * A is never stored.  A[j][i] = sigma_k * Z(seed, j, i), sigma_k = fl32(1/sqrt(k)), where Z is a
  * counter-based, approximately standard-normal function of (seed, row, column) evaluated on the fly
@@ -166,7 +166,7 @@ SGC_API int sgc_destroy(sgc_state* st);
 /* alpha of Eq. (8) ("a scaling factor"); must be finite. */
 SGC_API int sgc_set_alpha(sgc_state* st, float alpha);
 
-/* SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): replaces the measurement matrix by the one that new_seed
+/* SGCA re-projection (Appendix C, Algorithm 4): replaces the measurement matrix by the one that new_seed
  * names and re-aligns the optimizer state with it, M <- A' OMP_A(M), V <- A' OMP_A(V).  Call it after the sgc_step of
  * an iteration t with t mod T = 0: the recoveries of that step are reused, since OMP_A(M) = (1 - beta1^t) OMP_A(M^)
  * (OMP is scale-equivariant; the paper itself notes that the results of the first call can be kept).  From the next

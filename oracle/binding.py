@@ -244,7 +244,7 @@ class Oracle:
         lib().orc_set_recovery(self._h, 1 if shared_support else 0, float(residual_tol))
 
     def reproject(self, new_seed):
-        """SGCA (Algorithm 4, lines 9-12): M <- A' OMP_A(M), V <- A' OMP_A(V), A <- A' with A' named by new_seed."""
+        """SGCA (Algorithm 4): M <- A' OMP_A(M), V <- A' OMP_A(V), A <- A' with A' named by new_seed."""
         lib().orc_reproject(self._h, C.c_uint64(new_seed))
 
     def get(self, name):

@@ -6,17 +6,17 @@
 //
 // What it computes (paper notation):
 //   Sparsify_s            Section 3.2, text before Eq. (4): keep the s largest-magnitude entries
-//   p = A G~, q = A G~^2  Eq. (4) and the unnumbered equation after it; Algorithm 2 line 1
-//   k-space Adam          Algorithm 2 lines 2-5 (Algorithm 1 lines 1-4 in k dimensions)
+//   p = A G~, q = A G~^2  Eq. (4) and the unnumbered equation after it; Algorithm 2
+//   k-space Adam          Algorithm 2 (Algorithm 1 in k dimensions)
 //   OMP_A(y)              Eq. (7); Appendix B Algorithm 3.  Algorithm 3 is an algebraic rewrite
 //                         (inverse Cholesky) of textbook orthogonal matching pursuit; the oracle
 //                         is the textbook form: correlate, normalised argmax, dense least
 //                         squares on the support (Householder QR), residual.
-//   N = a*x^M/(sqrt(x^V)+eps), W <- W - eta*N      Eq. (8), Eq. (3); Algorithm 2 line 6
+//   N = a*x^M/(sqrt(x^V)+eps), W <- W - eta*N      Eq. (8), Eq. (3); Algorithm 2
 //
 // Readings of points the paper leaves open (all listed in the design notes of the repository):
-//   * V uses beta2 (Algorithm 2 line 3; the displayed Eq. (6) prints beta1, a typo).
-//   * Bias correction (Algorithm 2 lines 4-5) produces temporaries; M and V are stored uncorrected.
+//   * V uses beta2 (Algorithm 2; the displayed Eq. (6) prints beta1, a typo).
+//   * Bias correction (Algorithm 2) produces temporaries; M and V are stored uncorrected.
 //   * A has i.i.d. entries of standard deviation 1/sqrt(k) (Section 3.3).  Here
 //     A[j][i] = sigma_k * Z(seed, j, i) with sigma_k = fl32(1/sqrt(k)) and Z a counter-based
 //     approximately standard-normal value (a binary16 number) defined below; A is never stored.
@@ -27,7 +27,7 @@
 //   column, the treatment of Eq. (8) where the two supports differ or x^V <= 0, and the opt-in variant of
 //   orc_set_recovery (one shared support, early stop on the residual).
 //
-// Beyond the step itself: orc_reproject (SGCA, Appendix C, Algorithm 4 lines 9-12), orc_omp_tol / orc_least_squares /
+// Beyond the step itself: orc_reproject (SGCA, Appendix C, Algorithm 4), orc_omp_tol / orc_least_squares /
 // orc_set_recovery (the variant built on the remark after Eq. (8)); the chunked (MESGC) and projected (CESGC) forms of
 // Section 4.4 are compositions of these states written out in oracle/binding.py (cesgc_step) and in the tests.
 //
@@ -250,7 +250,7 @@ void orc_project(uint64_t seed, int32_t k, const uint32_t* idx, const float* val
     }
 }
 
-// ---- a3: k-space Adam (Algorithm 2 lines 2-5) -------------------------------------------------
+// ---- a3: k-space Adam (Algorithm 2) -------------------------------------------------
 // M,V: stored fp32 state, updated in place (uncorrected).  t is the 1-based step count of THIS step.
 // Mhat,Vhat: bias-corrected temporaries in fp64, computed from the stored (rounded) state.
 void orc_adam(float* M, float* V, const double* p, const double* q, int32_t k,
@@ -477,7 +477,7 @@ void orc_step(orc_state* st, const float* grad, float* weight) {
     orc_step_recover(st, weight);
 }
 
-// SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): with a new matrix A' (here: a new seed),
+// SGCA re-projection (Appendix C, Algorithm 4): with a new matrix A' (here: a new seed),
 //   M <- A' OMP_A(M),  V <- A' OMP_A(V),  A <- A'.
 // Reading: M and V are the stored moments (bias correction yields temporaries, as everywhere in this oracle); both
 // recoveries are run afresh on them with the old A, s iterations each, and the s-sparse results are projected with A'.

@@ -1,5 +1,5 @@
-// a2 + a3 fused: p = A G~, q = A G~^2 (Eq. 4 and the equation after it; Algorithm 2 line 1) followed by the
-// k-space Adam moments with bias correction (Algorithm 2 lines 2-5).  One thread per row of A; the s selected
+// a2 + a3 fused: p = A G~, q = A G~^2 (Eq. 4 and the equation after it; Algorithm 2) followed by the
+// k-space Adam moments with bias correction (Algorithm 2).  One thread per row of A; the s selected
 // columns of A are regenerated on the fly (k*s entries), sums are carried in fp64 in ascending column order.
 #include "sgc_internal.cuh"
 
@@ -48,7 +48,7 @@ k_project_adam(uint32_t seed_lo, uint32_t seed_hi, int k, int s, const uint32_t*
     r32[row] = make_float2((float)mh, (float)vh);
 }
 
-// SGCA re-projection (Appendix C, Algorithm 4, lines 9-12): M <- A' OMP_A(M), V <- A' OMP_A(V) for a new matrix A'.
+// SGCA re-projection (Appendix C, Algorithm 4): M <- A' OMP_A(M), V <- A' OMP_A(V) for a new matrix A'.
 // OMP is scale-equivariant, OMP_A(M) = (1 - beta1^t) OMP_A(M^), so the recoveries of the step that has just run are
 // reused (the paper notes that the results of the first call can be stored): row j of the new state is
 // c * sum_l A'[j][lambda_l] x_l over the recovered support, summed in fp64 in the order of selection.

@@ -1,5 +1,5 @@
 // a4 + a5: x^M = OMP_A(M^), x^V = OMP_A(V^) (Eq. 7; Appendix B Algorithm 3), then
-// N = alpha x^M / (sqrt(x^V) + eps) and W <- W - lr N (Eq. 8, Eq. 3; Algorithm 2 line 6).
+// N = alpha x^M / (sqrt(x^V) + eps) and W <- W - lr N (Eq. 8, Eq. 3; Algorithm 2).
 //
 // Algorithm 3 needs, for every pick, the argmax of |<A_i, r>| / ||A_i|| over all d columns ("Projection" and
 // "Select"), and A is regenerated rather than stored, so one such argmax costs k*d generated entries.  Two ways

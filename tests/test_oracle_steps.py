@@ -64,7 +64,7 @@ def test_projection_is_linear():
 
 # ---- a3 Adam in k-space ----------------------------------------------------------------------------
 def test_adam_constant_input_closed_form():
-    # Algorithm 2 lines 2-5 with M_0 = V_0 = 0 and constant p, q:  M_t = (1-b1^t) p,  Mhat_t = p.
+    # Algorithm 2 with M_0 = V_0 = 0 and constant p, q:  M_t = (1-b1^t) p,  Mhat_t = p.
     k, b1, b2 = 50, np.float32(0.9), np.float32(0.999)
     rng = np.random.default_rng(0)
     p = rng.standard_normal(k)
@@ -128,7 +128,7 @@ def test_combine_scatter_definition_and_guards():
     assert np.array_equal(W, want.astype(np.float32))
 
 
-# ---- SGCA re-projection (Appendix C, Algorithm 4, lines 9-12) ------------------------------------------------
+# ---- SGCA re-projection (Appendix C, Algorithm 4) ------------------------------------------------
 def test_reprojection_moves_an_exactly_sparse_state_to_the_new_matrix():
     # constant sparse gradient: M_t = (1 - b1^t) A g and V_t = (1 - b2^t) A g^2 exactly (closed form of the EMA), so
     # OMP recovers (1 - b^t) g and the re-projected states must be (1 - b^t) A' g, A' materialised with numpy
