@@ -9,10 +9,16 @@
 //                     end.  The top-s selection that follows decides on those values; a reference that forms B G in fp64
 //                     gets the same fp32 numbers but for a few elements in ten thousand (entries much smaller than
 //                     their terms), which differ by one ulp.  Slabs of B and G are staged in shared memory; the next ones travel
-//                     through registers while the current ones are worked on.
+//                     through registers while the current ones are worked on.  The rows of G are split over the CTAs of
+//                     a thread-block cluster (n / 32 column blocks alone would not fill the SMs); their partial sums
+//                     meet in the first CTA through distributed shared memory, added in rank order.
 //   k_cesgc_back      W += B^T U for the r x n matrix U that the SGC core left (U = -eta N has at most s non-zeros):
 //                     block = one column of U; columns without a non-zero cost one read of r values.
 #include "sgc_internal.cuh"
+
+#include <cooperative_groups.h>
+
+namespace cg = cooperative_groups;
 
 namespace sgc {
 namespace {
@@ -23,15 +29,23 @@ constexpr int kProjChunk = 64;           // rows of G per staged slab of B
 constexpr int kCesgcMaxR = 64;
 
 constexpr int kProjStage = 8;            // floats of each slab that one thread moves (at 256 threads: 64 x 32 floats)
+constexpr int kProjMaxSplit = 8;         // CTAs of a cluster (the portable limit), each with a range of G's rows
+constexpr int kProjResident = 4 * 148;   // CTAs of this kernel that the SMs hold at once (58 registers, 256 threads)
 
 __global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows))
 k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float* __restrict__ P, int r, int m, int n) {
     __shared__ float bs[kCesgcMaxR][kProjChunk];                      // B[:, row0 .. row0 + 64)
     __shared__ float gs[kProjChunk][kProjCols];                       // G[row0 .. row0 + 64, the block's columns]
+    cg::cluster_group cluster = cg::this_cluster();
     const int groups = (r + kProjRows - 1) / kProjRows;
     const int jl = threadIdx.x % kProjCols, ig = threadIdx.x / kProjCols;
     const int j = blockIdx.x * kProjCols + jl;
     const bool work = ig < groups && j < n;
+    // this CTA's rows of G: whole slabs, the same number for every CTA of the cluster (the last ranges may be empty)
+    const int slabs = (m + kProjChunk - 1) / kProjChunk;
+    const int part_rows = (slabs + (int)gridDim.y - 1) / (int)gridDim.y * kProjChunk;
+    const int m_begin = (int)blockIdx.y * part_rows;
+    const int m_end = m_begin + part_rows < m ? m_begin + part_rows : m;
     const int nb = r * kProjChunk, ng = kProjChunk * kProjCols;       // slab sizes
     const int per_b = (nb + blockDim.x - 1) / blockDim.x, per_g = (ng + blockDim.x - 1) / blockDim.x;   // <= kProjStage
     float pb[kProjStage], pg[kProjStage];                             // the next slabs, on their way through registers
@@ -42,20 +56,20 @@ k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float*
             pb[u] = 0.0f; pg[u] = 0.0f;
             if (u < per_b && eb < nb) {
                 const int i = eb / kProjChunk, q = eb % kProjChunk;
-                if (row0 + q < m) pb[u] = B[(size_t)i * m + row0 + q];
+                if (row0 + q < m_end) pb[u] = B[(size_t)i * m + row0 + q];
             }
             if (u < per_g && eg < ng) {
                 const int q = eg / kProjCols, c = eg % kProjCols;
                 const int col = blockIdx.x * kProjCols + c;
-                if (row0 + q < m && col < n) pg[u] = G[(size_t)(row0 + q) * n + col];
+                if (row0 + q < m_end && col < n) pg[u] = G[(size_t)(row0 + q) * n + col];
             }
         }
     };
     float hi[kProjRows], lo[kProjRows];
 #pragma unroll
     for (int u = 0; u < kProjRows; ++u) hi[u] = lo[u] = 0.0f;
-    fetch(0);
-    for (int row0 = 0; row0 < m; row0 += kProjChunk) {
+    fetch(m_begin);
+    for (int row0 = m_begin; row0 < m_end; row0 += kProjChunk) {
         __syncthreads();                                              // the previous slabs have been used up
 #pragma unroll
         for (int u = 0; u < kProjStage; ++u) {
@@ -64,9 +78,9 @@ k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float*
             if (u < per_g && e < ng) gs[e / kProjCols][e % kProjCols] = pg[u];
         }
         __syncthreads();
-        if (row0 + kProjChunk < m) fetch(row0 + kProjChunk);          // in flight while this slab is worked on
+        if (row0 + kProjChunk < m_end) fetch(row0 + kProjChunk);          // in flight while this slab is worked on
         if (!work) continue;
-        const int rows = m - row0 < kProjChunk ? m - row0 : kProjChunk;
+        const int rows = m_end - row0 < kProjChunk ? m_end - row0 : kProjChunk;
         for (int q = 0; q < rows; ++q) {
             const float g = gs[q][jl];
 #pragma unroll
@@ -82,13 +96,36 @@ k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float*
             }
         }
     }
+    // the partial sums of the cluster's CTAs, left in each one's shared memory (the slab of B is done with)
+    __syncthreads();
+    float* part_hi = &bs[0][0];
+    float* part_lo = part_hi + kCesgcMaxR * kProjCols;
+    static_assert(2 * kProjCols <= kProjChunk, "two 64 x 32 arrays in the slab of B");
     if (work) {
 #pragma unroll
         for (int u = 0; u < kProjRows; ++u) {
-            const int i = ig * kProjRows + u;
-            if (i < r) P[(size_t)i * n + j] = (float)((double)hi[u] + (double)lo[u]);
+            part_hi[(ig * kProjRows + u) * kProjCols + jl] = hi[u];
+            part_lo[(ig * kProjRows + u) * kProjCols + jl] = lo[u];
         }
     }
+    cluster.sync();
+    if (cluster.block_rank() == 0 && work) {
+        const unsigned split = cluster.num_blocks();
+#pragma unroll
+        for (int u = 0; u < kProjRows; ++u) {
+            const int i = ig * kProjRows + u;
+            if (i >= r) continue;
+            double acc = 0.0;
+            for (unsigned y = 0; y < split; ++y) {                    // rank order: the result does not depend on the schedule
+                const float* h = cluster.map_shared_rank(part_hi, y);
+                const float* l = cluster.map_shared_rank(part_lo, y);
+                acc += (double)h[i * kProjCols + jl];
+                acc += (double)l[i * kProjCols + jl];
+            }
+            P[(size_t)i * n + j] = (float)acc;
+        }
+    }
+    cluster.sync();                                                   // nobody leaves while its sums may still be read
 }
 
 __global__ void __launch_bounds__(256)
@@ -131,8 +168,21 @@ bool cesgc_shape_ok(int r, int m, int n) { return r >= 1 && r <= kCesgcMaxR && m
 cudaError_t launch_cesgc_project(const float* B, const float* G, float* P, int r, int m, int n, cudaStream_t stream) {
     const int groups = (r + kProjRows - 1) / kProjRows;
     const int threads = kProjCols * groups < 256 ? 256 : kProjCols * groups;      // at least 256: the slabs are staged 8 floats per thread
-    k_cesgc_project<<<(n + kProjCols - 1) / kProjCols, threads, 0, stream>>>(B, G, P, r, m, n);
-    return cudaGetLastError();
+    const int col_blocks = (n + kProjCols - 1) / kProjCols;
+    const int slabs = (m + kProjChunk - 1) / kProjChunk;
+    int split = kProjResident / col_blocks;                                         // one wave; a function of the shape alone
+    if (split > kProjMaxSplit) split = kProjMaxSplit;
+    if (split > slabs / 2) split = slabs / 2;                                       // at least two slabs per CTA
+    if (split < 1) split = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)col_blocks, (unsigned)split, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)split; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_cesgc_project, B, G, P, r, m, n);
 }
 
 cudaError_t launch_cesgc_back(const float* B, const float* U, float* W, int r, int m, int n, cudaStream_t stream) {
