@@ -560,7 +560,8 @@ def test_mesgc_batched_path_rejects_a_repeated_state(sgc):
 
 
 @pytest.mark.parametrize("m,n,r,c,k,sc", [(512, 256, 8, 4, 28, 4), (1000, 384, 32, 16, 56, 8), (4096, 512, 32, 8, 217, 31),
-                                          (300, 128, 8, 1, 320, 8)])          # the last one: a core too large for the batched chunk path
+                                          (300, 128, 8, 1, 320, 8),          # a core too large for the batched chunk path
+                                          (560, 100, 8, 2, 28, 4)])         # ragged columns; the last CTA of the projection's cluster has no rows
 def test_cesgc_step_matches_its_oracle(sgc, m, n, r, c, k, sc):
     # Section 4.4: SGC (chunked) on B G, update back through B^T; B = first r left-singular vectors of the first gradient
     hp = inputs.ADAM
@@ -587,7 +588,7 @@ def test_cesgc_step_matches_its_oracle(sgc, m, n, r, c, k, sc):
         # a few elements in ten thousand, which differ by one ulp (more for entries that are tiny against their terms,
         # never by more than the ulp of the largest entries)
         off = got_P != P
-        assert off.mean() <= 1e-3 and np.abs(got_P[off] - P[off]).max(initial=0.0) <= np.spacing(np.abs(P).max())
+        assert off.sum() <= max(1, 1e-3 * off.size) and np.abs(got_P[off] - P[off]).max(initial=0.0) <= np.spacing(np.abs(P).max())
         for i in range(c):
             st = ce.core.chunks[i]
             for name in ("sel_idx", "lamM", "lamV", "upd_idx"):
