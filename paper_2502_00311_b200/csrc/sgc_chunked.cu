@@ -150,7 +150,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 // recovery in registers, scores all columns of the tile in ascending order (a strict ">" keeps the lowest index).
 // Only the best two columns per recovery leave the block; columns already in the support are skipped when they show up
 // as a new best.
-__host__ __device__ constexpr int corr_ks(int kp) { return kp > 128 ? 2 : 1; }        // threads that share the rows of a residual
+__host__ __device__ constexpr int corr_ks(int kp) { return kp > 64 ? kp / 64 : 1; }   // threads that share the rows of a residual: 64 rows each
 __host__ __device__ constexpr int corr_group(int kp) { return kCorrBlock / corr_ks(kp); }   // recoveries per block
 
 // gate != nullptr: the launch is a fallback of the tensor-core route and returns at once when *gate == 0.
@@ -158,8 +158,9 @@ template <int KP>
 __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter, const int* gate) {
     if (gate != nullptr && *gate == 0) return;
     constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 32);      // columns per tile
-    constexpr int ZS = KP + 4;                                       // row stride of a tile column (16-byte multiple)
-    constexpr int KS = corr_ks(KP), KL = KP / KS;                    // at the largest k two threads hold half the rows each
+    constexpr int KS = corr_ks(KP), KL = KP / KS;                    // KS threads hold KL rows of a residual each
+    constexpr int ZS = KP + 4 * KS;                                  // stride of a tile column: every row part is followed by four
+                                                                     // floats, so that the KS parts a warp reads at once sit in different banks
     extern __shared__ float smem[];
     float* zt = smem;                                                // [TC][ZS]
     float* inv = smem + TC * ZS;                                     // [TC]
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             const int t = threadIdx.x % TC, part = threadIdx.x / TC;
             const long long col = tile + t;
             float n2 = 0.0f;
-            float* dst = zt + t * ZS + part * RG;
+            float* dst = zt + t * ZS;
             if (col < col1) {
                 const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)col);
                 uint32_t hw = key.ck + (uint32_t)(part * RG / 2) * key.mk;
@@ -204,12 +205,13 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
                     hw += key.mk;
                     if (row >= a.k) z.x = 0.0f;
                     if (row + 1 >= a.k) z.y = 0.0f;
-                    dst[q] = z.x; dst[q + 1] = z.y;
+                    const int at = row + 4 * (row / KL);
+                    dst[at] = z.x; dst[at + 1] = z.y;
                     n2 = __fmaf_rn(z.x, z.x, n2);
                     n2 = __fmaf_rn(z.y, z.y, n2);
                 }
             } else {
-                for (int q = 0; q < RG; ++q) dst[q] = 0.0f;
+                for (int q = 0; q < RG; ++q) { const int row = part * RG + q; dst[row + 4 * (row / KL)] = 0.0f; }
             }
             n2p[part * TC + t] = n2;
         }
@@ -221,10 +223,10 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             inv[threadIdx.x] = n2 > 0.0f ? 1.0f / sqrtf(n2) : 0.0f;
         }
         __syncthreads();
-        if (KS == 1 && !active) continue;                            // (with KS = 2 the shuffle below needs every lane)
+        if (KS == 1 && !active) continue;                            // (with KS > 1 the shuffles below need every lane)
         const int n_here = (int)((col1 - tile) < TC ? (col1 - tile) : TC);
         for (int t = 0; t < n_here; ++t) {
-            const float4* zc = reinterpret_cast<const float4*>(zt + t * ZS + h * KL);
+            const float4* zc = reinterpret_cast<const float4*>(zt + t * ZS + h * (KL + 4));
             float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
             for (int q = 0; q < KL / 4; ++q) {
@@ -235,7 +237,8 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
                 acc1 = __fmaf_rn(z.w, rr[4 * q + 3], acc1);
             }
             float dot = acc0 + acc1;
-            if (KS == 2) dot += __shfl_xor_sync(0xffffffffu, dot, 1);        // the other half of the rows
+#pragma unroll
+            for (int o = 1; o < KS; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // the other parts of the rows
             const float sc = fabsf(dot) * inv[t];
             if (active && sc > s2) {
                 const uint32_t col = (uint32_t)(tile + t);
@@ -269,7 +272,46 @@ struct PickSmem {
     uint32_t cidx[kRescoreCap];
     int n_c;
     float fred[kPickThreads / 32];
+    // what the update of a pick reads of the recovery's state, fetched in one round trip (pick_stage)
+    double F[kChunkMaxS * kChunkMaxS];
+    double r[kChunkMaxK], y[kChunkMaxK], x0[kChunkMaxS];
+    uint16_t z[kChunkMaxS * kChunkMaxK + 2];                          // (the columns start at z[0] or z[1]: see pick_columns)
 };
+
+// Copies the state that pick j of a recovery reads (the j earlier columns, F, x, y and the residual) into shared memory.
+// All loads are independent of one another, so they cost one trip to global memory instead of one per phase of the update.
+// A block-wide barrier has to follow before pick_finish reads them.
+// The staged columns keep the position inside a 32-bit word that they have in global memory, so that they can be copied
+// word by word.
+__device__ __forceinline__ uint16_t* pick_columns(PickSmem& sh, const uint16_t* zs) {
+    return sh.z + (((uintptr_t)zs >> 1) & 1u);
+}
+
+__device__ __forceinline__ void pick_stage(const ChunkArgs& a, const ChunkRef& ref, PickSmem& sh, int m, int j) {
+    const int t = threadIdx.x, k = a.k, s = a.s;
+    const uint16_t* zs = ref.zsel + (size_t)m * s * k;
+    {
+        uint16_t* zsh = pick_columns(sh, zs);
+        const int n = j * k, first = (int)(zsh - sh.z);               // elements before the first whole word: 0 or 1
+        if (n > 0) {
+            const int words = (n - first) / 2;
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(zs + first);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(zsh + first);
+            for (int w = t; w < words; w += kPickThreads) dst[w] = src[w];
+            if (t == 0 && first) zsh[0] = zs[0];
+            if (t == 1 && first + 2 * words < n) zsh[n - 1] = zs[n - 1];
+        }
+    }
+    const double* F = ref.F + (size_t)m * s * s;
+    for (int e = t; e < j * j; e += kPickThreads) {
+        const int l = e / j, i = e - l * j;
+        sh.F[l * kChunkMaxS + i] = F[(size_t)l * s + i];
+    }
+    if (t < j) sh.x0[t] = ref.x[(size_t)m * s + t];
+    const double* r = ref.r64 + (size_t)m * k;
+    const double* y = ref.y64 + (size_t)m * k;
+    for (int row = t; row < k; row += kPickThreads) { sh.r[row] = r[row]; sh.y[row] = y[row]; }
+}
 
 // sums of two values over the block; every thread receives both
 __device__ __forceinline__ void pick_sum2(PickSmem& sh, double& a, double& b) {
@@ -295,17 +337,18 @@ __device__ __forceinline__ float pick_max(PickSmem& sh, float v) {
 }
 
 // the decision among the nc candidates in sh.cidx and the update of the recovery `res` with the winner as pick j
-// (all kPickThreads threads of the block; nc is the same in every thread)
+// (all kPickThreads threads of the block; nc is the same in every thread; pick_stage has run for this recovery)
 __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& sh, int res, int j, int nc) {
     double* gv = sh.gv; double* cv = sh.cv; double* xs = sh.xs;
     const uint32_t* cidx = sh.cidx;
     const int m = res & 1, t = threadIdx.x, lane = t & 31, warp = t >> 5, k = a.k, s = a.s;
     double* r = ref.r64 + (size_t)m * k;
-    const double* y = ref.y64 + (size_t)m * k;
+    const double* y = sh.y;
     if (nc == 0) {                                                   // no column left to pick (d/c = iterations made)
         if (t == 0) { ref.cnt->stopped[m] = 1; ref.cnt->done[m] = j; }
         return;
     }
+    __syncthreads();                                                 // the staged state is complete
     // fp64 scores of the candidates
     double best_sc = -1.0, best_dot = 0.0, best_n2 = 1.0;
     uint32_t best_idx = kNoColumn;
@@ -315,16 +358,17 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double dot = 0.0, n2 = 0.0;
         for (int row = 2 * t; row < k; row += 2 * kPickThreads) {
             const float2 zz = half2_bits_to_float2(z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk));
-            dot += (double)zz.x * r[row];
+            dot += (double)zz.x * sh.r[row];
             n2 += (double)zz.x * (double)zz.x;
-            if (row + 1 < k) { dot += (double)zz.y * r[row + 1]; n2 += (double)zz.y * (double)zz.y; }
+            if (row + 1 < k) { dot += (double)zz.y * sh.r[row + 1]; n2 += (double)zz.y * (double)zz.y; }
         }
         pick_sum2(sh, dot, n2);
         const double sc = n2 > 0.0 ? dot * dot / n2 : 0.0;
         if (sc > best_sc || (sc == best_sc && idx < best_idx)) { best_sc = sc; best_idx = idx; best_dot = dot; best_n2 = n2; }
     }
-    // the new column, binary16 bits (exact)
+    // the new column, binary16 bits (exact): kept in the state and beside the staged ones
     uint16_t* zs = ref.zsel + (size_t)m * s * k;
+    uint16_t* zsh = pick_columns(sh, zs);
     double* F = ref.F + (size_t)m * s * s;
     double* xg = ref.x + (size_t)m * s;
     {
@@ -333,14 +377,15 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         for (int row = 2 * t; row < k; row += 2 * kPickThreads) {
             const uint32_t z2 = z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk);
             znew[row] = (uint16_t)(z2 & 0xFFFFu);
-            if (row + 1 < k) znew[row + 1] = (uint16_t)(z2 >> 16);
+            zsh[j * k + row] = (uint16_t)(z2 & 0xFFFFu);
+            if (row + 1 < k) { znew[row + 1] = (uint16_t)(z2 >> 16); zsh[j * k + row + 1] = (uint16_t)(z2 >> 16); }
         }
     }
     __syncthreads();
     const double sig2 = a.sigma * a.sigma;
-    const uint16_t* znew = zs + (size_t)j * k;
+    const uint16_t* znew = zsh + j * k;
     for (int l = warp; l < j; l += kPickThreads / 32) {              // g = A_Lambda^T a_new, one earlier column per warp
-        const uint16_t* zl = zs + (size_t)l * k;
+        const uint16_t* zl = zsh + l * k;
         double acc = 0.0;
         for (int row = lane; row < k; row += 32) acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));
         acc = warp_sum_d(acc);
@@ -351,7 +396,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double csq = 0.0;
         if (lane < j) {                                              // c = F^T g (F upper triangular, F(l, i) at F[l*s + i])
             double acc = 0.0;
-            for (int l = 0; l <= lane; ++l) acc += F[(size_t)l * s + lane] * gv[l];
+            for (int l = 0; l <= lane; ++l) acc += sh.F[l * kChunkMaxS + lane] * gv[l];
             cv[lane] = acc;
             csq = acc * acc;
         }
@@ -374,7 +419,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double fj = 0.0;                                             // this lane's entry of the new column of F
         if (lane < j) {
             double acc = 0.0;
-            for (int l = lane; l < j; ++l) acc += F[(size_t)lane * s + l] * cv[l];
+            for (int l = lane; l < j; ++l) acc += sh.F[lane * kChunkMaxS + l] * cv[l];
             fj = -gamma * acc;
             F[(size_t)lane * s + j] = fj;
         } else if (lane == j) {
@@ -382,7 +427,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
             F[(size_t)j * s + j] = fj;
         }
         if (lane <= j) {
-            const double xo = lane < j ? xg[lane] : 0.0;
+            const double xo = lane < j ? sh.x0[lane] : 0.0;
             const double xn = xo + aj * fj;
             xg[lane] = xn;
             xs[lane] = xn;
@@ -393,7 +438,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
     double rn2 = 0.0, unused = 0.0;
     for (int row = t; row < k; row += kPickThreads) {                // r = y - A_Lambda x
         double acc = 0.0;
-        for (int l = 0; l <= j; ++l) acc += xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
+        for (int l = 0; l <= j; ++l) acc += xs[l] * (double)half_bits_to_float(zsh[l * k + row]);
         const double rv = y[row] - a.sigma * acc;
         r[row] = rv;
         a.r32[(size_t)res * a.kp + row] = (float)rv;
@@ -416,6 +461,7 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick(ChunkArgs a, int it
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m]) return;
     const int j = iter;
+    pick_stage(a, ref, sh, m, j);                                    // (pick_max's barriers come before anything reads it)
     const Cand* cc = a.cand + (size_t)res * a.splits * 2;
     const int n_entries = a.splits * 2;
     float mx = -1.0f;
@@ -486,6 +532,7 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, in
     const int res = blockIdx.x, m = res & 1, t = threadIdx.x, j = iter;
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m] || a.unresolved[res]) return;
+    pick_stage(a, ref, sh, m, j);
     const unsigned int count = a.rep_count[res];
     bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;      // the same in every thread
     const uint2* rp = a.rep + (size_t)res * kChunkRepCap;
@@ -602,7 +649,7 @@ unsigned long long list_key(sgc_state* const* sts, int c) {
 template <int KP>
 cudaError_t corr_setup(size_t* smem_out) {
     constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 32);
-    const size_t smem = (size_t)(TC * (KP + 4) + TC + kCorrBlock) * sizeof(float);
+    const size_t smem = (size_t)(TC * (KP + 4 * corr_ks(KP)) + TC + kCorrBlock) * sizeof(float);
     *smem_out = smem;
     return cudaFuncSetAttribute(k_chunk_corr<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
