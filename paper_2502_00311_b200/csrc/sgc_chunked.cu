@@ -151,13 +151,14 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 // Only the best two columns per recovery leave the block; columns already in the support are skipped when they show up
 // as a new best.
 __host__ __device__ constexpr int corr_ks(int kp) { return kp > 64 ? kp / 64 : 1; }   // threads that share the rows of a residual: 64 rows each
+__host__ __device__ constexpr int corr_tile(int kp) { return kp <= 64 ? 256 : (kp <= 128 ? 128 : 32); }   // columns per tile
 __host__ __device__ constexpr int corr_group(int kp) { return kCorrBlock / corr_ks(kp); }   // recoveries per block
 
 // gate != nullptr: the launch is a fallback of the tensor-core route and returns at once when *gate == 0.
 template <int KP>
 __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter, const int* gate) {
     if (gate != nullptr && *gate == 0) return;
-    constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 32);      // columns per tile
+    constexpr int TC = corr_tile(KP);
     constexpr int KS = corr_ks(KP), KL = KP / KS;                    // KS threads hold KL rows of a residual each
     constexpr int ZS = KP + 4 * KS;                                  // stride of a tile column: every row part is followed by four
                                                                      // floats, so that the KS parts a warp reads at once sit in different banks
@@ -648,7 +649,7 @@ unsigned long long list_key(sgc_state* const* sts, int c) {
 
 template <int KP>
 cudaError_t corr_setup(size_t* smem_out) {
-    constexpr int TC = KP <= 64 ? 256 : (KP <= 128 ? 128 : 32);
+    constexpr int TC = corr_tile(KP);
     const size_t smem = (size_t)(TC * (KP + 4 * corr_ks(KP)) + TC + kCorrBlock) * sizeof(float);
     *smem_out = smem;
     return cudaFuncSetAttribute(k_chunk_corr<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -676,7 +677,7 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     ws->c = c; ws->key = key; ws->kp = padded_k(st0->k);
     // column splits: enough blocks for every SM twice over, at least one tile per split
     const int groups = (2 * c + corr_group(ws->kp) - 1) / corr_group(ws->kp);
-    const int tile = ws->kp <= 64 ? 256 : (ws->kp <= 128 ? 128 : 32);
+    const int tile = corr_tile(ws->kp);
     int splits = (2 * st0->sm_count + groups - 1) / groups;
     const long long max_splits = (st0->d + tile - 1) / tile;
     if (splits > max_splits) splits = (int)max_splits;
@@ -790,7 +791,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     a.sigma = (double)(float)(1.0 / sqrt((double)st0->k));
     a.r32 = ws->r32; a.cand = ws->cand; a.splits = ws->splits;
     a.cols_per_split = (int)((st0->d + ws->splits - 1) / ws->splits);
-    const int tile = ws->kp <= 64 ? 256 : (ws->kp <= 128 ? 128 : 32);
+    const int tile = corr_tile(ws->kp);
     a.cols_per_split = (a.cols_per_split + tile - 1) / tile * tile;
     a.kp64 = ws->kp64; a.rt = ws->rt; a.tau = ws->tau; a.inv_scale = ws->inv_scale; a.rep_count = ws->rep_count; a.rep = ws->rep;
     a.rnv = ws->rnv; a.unresolved = ws->unresolved; a.flags = ws->flags; a.z_rep = ws->z_rep;
