@@ -681,6 +681,27 @@ cudaError_t corr_setup(size_t* smem_out) {
     return cudaFuncSetAttribute(k_chunk_corr<KP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
+// blocks of k_chunk_corr<KP> that one SM holds at a time (0 on an error)
+template <int KP>
+int corr_resident() {
+    size_t smem = 0;
+    int blocks = 0;
+    if (corr_setup<KP>(&smem) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, k_chunk_corr<KP>, kCorrBlock, smem) != cudaSuccess) return 0;
+    return blocks;
+}
+
+int corr_resident(int kp) {
+    switch (kp) {
+        case 8: return corr_resident<8>();
+        case 16: return corr_resident<16>();
+        case 32: return corr_resident<32>();
+        case 64: return corr_resident<64>();
+        case 128: return corr_resident<128>();
+        default: return corr_resident<256>();
+    }
+}
+
 template <int KP>
 cudaError_t corr_launch(const ChunkArgs& a, int iter, size_t smem, cudaStream_t stream, const int* gate) {
     dim3 grid((unsigned int)a.splits, (unsigned int)((2 * a.c + corr_group(KP) - 1) / corr_group(KP)));
@@ -702,10 +723,12 @@ cudaError_t ensure_ws(sgc_state* const* sts, int c) {
     ChunkWs* ws = new (std::nothrow) ChunkWs();
     if (!ws) return cudaErrorMemoryAllocation;
     ws->c = c; ws->key = key; ws->kp = padded_k(st0->k);
-    // column splits: enough blocks for every SM twice over, at least one tile per split
+    // column splits: as many blocks as the SMs hold at a time (one wave), at least one tile per split
     const int groups = (2 * c + corr_group(ws->kp) - 1) / corr_group(ws->kp);
     const int tile = corr_tile(ws->kp);
-    int splits = (2 * st0->sm_count + groups - 1) / groups;
+    int resident = corr_resident(ws->kp);
+    if (resident < 1) { delete ws; return cudaErrorLaunchOutOfResources; }
+    int splits = resident * st0->sm_count / groups;
     const long long max_splits = (st0->d + tile - 1) / tile;
     if (splits > max_splits) splits = (int)max_splits;
     if (splits < 1) splits = 1;
