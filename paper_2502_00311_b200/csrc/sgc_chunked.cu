@@ -251,7 +251,8 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
         __syncthreads();
         if (KS == 1 && !active) continue;                            // (with KS > 1 the shuffles below need every lane)
         const int n_here = (int)((col1 - tile) < TC ? (col1 - tile) : TC);
-        for (int t = 0; t < n_here; ++t) {
+        // the score of tile column t for this thread's recovery (with KS > 1: every lane of the warp calls it)
+        auto score = [&](int t) -> float {
             const float4* zc = reinterpret_cast<const float4*>(zt + t * ZS + h * (KL + 4));
             float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
@@ -265,16 +266,31 @@ __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter
             float dot = acc0 + acc1;
 #pragma unroll
             for (int o = 1; o < KS; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);   // the other parts of the rows
-            const float sc = fabsf(dot) * inv[t];
-            if (active && sc > s2) {
-                const uint32_t col = (uint32_t)(tile + t);
-                bool taken = false;
-                for (int q = 0; q < iter; ++q) taken |= (sup[q] == col);
-                if (!taken) {
-                    if (sc > s1) { s2 = s1; i2 = i1; s1 = sc; i1 = col; }
-                    else { s2 = sc; i2 = col; }
-                }
+            return fabsf(dot);
+        };
+        auto offer = [&](float sc, int t) {                          // columns are offered in ascending order
+            if (!(sc > s2)) return;
+            const uint32_t col = (uint32_t)(tile + t);
+            bool taken = false;
+            for (int q = 0; q < iter; ++q) taken |= (sup[q] == col);
+            if (taken) return;
+            if (sc > s1) { s2 = s1; i2 = i1; s1 = sc; i1 = col; }
+            else { s2 = sc; i2 = col; }
+        };
+        // from 64 rows on, four columns at a time: four independent chains of multiply-adds, and one compare decides
+        // for all four whether any of them can enter the best two (with few rows the sweep is short, some lane of the
+        // warp nearly always has a new best, and the grouped form only adds work: 63 -> 67 us per step at k_c = 8)
+        int t = 0;
+        for (; KP >= 64 && t + 4 <= n_here; t += 4) {
+            const float4 iv = *reinterpret_cast<const float4*>(inv + t);
+            const float sc0 = score(t) * iv.x, sc1 = score(t + 1) * iv.y, sc2 = score(t + 2) * iv.z, sc3 = score(t + 3) * iv.w;
+            if (active && fmaxf(fmaxf(sc0, sc1), fmaxf(sc2, sc3)) > s2) {
+                offer(sc0, t); offer(sc1, t + 1); offer(sc2, t + 2); offer(sc3, t + 3);
             }
+        }
+        for (; t < n_here; ++t) {
+            const float sc = score(t) * inv[t];
+            if (active) offer(sc, t);
         }
     }
     if (have && h == 0) {
