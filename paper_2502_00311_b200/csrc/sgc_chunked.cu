@@ -20,7 +20,7 @@
 namespace sgc {
 namespace {
 
-constexpr int kFrontThreads = 512;
+constexpr int kFrontThreads = 512;         // at most; short chunks take 256 or 128
 constexpr int kCorrBlock = 256;          // residuals per block of k_chunk_corr
 constexpr int kChunkMaxS = 32;
 constexpr int kChunkMaxK = 256;
@@ -66,7 +66,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 #pragma unroll
     for (int q = 0; q < CAP; ++q) top[q] = 0ull;                    // no real key is 0
     const long long nvec = a.dc >> 2;                                // chunks start on 16-byte boundaries, dc % 4 == 0
-    for (long long v = threadIdx.x; v < nvec; v += kFrontThreads) {
+    for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
         const float4 f = __ldcs(reinterpret_cast<const float4*>(g) + v);
         const float e[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
@@ -88,8 +88,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
         if (lane == 0) wmax[warp] = m;
         __syncthreads();
         unsigned long long best = 0ull;
-#pragma unroll
-        for (int w = 0; w < kFrontThreads / 32; ++w) best = wmax[w] > best ? wmax[w] : best;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) best = wmax[w] > best ? wmax[w] : best;
         if (top[0] == best && best != 0ull) {                        // keys are unique: exactly one thread pops
 #pragma unroll
             for (int q = 0; q + 1 < CAP; ++q) top[q] = top[q + 1];
@@ -123,7 +122,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
     }
     __syncthreads();
     // a2 + a3: thread = row; fp64 sums in ascending column order (the arithmetic of the one-state kernel, term by term)
-    for (int row = threadIdx.x; row < k; row += kFrontThreads) {
+    for (int row = threadIdx.x; row < k; row += blockDim.x) {
         double accp = 0.0, accq = 0.0;
         for (int i = 0; i < s; ++i) {
             const double av = a.sigma * (double)z_at(keys[i], (uint32_t)row);
@@ -868,12 +867,15 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     const double b1 = (double)st0->beta1, b2 = (double)st0->beta2;
     const double c1 = 1.0 - pow(b1, (double)st0->t), c2 = 1.0 - pow(b2, (double)st0->t);
     const int s = st0->s;
-    if (s <= 1) k_chunk_front<1><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 2) k_chunk_front<2><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 4) k_chunk_front<4><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 8) k_chunk_front<8><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 16) k_chunk_front<16><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else k_chunk_front<32><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    // threads per chunk: at least eight 16-byte loads each, so that short chunks get more blocks per SM and cheaper
+    // block-wide rounds
+    const int ft = st0->d >= 16384 ? kFrontThreads : (st0->d >= 8192 ? 256 : 128);
+    if (s <= 1) k_chunk_front<1><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 2) k_chunk_front<2><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 4) k_chunk_front<4><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 8) k_chunk_front<8><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 16) k_chunk_front<16><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else k_chunk_front<32><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
     *launches += 1;
     size_t smem = 0;
     switch (ws->kp) {
