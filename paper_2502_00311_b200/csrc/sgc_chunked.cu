@@ -20,7 +20,7 @@
 namespace sgc {
 namespace {
 
-constexpr int kFrontThreads = 512;         // at most; short chunks take 256 or 128
+constexpr int kFrontThreads = 512;
 constexpr int kCorrBlock = 256;          // residuals per block of k_chunk_corr
 constexpr int kChunkMaxS = 32;
 constexpr int kChunkMaxK = 256;
@@ -66,7 +66,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
 #pragma unroll
     for (int q = 0; q < CAP; ++q) top[q] = 0ull;                    // no real key is 0
     const long long nvec = a.dc >> 2;                                // chunks start on 16-byte boundaries, dc % 4 == 0
-    for (long long v = threadIdx.x; v < nvec; v += blockDim.x) {
+    for (long long v = threadIdx.x; v < nvec; v += kFrontThreads) {
         const float4 f = __ldcs(reinterpret_cast<const float4*>(g) + v);
         const float e[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
@@ -88,7 +88,8 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
         if (lane == 0) wmax[warp] = m;
         __syncthreads();
         unsigned long long best = 0ull;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) best = wmax[w] > best ? wmax[w] : best;
+#pragma unroll
+        for (int w = 0; w < kFrontThreads / 32; ++w) best = wmax[w] > best ? wmax[w] : best;
         if (top[0] == best && best != 0ull) {                        // keys are unique: exactly one thread pops
 #pragma unroll
             for (int q = 0; q + 1 < CAP; ++q) top[q] = top[q + 1];
@@ -122,7 +123,7 @@ k_chunk_front(ChunkArgs a, const float* __restrict__ grad, double b1, double b2,
     }
     __syncthreads();
     // a2 + a3: thread = row; fp64 sums in ascending column order (the arithmetic of the one-state kernel, term by term)
-    for (int row = threadIdx.x; row < k; row += blockDim.x) {
+    for (int row = threadIdx.x; row < k; row += kFrontThreads) {
         double accp = 0.0, accq = 0.0;
         for (int i = 0; i < s; ++i) {
             const double av = a.sigma * (double)z_at(keys[i], (uint32_t)row);
@@ -313,27 +314,41 @@ struct PickSmem {
     uint32_t cidx[kRescoreCap];
     int n_c;
     float fred[kPickThreads / 32];
-    // what the update of a pick reads of the recovery's state, fetched in one round trip (pick_stage)
-    double F[kChunkMaxS * kChunkMaxS];
-    double r[kChunkMaxK], y[kChunkMaxK], x0[kChunkMaxS];
-    uint16_t z[kChunkMaxS * kChunkMaxK + 2];                          // (the columns start at z[0] or z[1]: see pick_columns)
 };
+
+// What the update of a pick reads of the recovery's state, fetched in one round trip (pick_stage), lives in dynamic
+// shared memory sized by s_c and k_c (pick_dyn_bytes), so that small problems keep many blocks per SM:
+// F [s][s], r [k], y [k], x0 [s] as doubles, then the columns z [s * k + 2] (they start at z[0] or z[1]: see pick_columns).
+struct PickDyn { double* F; double* r; double* y; double* x0; uint16_t* z; };
+
+__device__ __forceinline__ PickDyn pick_dyn(const ChunkArgs& a) {
+    extern __shared__ double pick_mem[];
+    PickDyn d;
+    d.F = pick_mem; d.r = d.F + a.s * a.s; d.y = d.r + a.k; d.x0 = d.y + a.k;
+    d.z = reinterpret_cast<uint16_t*>(d.x0 + a.s);
+    return d;
+}
+
+size_t pick_dyn_bytes(int s, int k) {
+    return (size_t)(s * s + 2 * k + s) * sizeof(double) + ((size_t)(s * k + 2) * sizeof(uint16_t) + 7) / 8 * 8;
+}
 
 // Copies the state that pick j of a recovery reads (the j earlier columns, F, x, y and the residual) into shared memory.
 // All loads are independent of one another, so they cost one trip to global memory instead of one per phase of the update.
 // A block-wide barrier has to follow before pick_finish reads them.
 // The staged columns keep the position inside a 32-bit word that they have in global memory, so that they can be copied
 // word by word.
-__device__ __forceinline__ uint16_t* pick_columns(PickSmem& sh, const uint16_t* zs) {
-    return sh.z + (((uintptr_t)zs >> 1) & 1u);
+__device__ __forceinline__ uint16_t* pick_columns(const PickDyn& dy, const uint16_t* zs) {
+    return dy.z + (((uintptr_t)zs >> 1) & 1u);
 }
 
-__device__ __forceinline__ void pick_stage(const ChunkArgs& a, const ChunkRef& ref, PickSmem& sh, int m, int j) {
+__device__ __forceinline__ void pick_stage(const ChunkArgs& a, const ChunkRef& ref, int m, int j) {
     const int t = threadIdx.x, k = a.k, s = a.s;
+    const PickDyn dy = pick_dyn(a);
     const uint16_t* zs = ref.zsel + (size_t)m * s * k;
     {
-        uint16_t* zsh = pick_columns(sh, zs);
-        const int n = j * k, first = (int)(zsh - sh.z);               // elements before the first whole word: 0 or 1
+        uint16_t* zsh = pick_columns(dy, zs);
+        const int n = j * k, first = (int)(zsh - dy.z);               // elements before the first whole word: 0 or 1
         if (n > 0) {
             const int words = (n - first) / 2;
             const uint32_t* src = reinterpret_cast<const uint32_t*>(zs + first);
@@ -346,12 +361,12 @@ __device__ __forceinline__ void pick_stage(const ChunkArgs& a, const ChunkRef& r
     const double* F = ref.F + (size_t)m * s * s;
     for (int e = t; e < j * j; e += kPickThreads) {
         const int l = e / j, i = e - l * j;
-        sh.F[l * kChunkMaxS + i] = F[(size_t)l * s + i];
+        dy.F[l * s + i] = F[(size_t)l * s + i];
     }
-    if (t < j) sh.x0[t] = ref.x[(size_t)m * s + t];
+    if (t < j) dy.x0[t] = ref.x[(size_t)m * s + t];
     const double* r = ref.r64 + (size_t)m * k;
     const double* y = ref.y64 + (size_t)m * k;
-    for (int row = t; row < k; row += kPickThreads) { sh.r[row] = r[row]; sh.y[row] = y[row]; }
+    for (int row = t; row < k; row += kPickThreads) { dy.r[row] = r[row]; dy.y[row] = y[row]; }
 }
 
 // sums of two values over the block; every thread receives both
@@ -384,7 +399,8 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
     const uint32_t* cidx = sh.cidx;
     const int m = res & 1, t = threadIdx.x, lane = t & 31, warp = t >> 5, k = a.k, s = a.s;
     double* r = ref.r64 + (size_t)m * k;
-    const double* y = sh.y;
+    const PickDyn dy = pick_dyn(a);
+    const double* y = dy.y;
     if (nc == 0) {                                                   // no column left to pick (d/c = iterations made)
         if (t == 0) { ref.cnt->stopped[m] = 1; ref.cnt->done[m] = j; }
         return;
@@ -399,9 +415,9 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double dot = 0.0, n2 = 0.0;
         for (int row = 2 * t; row < k; row += 2 * kPickThreads) {
             const float2 zz = half2_bits_to_float2(z_pair_from_word(key.ck + (uint32_t)(row >> 1) * key.mk));
-            dot += (double)zz.x * sh.r[row];
+            dot += (double)zz.x * dy.r[row];
             n2 += (double)zz.x * (double)zz.x;
-            if (row + 1 < k) { dot += (double)zz.y * sh.r[row + 1]; n2 += (double)zz.y * (double)zz.y; }
+            if (row + 1 < k) { dot += (double)zz.y * dy.r[row + 1]; n2 += (double)zz.y * (double)zz.y; }
         }
         pick_sum2(sh, dot, n2);
         const double sc = n2 > 0.0 ? dot * dot / n2 : 0.0;
@@ -409,7 +425,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
     }
     // the new column, binary16 bits (exact): kept in the state and beside the staged ones
     uint16_t* zs = ref.zsel + (size_t)m * s * k;
-    uint16_t* zsh = pick_columns(sh, zs);
+    uint16_t* zsh = pick_columns(dy, zs);
     double* F = ref.F + (size_t)m * s * s;
     double* xg = ref.x + (size_t)m * s;
     {
@@ -437,7 +453,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double csq = 0.0;
         if (lane < j) {                                              // c = F^T g (F upper triangular, F(l, i) at F[l*s + i])
             double acc = 0.0;
-            for (int l = 0; l <= lane; ++l) acc += sh.F[l * kChunkMaxS + lane] * gv[l];
+            for (int l = 0; l <= lane; ++l) acc += dy.F[l * s + lane] * gv[l];
             cv[lane] = acc;
             csq = acc * acc;
         }
@@ -460,7 +476,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
         double fj = 0.0;                                             // this lane's entry of the new column of F
         if (lane < j) {
             double acc = 0.0;
-            for (int l = lane; l < j; ++l) acc += sh.F[lane * kChunkMaxS + l] * cv[l];
+            for (int l = lane; l < j; ++l) acc += dy.F[lane * s + l] * cv[l];
             fj = -gamma * acc;
             F[(size_t)lane * s + j] = fj;
         } else if (lane == j) {
@@ -468,7 +484,7 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
             F[(size_t)j * s + j] = fj;
         }
         if (lane <= j) {
-            const double xo = lane < j ? sh.x0[lane] : 0.0;
+            const double xo = lane < j ? dy.x0[lane] : 0.0;
             const double xn = xo + aj * fj;
             xg[lane] = xn;
             xs[lane] = xn;
@@ -503,7 +519,7 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick(ChunkArgs a, int it
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m]) return;
     const int j = iter;
-    pick_stage(a, ref, sh, m, j);                                    // (pick_max's barriers come before anything reads it)
+    pick_stage(a, ref, m, j);                                    // (pick_max's barriers come before anything reads it)
     const Cand* cc = a.cand + (size_t)res * a.splits * 2;
     const int n_entries = a.splits * 2;
     float mx = -1.0f;
@@ -574,7 +590,7 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, in
     const int res = blockIdx.x, m = res & 1, t = threadIdx.x, j = iter;
     const ChunkRef ref = a.table[res >> 1];
     if (ref.cnt->stopped[m] || a.unresolved[res]) return;
-    pick_stage(a, ref, sh, m, j);
+    pick_stage(a, ref, m, j);
     const unsigned int count = a.rep_count[res];
     bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;      // the same in every thread
     const uint2* rp = a.rep + (size_t)res * kChunkRepCap;
@@ -867,15 +883,12 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     const double b1 = (double)st0->beta1, b2 = (double)st0->beta2;
     const double c1 = 1.0 - pow(b1, (double)st0->t), c2 = 1.0 - pow(b2, (double)st0->t);
     const int s = st0->s;
-    // threads per chunk: at least eight 16-byte loads each, so that short chunks get more blocks per SM and cheaper
-    // block-wide rounds
-    const int ft = st0->d >= 16384 ? kFrontThreads : (st0->d >= 8192 ? 256 : 128);
-    if (s <= 1) k_chunk_front<1><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 2) k_chunk_front<2><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 4) k_chunk_front<4><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 8) k_chunk_front<8><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else if (s <= 16) k_chunk_front<16><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
-    else k_chunk_front<32><<<c, ft, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    if (s <= 1) k_chunk_front<1><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 2) k_chunk_front<2><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 4) k_chunk_front<4><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 8) k_chunk_front<8><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else if (s <= 16) k_chunk_front<16><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
+    else k_chunk_front<32><<<c, kFrontThreads, 0, stream>>>(a, grad, b1, b2, c1, c2);
     *launches += 1;
     size_t smem = 0;
     switch (ws->kp) {
@@ -902,7 +915,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
                                 st0->sm_count, stream);
             }
             if (e != cudaSuccess) return e;
-            k_chunk_pick_rep<<<2 * c, kPickThreads, 0, stream>>>(a, iter);
+            k_chunk_pick_rep<<<2 * c, kPickThreads, pick_dyn_bytes(s, st0->k), stream>>>(a, iter);
             *launches += 2 + ws->passes;
             gate = ws->flags;
         }
@@ -915,7 +928,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
             default: e = corr_launch<256>(a, iter, smem, stream, gate); break;
         }
         {
-            ChainedLaunch l(dim3((unsigned int)(2 * c)), dim3(kPickThreads), 0, stream);
+            ChainedLaunch l(dim3((unsigned int)(2 * c)), dim3(kPickThreads), pick_dyn_bytes(s, st0->k), stream);
             const unsigned char* only = gate ? ws->unresolved : nullptr;
             if (e == cudaSuccess) e = cudaLaunchKernelEx(&l.cfg, k_chunk_pick, a, iter, gate, only);
         }
