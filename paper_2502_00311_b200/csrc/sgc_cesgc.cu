@@ -30,11 +30,11 @@ constexpr int kCesgcMaxR = 64;
 
 constexpr int kProjStage = 8;            // floats of each slab that one thread moves (at 256 threads: 64 x 32 floats)
 constexpr int kProjMaxSplit = 8;         // CTAs of a cluster (the portable limit), each with a range of G's rows
-constexpr int kProjResident = 4 * 148;   // CTAs of this kernel that the SMs hold at once (58 registers, 256 threads)
+constexpr int kProjResident = 4 * 148;   // CTAs of this kernel that the SMs hold at once (64 registers, 256 threads)
 
-__global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows))
+__global__ void __launch_bounds__(kProjCols * (kCesgcMaxR / kProjRows), 2)   // 64 registers: four blocks of 256 threads per SM
 k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float* __restrict__ P, int r, int m, int n) {
-    __shared__ float bs[kCesgcMaxR][kProjChunk];                      // B[:, row0 .. row0 + 64)
+    __shared__ __align__(16) float bs[kCesgcMaxR][kProjChunk];       // B[:, row0 .. row0 + 64)
     __shared__ float gs[kProjChunk][kProjCols];                       // G[row0 .. row0 + 64, the block's columns]
     cg::cluster_group cluster = cg::this_cluster();
     const int groups = (r + kProjRows - 1) / kProjRows;
@@ -80,19 +80,24 @@ k_cesgc_project(const float* __restrict__ B, const float* __restrict__ G, float*
         __syncthreads();
         if (row0 + kProjChunk < m_end) fetch(row0 + kProjChunk);          // in flight while this slab is worked on
         if (!work) continue;
-        const int rows = m_end - row0 < kProjChunk ? m_end - row0 : kProjChunk;
-        for (int q = 0; q < rows; ++q) {
-            const float g = gs[q][jl];
+        // rows of this slab, rounded up to four: what lies beyond m_end was staged as zeros and adds nothing
+        const int rows = ((m_end - row0 < kProjChunk ? m_end - row0 : kProjChunk) + 3) & ~3;
+        for (int q = 0; q < rows; q += 4) {
+            const float g4[4] = {gs[q][jl], gs[q + 1][jl], gs[q + 2][jl], gs[q + 3][jl]};
 #pragma unroll
             for (int u = 0; u < kProjRows; ++u) {
-                const float b = bs[ig * kProjRows + u][q];
-                const float p = __fmul_rn(b, g);
-                const float pe = __fmaf_rn(b, g, -p);                 // b g = p + pe exactly
-                const float t = __fadd_rn(hi[u], p);
-                const float v = __fsub_rn(t, hi[u]);
-                const float te = __fadd_rn(__fsub_rn(hi[u], __fsub_rn(t, v)), __fsub_rn(p, v));   // hi + p = t + te exactly
-                hi[u] = t;
-                lo[u] = __fadd_rn(lo[u], __fadd_rn(te, pe));
+                const float4 b4 = *reinterpret_cast<const float4*>(&bs[ig * kProjRows + u][q]);   // one address per warp
+                const float bq[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {                         // ascending rows of G: the order of the sums is fixed
+                    const float p = __fmul_rn(bq[e], g4[e]);
+                    const float pe = __fmaf_rn(bq[e], g4[e], -p);     // b g = p + pe exactly
+                    const float t = __fadd_rn(hi[u], p);
+                    const float v = __fsub_rn(t, hi[u]);
+                    const float te = __fadd_rn(__fsub_rn(hi[u], __fsub_rn(t, v)), __fsub_rn(p, v));   // hi + p = t + te exactly
+                    hi[u] = t;
+                    lo[u] = __fadd_rn(lo[u], __fadd_rn(te, pe));
+                }
             }
         }
     }
