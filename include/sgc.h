@@ -52,7 +52,8 @@ enum {
     SGC_ERR_WHAT = -5,        /* unknown selector for sgc_get                                  */
     SGC_ERR_SIZE = -6,        /* destination buffer too small                                  */
     SGC_ERR_GROUP = -7,       /* states of a group do not share (d, k, s, seed)                */
-    SGC_ERR_NOSTEP = -8       /* a record was requested before the first step                  */
+    SGC_ERR_NOSTEP = -8,      /* a record was requested before the first step                  */
+    SGC_ERR_DEVICE = -9       /* the current device is not the one the state was created on    */
 };
 
 /* bits of the status word (sticky until sgc_clear_status) */
@@ -63,7 +64,9 @@ enum {
     SGC_STATUS_NEGATIVE_V = 1u << 3,       /* a recovered second-moment entry was <= 0; skipped   */
     SGC_STATUS_CANDIDATE_OVERFLOW = 1u << 4, /* a bounded candidate buffer overflowed; the step
                                                 fell back to its slower exact path               */
-    SGC_STATUS_SELECT_FALLBACK = 1u << 5   /* the sampled top-s threshold missed; exact fallback ran */
+    SGC_STATUS_SELECT_FALLBACK = 1u << 5,  /* the sampled top-s threshold missed; exact fallback ran */
+    SGC_STATUS_TIMEOUT = 1u << 6           /* a bounded wait inside a tensor-core screening pass ran out; the pass's
+                                              reports were discarded and the step finished on its slower exact path */
 };
 
 /* selectors for sgc_get: records of the LAST step, copied to a host buffer */
@@ -109,7 +112,7 @@ enum {
  * workspace on the current device; the library owns them until sgc_destroy.
  *   out    host pointer receiving the handle (set to NULL on failure)
  *   d      length of the flat weight / gradient vector, 1 <= d < 2^32
- *   k      rows of A (dimension of the compressed space), 1 <= k <= 65536
+ *   k      rows of A (dimension of the compressed space), 1 <= k <= 16384
  *   s      sparsity, 1 <= s <= min(k, d), s <= 1024
  *   seed   names the matrix A
  *   lr     learning rate eta of Eq. (3); beta1, beta2, eps: Algorithm 2 "Require"
@@ -204,6 +207,20 @@ SGC_API int sgc_set_state(sgc_state* st, const float* M, const float* V, int64_t
 /* Clears the sticky status word. */
 SGC_API int sgc_clear_status(sgc_state* st);
 
+/* The status word (SGC_STATUS_* bits, sticky until sgc_clear_status): synchronises with the state's last step and
+ * stores the word in *out (host pointer).  Same value as sgc_get(st, SGC_GET_STATUS, ...). */
+SGC_API int sgc_status(sgc_state* st, uint32_t* out);
+
+/* Bound, in nanoseconds, of every wait on a hardware barrier inside the tensor-core screening pass (the only kernel of
+ * this library whose warps wait for one another through memory).  When a wait runs out, the pass records the fact,
+ * lets the copies and matrix operations in flight finish, releases its tensor memory and returns; the step then
+ * discards the pass's reports, finishes on the exact lock-step path and sets SGC_STATUS_TIMEOUT.  The paper has no
+ * counterpart: this is failure handling, and the setter exists so that the path can be exercised (a bound of a few
+ * nanoseconds makes ordinary waits run out without anything being broken).
+ *   st   the state whose passes are meant; NULL sets the bound used by sgc_screen (process-wide)
+ *   ns   0 restores the default of two seconds */
+SGC_API int sgc_set_wait_limit(sgc_state* st, uint64_t ns);
+
 /* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out);
 
@@ -221,7 +238,8 @@ SGC_API int sgc_last_launches(sgc_state* st, int32_t* out);
  *   out_status  device pointer to one uint32 receiving SGC_STATUS_* bits of this call, or NULL
  *   stream      a cudaStream_t; all work is enqueued there, the call does not synchronise
  * The first call on each device looks up the device address of the static array (cudaGetSymbolAddress)
- * and should therefore come before any stream capture.  Every call on a device shares that array and
+ * and should therefore come before any stream capture; devices with an index of 64 or more are not served
+ * (SGC_ERR_DIM).  Every call on a device shares that array and
  * finds the previous call's contents in it: what must start at zero is cleared on `stream` first.  Calls
  * that overlap on the GPU race on the array; serialise them (one stream, or events between streams). */
 SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t s, uint32_t* out_idx, float* out_val,

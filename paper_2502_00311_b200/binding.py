@@ -14,7 +14,8 @@ _lib = None
 
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_cesgc_step", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
            "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
-           "sgc_set_mode", "sgc_set_recovery", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version"]
+           "sgc_set_mode", "sgc_set_recovery", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version", "sgc_status",
+           "sgc_set_wait_limit"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -34,6 +35,7 @@ STATUS_SUPPORT_MISMATCH = 4
 STATUS_NEGATIVE_V = 8
 STATUS_CANDIDATE_OVERFLOW = 16
 STATUS_SELECT_FALLBACK = 32
+STATUS_TIMEOUT = 64
 
 
 class SgcError(RuntimeError):
@@ -72,6 +74,10 @@ def lib():
         L.sgc_set_state.argtypes = [vp, vp, vp, C.c_int64]
         L.sgc_clear_status.restype = C.c_int
         L.sgc_clear_status.argtypes = [vp]
+        L.sgc_status.restype = C.c_int
+        L.sgc_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+        L.sgc_set_wait_limit.restype = C.c_int
+        L.sgc_set_wait_limit.argtypes = [vp, C.c_uint64]
         L.sgc_last_launches.restype = C.c_int
         L.sgc_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
         L.sgc_set_profile.restype = C.c_int
@@ -109,6 +115,11 @@ def version():
 def _check(rc, where):
     if rc != 0:
         raise SgcError(rc, where)
+
+
+def set_screen_wait_limit(ns):
+    """Bound (ns) of the waits inside the pass that sgc_screen launches; 0 restores the default."""
+    _check(lib().sgc_set_wait_limit(None, C.c_uint64(int(ns))), "sgc_set_wait_limit")
 
 
 def _dev_ptr(t, n, what):
@@ -216,6 +227,15 @@ class Sgc:
             raise ValueError("M and V must have k elements")
         _check(lib().sgc_set_state(self._h, M.ctypes.data_as(C.c_void_p), V.ctypes.data_as(C.c_void_p), int(t)),
                "sgc_set_state")
+
+    def status(self):
+        out = C.c_uint32(0)
+        _check(lib().sgc_status(self._h, C.byref(out)), "sgc_status")
+        return out.value
+
+    def set_wait_limit(self, ns):
+        """Bound (ns) of the waits inside this state's screening passes; 0 restores the default."""
+        _check(lib().sgc_set_wait_limit(self._h, C.c_uint64(int(ns))), "sgc_set_wait_limit")
 
     def clear_status(self):
         _check(lib().sgc_clear_status(self._h), "sgc_clear_status")

@@ -1,5 +1,6 @@
 // C ABI of the SGC library (include/sgc.h): argument checks, state life cycle, step orchestration.
 #include <math.h>
+#include <atomic>
 #include <new>
 #include <string.h>
 
@@ -8,6 +9,14 @@
 namespace {
 
 inline size_t align_up(size_t v) { return (v + 255) & ~(size_t)255; }
+
+std::atomic<unsigned long long> g_screen_wait_limit_ns{0};      // sgc_screen's bound on the waits of its pass; 0 = default
+
+// a state may only be stepped on the device it was created on
+bool on_own_device(const sgc_state* st) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == st->device;
+}
 
 template <class T>
 T* carve(unsigned char* base, size_t& off, size_t count) {
@@ -149,12 +158,15 @@ SGC_API int sgc_create(sgc_state** out, int64_t d, int32_t k, int32_t s, uint64_
 SGC_API int sgc_step(sgc_state* st, const float* grad, float* weight, void* stream) {
     if (!st || !grad || !weight) return SGC_ERR_NULL;
     if (((uintptr_t)grad & 15u) || ((uintptr_t)weight & 15u)) return SGC_ERR_ALIGN;
+    if (!on_own_device(st)) return SGC_ERR_DEVICE;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    st->t += 1;
     int launches = 0;
+    // t counts the steps whose gradient has entered M and V: it moves once the kernel that updates them is enqueued
+    st->t += 1;
     cudaError_t e = sgc::launch_select(st, grad, cs, &launches);
     if (e == cudaSuccess) e = sgc::launch_project_adam(st, cs, &launches);
-    if (e == cudaSuccess) e = sgc::launch_recover(st, weight, cs, &launches);
+    if (e != cudaSuccess) { st->t -= 1; return (int)e; }
+    e = sgc::launch_recover(st, weight, cs, &launches);
     st->last_stream = cs; st->has_stream = true; st->stepped = true; st->last_launches = launches;
     return (int)e;
 }
@@ -169,6 +181,7 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
             return SGC_ERR_GROUP;
         if (((uintptr_t)grads[i] & 15u) || ((uintptr_t)weights[i] & 15u)) return SGC_ERR_ALIGN;
         for (int32_t j = 0; j < i; ++j) if (states[j] == states[i]) return SGC_ERR_GROUP;
+        if (!on_own_device(states[i])) return SGC_ERR_DEVICE;
     }
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     std::vector<int> launches((size_t)n, 0);
@@ -178,6 +191,7 @@ SGC_API int sgc_step_group(sgc_state* const* states, const float* const* grads, 
         st->t += 1;
         e = sgc::launch_select(st, grads[i], cs, &launches[i]);
         if (e == cudaSuccess) e = sgc::launch_project_adam(st, cs, &launches[i]);
+        if (e != cudaSuccess) st->t -= 1;                           // this state's moments were not touched
     }
     int shared = 0;
     if (e == cudaSuccess) e = sgc::launch_recover_group(states, weights, n, cs, &shared);   // a4 + a5, passes shared per batch
@@ -200,6 +214,7 @@ SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* g
     for (int32_t i = 0; i < c && alike; ++i) {
         if (!states[i]) return SGC_ERR_NULL;
         alike = states[i]->d == dc && states[i]->k == states[0]->k && states[i]->s == states[0]->s && states[i]->seed == states[0]->seed;
+        if (!on_own_device(states[i])) return SGC_ERR_DEVICE;
     }
     if (!alike) return SGC_ERR_GROUP;
     if (sgc::chunked_batch_eligible(states, c)) {
@@ -210,6 +225,7 @@ SGC_API int sgc_step_chunked(sgc_state* const* states, int32_t c, const float* g
         int launches = 0;
         const cudaError_t e = sgc::launch_chunked_batch(states, c, grad, weight, cs, &launches);
         if (e == cudaErrorInvalidValue) { for (int32_t i = 0; i < c; ++i) states[i]->t -= 1; return SGC_ERR_GROUP; }
+        if (e != cudaSuccess && launches == 0) { for (int32_t i = 0; i < c; ++i) states[i]->t -= 1; return (int)e; }
         for (int32_t i = 0; i < c; ++i) {
             sgc_state* st = states[i];
             st->last_stream = cs; st->has_stream = true; st->stepped = true;
@@ -360,6 +376,20 @@ SGC_API int sgc_clear_status(sgc_state* st) {
     return (int)e;
 }
 
+SGC_API int sgc_status(sgc_state* st, uint32_t* out) {
+    if (!st || !out) return SGC_ERR_NULL;
+    cudaError_t e = cudaSuccess;
+    if (st->has_stream) e = cudaStreamSynchronize(st->last_stream);
+    if (e == cudaSuccess) e = cudaMemcpy(out, &st->cnt->status, sizeof(uint32_t), cudaMemcpyDeviceToHost);
+    return (int)e;
+}
+
+SGC_API int sgc_set_wait_limit(sgc_state* st, uint64_t ns) {
+    if (st) st->wait_limit_ns = (unsigned long long)ns;
+    else g_screen_wait_limit_ns.store((unsigned long long)ns);
+    return SGC_OK;
+}
+
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out) {
     if (!st || !out) return SGC_ERR_NULL;
     *out = st->last_launches;
@@ -409,7 +439,7 @@ SGC_API int sgc_z_block(uint64_t seed, int64_t row0, int64_t nrows, int64_t col0
 SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uint16_t* rt, const float* tau, uint32_t* rep_count,
                        uint32_t* rep, int32_t rep_cap, int32_t* error_flag, void* stream) {
     if (!rt || !tau || !rep_count || !rep || !error_flag) return SGC_ERR_NULL;
-    if (d < 1 || d >= ((int64_t)1 << 32) || k < 64 || k > sgc::kMaxK || k % 64 != 0 || n < 32 || n > sgc::kPassMaxN ||
+    if (d < 1 || d >= ((int64_t)1 << 32) || k < 64 || k > sgc::kPassMaxK || k % 64 != 0 || n < 32 || n > sgc::kPassMaxN ||
         n % 32 != 0 || rep_cap < 1)
         return SGC_ERR_DIM;
     if (((uintptr_t)rt & 15u) || ((uintptr_t)rep & 7u)) return SGC_ERR_ALIGN;
@@ -426,7 +456,7 @@ SGC_API int sgc_screen(uint64_t seed, int64_t d, int32_t k, int32_t n, const uin
         int* errors[sgc::kPassMaxBatch] = {error_flag};
         if (e == cudaSuccess)
             e = sgc::launch_pass(map, seed, (uint64_t)d, k, n, tau, nullptr, nullptr, rep_count, reinterpret_cast<uint2*>(rep), rep_cap,
-                                 nullptr, errors, sms, cs);
+                                 nullptr, errors, sms, cs, nullptr, nullptr, 0, g_screen_wait_limit_ns.load());
     }
     return (int)e;
 }
@@ -435,7 +465,7 @@ SGC_API const char* sgc_strerror(int code) {
     switch (code) {
         case SGC_OK: return "success";
         case SGC_ERR_NULL: return "a required pointer is NULL";
-        case SGC_ERR_DIM: return "dimension out of range (need 1 <= s <= min(k, d), d < 2^32, k <= 65536, s <= 1024; "
+        case SGC_ERR_DIM: return "dimension out of range (need 1 <= s <= min(k, d), d < 2^32, k <= 16384, s <= 1024; "
                                  "the speculative recovery and sgc_screen need k to be a multiple of 64)";
         case SGC_ERR_HYPER: return "hyper-parameter out of range (beta in [0,1), eps > 0, finite lr and alpha)";
         case SGC_ERR_ALIGN: return "grad and weight must be 16-byte aligned";
@@ -443,6 +473,7 @@ SGC_API const char* sgc_strerror(int code) {
         case SGC_ERR_SIZE: return "destination buffer too small";
         case SGC_ERR_GROUP: return "states of a group must be distinct and share d, k, s and seed";
         case SGC_ERR_NOSTEP: return "no step has run yet";
+        case SGC_ERR_DEVICE: return "the state belongs to another device than the current one";
         default: break;
     }
     if (code > 0) return cudaGetErrorString((cudaError_t)code);

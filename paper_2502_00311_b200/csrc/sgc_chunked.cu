@@ -40,6 +40,7 @@ struct ChunkArgs {
     uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; uint2* rep;
     double* rnv; unsigned char* unresolved; int* flags;
     double z_rep;
+    int epoch0;                          // flags[0] == epoch0 + iteration: that iteration left a recovery unresolved
 };
 
 __device__ __forceinline__ double warp_sum_d(double v) {
@@ -178,11 +179,12 @@ struct ChainedLaunch {
     }
 };
 
-// gate != nullptr: the launch is a fallback of the tensor-core route and returns at once when *gate == 0.
+// gate != nullptr: the launch is a fallback of the tensor-core route and returns at once unless *gate names this
+// iteration (a.epoch): the word holds the epoch of the last iteration that left a recovery unresolved.
 template <int KP>
 __global__ void __launch_bounds__(kCorrBlock) k_chunk_corr(ChunkArgs a, int iter, const int* gate) {
     after_previous_kernel(a.early);
-    if (gate != nullptr && *gate == 0) return;
+    if (gate != nullptr && *gate != a.epoch0 + iter) return;
     constexpr int TC = corr_tile(KP);
     constexpr int KS = corr_ks(KP), KL = KP / KS;                    // KS threads hold KL rows of a residual each
     constexpr int ZS = KP + 4 * KS;                                  // stride of a tile column: every row part is followed by four
@@ -509,11 +511,12 @@ __device__ void pick_finish(const ChunkArgs& a, const ChunkRef& ref, PickSmem& s
 }
 
 // SIMT route: the candidates are the columns that phase A left within 2e-3 (relative) of the best fp32 score.
-// only != nullptr: a second chance for the recoveries that the tensor-core route marked unresolved; *gate == 0 skips it.
+// only != nullptr: a second chance for the recoveries that the tensor-core route marked unresolved; skipped unless *gate
+// names this iteration.
 __global__ void __launch_bounds__(kPickThreads) k_chunk_pick(ChunkArgs a, int iter, const int* gate, const unsigned char* only) {
     __shared__ PickSmem sh;
     after_previous_kernel(a.early);
-    if (gate != nullptr && *gate == 0) return;
+    if (gate != nullptr && *gate != a.epoch0 + iter) return;
     const int res = blockIdx.x, m = res & 1, t = threadIdx.x;
     if (only != nullptr && !only[res]) return;
     const ChunkRef ref = a.table[res >> 1];
@@ -550,10 +553,9 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick(ChunkArgs a, int it
 // reports every (column, recovery) pair above it, and k_chunk_pick_rep takes the candidates from the reports: every
 // column within twice the pass's error bound of the best report.  Whatever that cannot settle (no report, too many, a
 // window that reaches below the threshold, a zero residual) is marked unresolved and goes through the fp32 route.
-__global__ void __launch_bounds__(64) k_chunk_rt(ChunkArgs a, int n_rows) {
+__global__ void __launch_bounds__(64) k_chunk_rt(ChunkArgs a, int n_rows, int iter) {
     __shared__ double red[2];
     const int row = blockIdx.x, t = threadIdx.x;
-    if (row == 0 && t == 0) a.flags[0] = 0;
     const float inf = __int_as_float(0x7f800000);
     bool live = row < 2 * a.c;
     const ChunkRef* ref = live ? &a.table[row >> 1] : nullptr;
@@ -570,7 +572,7 @@ __global__ void __launch_bounds__(64) k_chunk_rt(ChunkArgs a, int n_rows) {
     __syncthreads();
     const double rn = sqrt(red[0] + red[1]);
     if (!(rn > 0.0) || !isfinite(rn)) {                               // nothing to screen: the fp32 route decides
-        if (t == 0) { a.tau[row] = inf; a.rep_count[row] = 0u; a.unresolved[row] = 1; a.flags[0] = 1; }
+        if (t == 0) { a.tau[row] = inf; a.rep_count[row] = 0u; a.unresolved[row] = 1; a.flags[0] = a.epoch0 + iter; }   // every writer of an iteration stores the same value
         return;
     }
     const double sc = residual_scale(rn);
@@ -592,7 +594,8 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, in
     if (ref.cnt->stopped[m] || a.unresolved[res]) return;
     pick_stage(a, ref, m, j);
     const unsigned int count = a.rep_count[res];
-    bool give_up = a.flags[1] != 0 || count == 0u || count > (unsigned int)kChunkRepCap;      // the same in every thread
+    const bool timed_out = a.flags[1] != 0;                          // a wait inside a pass of this step ran out: its reports are void
+    bool give_up = timed_out || count == 0u || count > (unsigned int)kChunkRepCap;      // the same in every thread
     const uint2* rp = a.rep + (size_t)res * kChunkRepCap;
     const uint32_t* sup = ref.lam + (size_t)m * a.s;
     float smax = -1.0f;
@@ -609,7 +612,7 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, in
     float lo = 0.0f;
     if (!give_up) {
         const double rn = a.rnv[res];
-        lo = (float)((double)smax - 2.0 * screen_margin(rn, (double)smax));
+        lo = (float)((double)smax - 2.0 * screen_margin(rn, (double)smax, a.kp64));
         // the window must stay above the report threshold, or a column inside it may not have been reported
         if (!((double)lo > a.z_rep * rn / sqrt((double)a.k) * 1.001)) give_up = true;
     }
@@ -629,7 +632,10 @@ __global__ void __launch_bounds__(kPickThreads) k_chunk_pick_rep(ChunkArgs a, in
         if (sh.n_c > kRescoreCap) give_up = true;
     }
     if (give_up) {
-        if (t == 0) { a.unresolved[res] = 1; a.flags[0] = 1; }
+        if (t == 0) {
+            a.unresolved[res] = 1; a.flags[0] = a.epoch0 + iter;
+            if (timed_out) atomicOr(&ref.cnt->status, (unsigned int)SGC_STATUS_TIMEOUT);
+        }
         return;
     }
     pick_finish(a, ref, sh, res, j, sh.n_c);
@@ -880,6 +886,12 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
     a.cols_per_split = (a.cols_per_split + tile - 1) / tile * tile;
     a.kp64 = ws->kp64; a.rt = ws->rt; a.tau = ws->tau; a.inv_scale = ws->inv_scale; a.rep_count = ws->rep_count; a.rep = ws->rep;
     a.rnv = ws->rnv; a.unresolved = ws->unresolved; a.flags = ws->flags; a.z_rep = ws->z_rep;
+    // names the iterations of this step in the gate word: 1 + (step count mod 2^20) * 64 + iteration, never 0
+    a.epoch0 = 1 + (int)((st0->t & 0xFFFFF) * 64);
+    if (ws->tensor) {
+        e = cudaMemsetAsync(ws->flags + 1, 0, sizeof(int), stream);      // the time-out flag is per step
+        if (e != cudaSuccess) return e;
+    }
     const double b1 = (double)st0->beta1, b2 = (double)st0->beta2;
     const double c1 = 1.0 - pow(b1, (double)st0->t), c2 = 1.0 - pow(b2, (double)st0->t);
     const int s = st0->s;
@@ -904,7 +916,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
         const int* gate = nullptr;
         if (ws->tensor) {
             // phase A on the tensor cores; the fp32 kernels below then only run for what the reports left open
-            k_chunk_rt<<<ws->n_rows, 64, 0, stream>>>(a, ws->n_rows);
+            k_chunk_rt<<<ws->n_rows, 64, 0, stream>>>(a, ws->n_rows, iter);
             const int* gates[kPassMaxBatch] = {ws->flags + 2};
             int* errors[kPassMaxBatch] = {ws->flags + 1};
             for (int p = 0; p < ws->passes && e == cudaSuccess; ++p) {
@@ -912,7 +924,7 @@ cudaError_t launch_chunked_batch(sgc_state* const* sts, int c, const float* grad
                 const size_t r0 = (size_t)p * kPassMaxN;
                 e = launch_pass(ws->tmap[p], st0->seed, (uint64_t)st0->d, ws->kp64, n_p, ws->tau + r0, ws->inv_scale + r0,
                                 ws->inv_norm, ws->rep_count + r0, ws->rep + r0 * kChunkRepCap, kChunkRepCap, gates, errors,
-                                st0->sm_count, stream);
+                                st0->sm_count, stream, nullptr, nullptr, 0, st0->wait_limit_ns);
             }
             if (e != cudaSuccess) return e;
             k_chunk_pick_rep<<<2 * c, kPickThreads, pick_dyn_bytes(s, st0->k), stream>>>(a, iter);

@@ -94,7 +94,8 @@ __device__ __forceinline__ float z_at(const ColKey& key, uint32_t row) { return 
 // ------------------------------------------------------------------------------------------------
 // limits
 // ------------------------------------------------------------------------------------------------
-constexpr int kMaxK = 65536;
+constexpr int kMaxK = 16384;           // rows of A of a state: the lock-step kernel keeps both residuals (8 bytes per row) in shared memory
+constexpr int kPassMaxK = 65536;       // rows of A of the stand-alone screening pass (sgc_screen)
 constexpr int kMaxS = 1024;
 constexpr int kSelCap = 32768;          // candidate slots of the top-s filter
 constexpr int kSelBins = 4096;          // 12-bit magnitude histogram of the sample
@@ -120,17 +121,24 @@ constexpr int kPassMaxN = 256;          // residuals per screening pass (UMMA N)
 constexpr int kPassMaxBatch = 8;        // states whose residuals one screening pass can serve (kPassMaxN / 32)
 constexpr int kMaxRounds = 24;          // speculate / screen / resolve rounds enqueued per step
 constexpr int kTensorMapBytes = 128;    // sizeof(CUtensorMap)
-// |score computed by the screening pass - exact score| <= kScreenMargin * ||r|| + kScreenNormMargin * score:
-// the residual is rounded to binary16 (relative error 2^-11 per element, hence at most 2^-11 ||r|| by
-// Cauchy-Schwarz), and the pass accumulates the column norm in short binary16 partial sums (error ~1e-4 relative)
-constexpr double kScreenMargin = 5.5e-4;
+// |score computed by the screening pass - exact score| <= (kScreenMargin + k * kScreenAccMargin) * ||r|| + kScreenNormMargin * score:
+//   * the residual is rounded to binary16: relative error 2^-11 per element, hence at most 2^-11 ||r|| (4.9e-4) in the
+//     normalised score by Cauchy-Schwarz (Z itself is exact in binary16);
+//   * the k products are summed in fp32 inside the tensor cores: at most k * 2^-23 * sum |z_i r_i| <= k * 2^-23 ||Z_i|| ||r||
+//     whatever the order of the additions and whether intermediate sums are rounded or truncated;
+//   * 1 / ||Z_i|| comes from a binary16 table (relative error 2^-11), or is accumulated in short binary16 partial sums by the
+//     stand-alone pass (about 1e-4): kScreenNormMargin covers both.
+constexpr double kScreenMargin = 4.9e-4;
+constexpr double kScreenAccMargin = 1.1920928955078125e-7;      // 2^-23 per row of A
 constexpr double kScreenNormMargin = 1.0e-3;
 
 // binary16 residual rows of the screening pass
 __device__ __forceinline__ uint16_t half_rn_bits(double v) { return __half_as_ushort(__double2half(v)); }   // nearest even
 
-// bound on |score seen by the screening pass - exact score| for a residual of norm rn and a score near ps
-__device__ __forceinline__ double screen_margin(double rn, double ps) { return kScreenMargin * rn + kScreenNormMargin * ps; }
+// bound on |score seen by the screening pass - exact score| for a residual of norm rn over k rows and a score near ps
+__device__ __forceinline__ double screen_margin(double rn, double ps, int k) {
+    return (kScreenMargin + (double)k * kScreenAccMargin) * rn + kScreenNormMargin * ps;
+}
 
 // power-of-two scale that brings a residual of norm rn into [2^12, 2^13): no binary16 overflow, and entries
 // down to 2^-26 of the norm stay normal numbers
@@ -158,7 +166,7 @@ struct SpecCtl {
     int finished[2];        // recovery of this residual complete
     int n_cand;             // length of the candidate list
     int rounds;             // screening passes that did work in the last step
-    int pass_error;         // a wait inside the screening pass expired
+    int pass_error;         // a wait inside the screening pass expired (reported as SGC_STATUS_TIMEOUT)
     int stop[2];            // scratch of the cooperative kernel: speculation of residual m has ended
     int list_exact[2];      // 1: the last speculation of residual m compared every list member exactly
     int list_version;       // bumped whenever the candidate list changes
@@ -212,7 +220,8 @@ struct ChunkWs {
     uint16_t* inv_norm;         // [d/c] 1 / ||Z_i|| over the k_c rows, binary16
     double* rnv;                // [2c] ||r|| of every recovery at the start of the iteration
     unsigned char* unresolved;  // [2c] 1: the reports did not settle this recovery's pick; the fp32 route decides it
-    int* flags;                 // [0] some recovery is unresolved, [1] a wait inside a pass expired, [2] constant 1 (gate)
+    int* flags;                 // [0] epoch of the last iteration that left a recovery unresolved, [1] a wait inside a pass of
+                                // this step expired, [2] constant 1 (gate)
     double z_rep;               // report threshold in units of ||r|| / sqrt(k_c)
     unsigned char tmap[8][128]; // tensor maps of the row blocks of rt, one per pass
 };
@@ -281,6 +290,7 @@ struct sgc_state {
     uint32_t* wide_list;        // [2][kWideCap]
     unsigned int* wide_count;   // [2]
     unsigned int* wide_bits;    // [2] bitmaps over [0, d): the column is in the stream's wide list
+    unsigned long long wait_limit_ns;   // bound of the waits inside this state's screening passes; 0 = the default
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };
@@ -289,10 +299,10 @@ namespace sgc {
 enum Phase { kPhaseSample = 0, kPhaseFilter = 1, kPhasePick = 2, kPhaseProject = 3, kPhaseCorr = 4, kPhaseBook = 5,
              kPhaseScatter = 6, kPhasePass = 7, kNumPhases = 8 };
 
-// Brackets the launches issued during its lifetime with a pair of events when profiling is on.
+// Brackets the launches issued during its lifetime with a pair of events when profiling is on (no state: never).
 struct PhaseTimer {
     sgc_state* st; cudaStream_t stream; bool on;
-    PhaseTimer(sgc_state* s, cudaStream_t cs, int phase, int n_launches) : st(s), stream(cs), on(s->profile) {
+    PhaseTimer(sgc_state* s, cudaStream_t cs, int phase, int n_launches) : st(s), stream(cs), on(s != nullptr && s->profile) {
         if (!on) return;
         while (st->ev_pool->size() < st->ev_used + 2) {
             cudaEvent_t e;
@@ -348,6 +358,6 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k);
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
                         int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide = nullptr,
-                        const int* sel = nullptr, int sel_value = 0);
+                        const int* sel = nullptr, int sel_value = 0, unsigned long long wait_limit_ns = 0);   // 0: the default (2 s)
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream);
 }  // namespace sgc

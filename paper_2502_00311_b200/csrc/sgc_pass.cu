@@ -6,8 +6,9 @@
 //   K-major 128-byte-swizzled layout the UMMA descriptors expect;
 //   R^T (N x k, binary16, one residual per row, each row scaled by a power of two) arrives chunk by chunk through TMA;
 //   accumulators live in tensor memory (fp32, 128 lanes = 128 columns of A, N columns each);
-//   the epilogue reads them back with tcgen05.ld, divides by the column norm ||Z_i|| (accumulated by the
-//   generator threads as a by-product) and appends every (column, residual) pair whose score
+//   the epilogue reads them back with tcgen05.ld, divides by the column norm ||Z_i|| (read from the state's table of
+//   1 / ||Z_i||, filled once at creation; only the stand-alone pass of sgc_screen, which has no state, lets its
+//   generator threads accumulate the norm as a by-product) and appends every (column, residual) pair whose score
 //   |<Z_i, R_n>| / ||Z_i|| reaches the residual's threshold tau_n to that residual's report list.
 //
 // Nothing of size d is written: the output is the short report lists.  The pass serves two purposes of the
@@ -16,8 +17,9 @@
 //
 // One persistent CTA per SM; warp roles: 0 = TMA producer, 1 = MMA issuer (owns the tensor-memory
 // allocation), 2-5 = epilogue (one per 32-lane quadrant of tensor memory), 6-21 = generators.
-// Every wait on an mbarrier is bounded (two seconds); on expiry the CTA records an error, leaves all loops,
-// frees its tensor memory and returns.
+// Every wait on an mbarrier is bounded (two seconds unless the caller sets another limit); on expiry the CTA records an
+// error, leaves all loops, waits for the matrix operations and copies it still has in flight, frees its tensor memory and
+// returns.
 #include <cuda.h>
 
 #include <mutex>
@@ -35,7 +37,7 @@ constexpr int kSuperCols = 2 * kTileCols;                    // columns of A per
 constexpr int kChunkRows = 64;                               // rows of A per pipeline stage (128 B of binary16)
 constexpr int kTileBytes = kTileCols * kChunkRows * 2;       // 16384
 constexpr int kNormRing = 8;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default bound of every mbarrier wait
 
 struct PassArgs {
     uint32_t seed_lo, seed_hi;
@@ -62,6 +64,7 @@ struct PassArgs {
     const int* sel; int sel_value;    // optional: the kernel returns at once unless *sel == sel_value (which of two widths runs)
     const int* gate[kPassMaxBatch];   // optional: the kernel returns at once when every *gate is 0 (one per batched state)
     int* error[kPassMaxBatch];        // set to 1 when a wait expired (one per batched state)
+    unsigned long long wait_limit_ns; // bound of every mbarrier wait
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------------
@@ -93,23 +96,27 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // bounded wait: false when the limit expired or another thread of the CTA already gave up.  sleep_ns > 0 backs
-// off between polls so that a waiting warp leaves the issue slots to the generator warps.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns) {
+// off between polls so that a waiting warp leaves the issue slots to the generator warps.  The clock is read every
+// 64th poll, or at every poll when the limit is so short (under a millisecond) that the caller wants waits to expire.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns,
+                                            unsigned long long limit_ns) {
+    const uint32_t every = limit_ns < 1000000ull ? 0u : 63u;
     unsigned long long t0 = 0;
     for (uint32_t i = 0;; ++i) {
         if (sleep_ns) __nanosleep(sleep_ns);
         if (mbar_try(bar, parity)) return true;
-        if ((i & 63u) == 63u) {
+        if ((i & every) == every) {
             if (*abort_flag) return false;
             const unsigned long long t = global_ns();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            else if (t - t0 > limit_ns) { *abort_flag = 1; return false; }
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int sleep_ns,
+                                          unsigned long long limit_ns) {
     if (mbar_try(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, sleep_ns);
+    return mbar_wait_slow(bar, parity, abort_flag, sleep_ns, limit_ns);
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -165,7 +172,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 //   stages x { A tile 0 (16 KB) | A tile 1 (16 KB) | R^T chunk (n x 128 B) }
 //   norms  float[kNormRing][256][2]      partial ||Z_i||^2 of the two generator threads of each column
 //   tau    float[256], 1 / tau float[256]
-//   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2];  tensor-memory base;  abort flag
+//   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2], drain;  tensor-memory base;  abort flag
 // WIDE: the two-level screening code (wide-list harvest, list passes) is compiled in
 template <bool TABLE, bool WIDE>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
@@ -200,8 +207,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     float* itau_s = tau_s + 256;                                     // 1 / tau: a group of 16 residuals is skipped on one compare
     uint64_t* bars = reinterpret_cast<uint64_t*>(itau_s + 256);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8u * a.stages;
-    const uint32_t bar_accf = bar_empty + 8u * a.stages, bar_acce = bar_accf + 16u;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 4);
+    const uint32_t bar_accf = bar_empty + 8u * a.stages, bar_acce = bar_accf + 16u, bar_drain = bar_acce + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 5);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -216,6 +223,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             mbar_init(bar_accf + 8u * b, 1);
             mbar_init(bar_acce + 8u * b, 4);
         }
+        mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
@@ -243,7 +251,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x) {
                 for (int kc = 0; kc < kc_count; ++kc) {
-                    if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 256)) { ok = false; break; }
+                    if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 256, a.wait_limit_ns)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u);
                     tma_load_2d(base + st * stage_bytes + 2 * kTileBytes, &tmap, kc * kChunkRows, 0, bar_full + 8u * st);
                     if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
@@ -262,11 +270,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x, ++sweep_i) {
                 const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
-                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 32)) { ok = false; break; }
+                if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 32, a.wait_limit_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t acc0 = tmem_base + buf * acc_cols, acc1 = acc0 + a.n;
                 for (int kc = 0; kc < kc_count; ++kc) {
-                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 0)) { ok = false; break; }
+                    if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 0, a.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t lo = desc_lo0 + st * stage_step;
                     const uint32_t first = kc != 0 ? 1u : 0u;
@@ -289,7 +297,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         bool ok = true;
         for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x, ++sweep_i) {
             const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag, 512))) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag, 512, a.wait_limit_ns))) { ok = false; break; }
             tc_fence_after();
             const float* nr = norms + (size_t)(sweep_i % kNormRing) * kSuperCols * 2;
 #pragma unroll 1
@@ -376,7 +384,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             uint32_t h = key.ck + (uint32_t)(half * 16) * key.mk;   // one word per row pair
             const uint32_t skip = 16u * key.mk;                  // the other generator thread of this column owns the next 32 rows
             for (int kc = 0; kc < kc_count; ++kc) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 0))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 0, a.wait_limit_ns))) { ok = false; break; }
                 const uint32_t dst = base + st * stage_bytes;
 #pragma unroll
                 for (int c = 0; c < 4; c += 2) {
@@ -408,9 +416,17 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
+        // A wait ran out.  Every role has left its loop, so nothing new is issued from here on; what may still be in
+        // flight are the copies of at most `stages` chunks of R^T and the MMAs of as many stages.  The MMAs are waited
+        // for explicitly (a commit on a barrier of its own arrives once every MMA this thread issued has completed);
+        // the copies (a few KB each, microseconds) get 200 us to land before shared and tensor memory are released.
         if (threadIdx.x == 0)
             for (int q = 0; q < kPassMaxBatch; ++q) if (a.error[q]) atomicExch(a.error[q], 1);
-        // give copies and MMAs still in flight time to land before shared and tensor memory are released
+        if (warp == 1 && lane == 0) {
+            umma_commit(bar_drain);
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try(bar_drain, 0u) && global_ns() - t0 < 2000000ull) __nanosleep(1000);
+        }
         const unsigned long long t0 = global_ns();
         while (global_ns() - t0 < 200000ull) __nanosleep(1000);
         __syncthreads();
@@ -465,7 +481,7 @@ cudaError_t get_encoder(EncodeTiledFn* out) {
 
 size_t pass_smem_bytes(int n, int stages) {
     return 1024 + (size_t)stages * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 512) +
-           8 * (2 * (size_t)stages + 4) + 16;
+           8 * (2 * (size_t)stages + 5) + 16;
 }
 
 }  // namespace
@@ -508,8 +524,9 @@ cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cu
 cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int n, const float* tau, const float* inv_scale,
                         const uint16_t* inv_norm, unsigned int* rep_count, uint2* rep, int rep_cap, const int* const* gates,
                         int* const* errors, int sm_count, cudaStream_t stream, const PassWide* wide, const int* sel,
-                        int sel_value) {
+                        int sel_value, unsigned long long wait_limit_ns) {
     PassArgs a;
+    a.wait_limit_ns = wait_limit_ns ? wait_limit_ns : kWaitLimitNs;
     a.sel = sel; a.sel_value = sel_value;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;

@@ -395,7 +395,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
         if (threadIdx.x == 0) {
             const double ps = sqrt(sh.best_score), rn = sh.cur_rnorm, unit = rn / sqrt((double)k);
             a.pick_score[(size_t)m * s + j] = ps;
-            double t = ps - screen_margin(rn, ps);
+            double t = ps - screen_margin(rn, ps, k);
             if (t > a.z_harvest * unit) t = a.z_harvest * unit;
             if (t < a.z_floor * unit) t = a.z_floor * unit;
             a.tau[m * a.half_n + spec_c] = (float)(t * residual_scale(rn));     // row spec_c was scaled with this norm
@@ -1040,7 +1040,7 @@ __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
         double tau;
         if (j < hi) {
             const double ps = a.pick_score[(size_t)m * s + j];
-            tau = ps - screen_margin(rn, ps);
+            tau = ps - screen_margin(rn, ps, k);
             if (tau > a.z_harvest * unit) tau = a.z_harvest * unit;
             if (tau < a.z_floor * unit) tau = a.z_floor * unit;
         } else {
@@ -1173,7 +1173,11 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
     const bool mini = ra.mini != 0;
     if (!ctl->round_active) return;
     if (ctl->fallback || ctl->pass_error) {
-        if (threadIdx.x == 0) { ctl->fallback = 1; ctl->round_active = 0; }
+        // a wait inside the screening pass ran out: its reports are void, the remaining picks are made in lock-step
+        if (threadIdx.x == 0) {
+            if (ctl->pass_error) atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_TIMEOUT);
+            ctl->fallback = 1; ctl->round_active = 0;
+        }
         return;
     }
     if (mini) {
@@ -1204,7 +1208,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             const uint32_t pick = a.lam[(size_t)m * s + j];
             const double ps = a.pick_score[(size_t)m * s + j];
             const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
-            const float floor_sc = (float)ps - (float)screen_margin(rn, ps);
+            const float floor_sc = (float)ps - (float)screen_margin(rn, ps, a.k);
             const bool skip_members = ctl->list_exact[m] != 0;
             bool hit = false;
             for (unsigned int e = threadIdx.x & 31; e < count; e += 32) {
@@ -1234,7 +1238,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             const uint32_t pick = lam[j];
             const double ps = a.pick_score[(size_t)m * s + j];
             const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
-            const float margin = (float)screen_margin(rn, ps);
+            const float margin = (float)screen_margin(rn, ps, a.k);
             if (threadIdx.x == 0) sh.cand_idx[0] = pick;
             const int nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, j, pick, (float)ps - margin,
                                                2.0f * margin, 1);
@@ -1286,7 +1290,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                 const int n = m * a.half_n + (hi - base);
                 const unsigned int count = a.rep_count[n];
                 const double rn = hi == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + hi - 1];
-                const float margin = (float)screen_margin(rn, 8.0 * rn / sqrt((double)a.k));    // scores near the noise maximum
+                const float margin = (float)screen_margin(rn, 8.0 * rn / sqrt((double)a.k), a.k);    // scores near the noise maximum
                 int nc = -1;
                 if (count >= 1u && count <= (unsigned int)ra.rep_cap)
                     nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, hi, kNoColumn, 0.0f, 2.0f * margin, 0);
@@ -1590,12 +1594,15 @@ double normal_tail_threshold(double d, double target) { return normal_tail_thres
 
 cudaError_t configure_recover(sgc_state* st) {
     const size_t smem = ((size_t)st->k + 1) * sizeof(float2);
-    cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // the opt-in shared-memory limit belongs to the kernel, not to a state: it is set to what the largest supported k
+    // needs, so that states of any size can live side by side on a device
+    constexpr size_t smem_max = ((size_t)kMaxK + 1) * sizeof(float2);
+    static_assert(smem_max + 48 * 1024 <= 227 * 1024, "k_omp: dynamic plus static shared memory must fit one SM");
+    static_assert((size_t)kMaxK * 2 <= 48 * 1024, "k_gram_matrix stages one binary16 column without opting in");
+    cudaError_t e = cudaFuncSetAttribute(k_omp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     int occ = 0;
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_spec_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess && (size_t)st->k * 2 > 48 * 1024)
-        e = cudaFuncSetAttribute(k_gram_matrix, cudaFuncAttributeMaxDynamicSharedMemorySize, st->k * 2);
+    e = cudaFuncSetAttribute(k_spec_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_omp, kOmpThreads, smem);
     if (e != cudaSuccess) return e;
@@ -1717,7 +1724,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     if (two_widths && e == cudaSuccess) {
                         e = launch_pass(st->tmap_half, st->seed, (uint64_t)st->d, st->k, st->pass_n_half, st->tau,
                                         st->inv_scale, st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors,
-                                        st->sm_count, stream, &lp, &st->ctl->narrow, 1);
+                                        st->sm_count, stream, &lp, &st->ctl->narrow, 1, st->wait_limit_ns);
                         *launches += 1;
                     }
                     *launches += 1;
@@ -1761,11 +1768,12 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
                                     lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
                                     lead->sm_count, stream, two_level ? &wide : nullptr,
-                                    two_widths ? &lead->ctl->narrow : nullptr, 0);
+                                    two_widths ? &lead->ctl->narrow : nullptr, 0, lead->wait_limit_ns);
                     if (two_widths && e == cudaSuccess) {
                         e = launch_pass(lead->tmap_half, lead->seed, (uint64_t)lead->d, lead->k, lead->pass_n_half, lead->tau,
                                         lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
-                                        lead->sm_count, stream, two_level ? &wide : nullptr, &lead->ctl->narrow, 1);
+                                        lead->sm_count, stream, two_level ? &wide : nullptr, &lead->ctl->narrow, 1,
+                                        lead->wait_limit_ns);
                         *launches += 1;
                     }
                     *launches += 1;

@@ -233,43 +233,67 @@ k_pick(const float* __restrict__ grad, unsigned long long d, unsigned int s, con
     }
 }
 
-}  // namespace
+// Launch geometry of the selection for a vector of length d with s kept entries: one definition for every caller.
+struct SelectPlan {
+    int direct;                 // the whole vector fits in the candidate list: no threshold needed
+    unsigned int n_chunks;      // sample: 256-element chunks, between 2^10 and 2^16 of them
+    unsigned int target;        // rank in the sample that corresponds to max(2048, 8 s) survivors in the vector
+    int sample_grid;
+    unsigned int filter_blocks;
+};
 
-cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches) {
-    const unsigned long long d = (unsigned long long)st->d;
-    const int direct = d <= (unsigned long long)kSelCap;
-    // sample size: 256-element chunks, between 2^10 and 2^16 of them
+SelectPlan plan_select(unsigned long long d, int s, int sm_count) {
+    SelectPlan p;
+    p.direct = d <= (unsigned long long)kSelCap;
     unsigned long long n_chunks = d / 16384ull;
     if (n_chunks < 1024ull) n_chunks = 1024ull;
     if (n_chunks > 65536ull) n_chunks = 65536ull;
     unsigned long long n_sample = n_chunks * kSampleChunk;
     if (n_sample > d) n_sample = d;
-    unsigned long long want = 8ull * (unsigned long long)st->s;
+    unsigned long long want = 8ull * (unsigned long long)s;
     if (want < 2048ull) want = 2048ull;
     unsigned long long target = (want * n_sample + d - 1) / d;       // rank in the sample
     if (target < 32ull) target = 32ull;
-    int sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
-    if (sample_grid < 1) sample_grid = 1;
-    {
-        PhaseTimer timer(st, stream, kPhaseSample, 1);
-        k_sample<<<direct ? 1 : sample_grid, kSampleThreads, 0, stream>>>(grad, d, (unsigned int)n_chunks, (unsigned int)target,
-                                                                          st->sel_hist, st->cnt, direct);
-    }
-    unsigned long long n4 = d >> 2;
+    p.n_chunks = (unsigned int)n_chunks;
+    p.target = (unsigned int)target;
+    p.sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
+    if (p.sample_grid < 1) p.sample_grid = 1;
+    const unsigned long long n4 = d >> 2;
     unsigned long long blocks = (n4 + 512ull * 4ull - 1) / (512ull * 4ull);
-    const unsigned long long max_blocks = (unsigned long long)st->sm_count * 4ull;
+    const unsigned long long max_blocks = (unsigned long long)sm_count * 4ull;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks < 1) blocks = 1;
+    p.filter_blocks = (unsigned int)blocks;
+    return p;
+}
+
+// The three launches of the selection on `stream`; hist and the counters must be zero on entry (k_sample leaves them
+// so for the next call).  `timed` (may be null) receives the per-kernel timing when profiling is on.
+cudaError_t enqueue_select(const float* grad, unsigned long long d, int s, int sm_count, unsigned int* hist,
+                           unsigned long long* cand, Counters* cnt, uint32_t* out_idx, float* out_val, cudaStream_t stream,
+                           sgc_state* timed) {
+    const SelectPlan p = plan_select(d, s, sm_count);
     {
-        PhaseTimer timer(st, stream, kPhaseFilter, 1);
-        k_filter<<<(unsigned int)blocks, 512, 0, stream>>>(grad, d, st->sel_cand, st->cnt);
+        PhaseTimer timer(timed, stream, kPhaseSample, 1);
+        k_sample<<<p.direct ? 1 : p.sample_grid, kSampleThreads, 0, stream>>>(grad, d, p.n_chunks, p.target, hist, cnt, p.direct);
     }
     {
-        PhaseTimer timer(st, stream, kPhasePick, 1);
-        k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)st->s, st->sel_cand, st->cnt, st->sel_idx, st->sel_val);
+        PhaseTimer timer(timed, stream, kPhaseFilter, 1);
+        k_filter<<<p.filter_blocks, 512, 0, stream>>>(grad, d, cand, cnt);
     }
-    *launches += 3;
+    {
+        PhaseTimer timer(timed, stream, kPhasePick, 1);
+        k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)s, cand, cnt, out_idx, out_val);
+    }
     return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches) {
+    *launches += 3;
+    return enqueue_select(grad, (unsigned long long)st->d, st->s, st->sm_count, st->sel_hist, st->sel_cand, st->cnt,
+                          st->sel_idx, st->sel_val, stream, st);
 }
 
 }  // namespace sgc
@@ -346,28 +370,8 @@ extern "C" SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t
     // counters and histogram must start at zero; the candidate list is overwritten before it is read
     e = cudaMemsetAsync(setup.ptr, 0, kStaticCandOff, cs);
     if (e != cudaSuccess) return (int)e;
-    const unsigned long long du = (unsigned long long)d;
-    const int direct = du <= (unsigned long long)kSelCap;
-    unsigned long long n_chunks = du / 16384ull;
-    if (n_chunks < 1024ull) n_chunks = 1024ull;
-    if (n_chunks > 65536ull) n_chunks = 65536ull;
-    unsigned long long n_sample = n_chunks * kSampleChunk;
-    if (n_sample > du) n_sample = du;
-    unsigned long long want = 8ull * (unsigned long long)s;
-    if (want < 2048ull) want = 2048ull;
-    unsigned long long target = (want * n_sample + du - 1) / du;
-    if (target < 32ull) target = 32ull;
-    int sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
-    if (sample_grid < 1) sample_grid = 1;
-    k_sample<<<direct ? 1 : sample_grid, kSampleThreads, 0, cs>>>(grad, du, (unsigned int)n_chunks, (unsigned int)target,
-                                                                  hist, cnt, direct);
-    unsigned long long n4 = du >> 2;
-    unsigned long long blocks = (n4 + 512ull * 4ull - 1) / (512ull * 4ull);
-    const unsigned long long max_blocks = (unsigned long long)setup.sm_count * 4ull;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (blocks < 1) blocks = 1;
-    k_filter<<<(unsigned int)blocks, 512, 0, cs>>>(grad, du, cand, cnt);
-    k_pick<<<1, kPickThreads, 0, cs>>>(grad, du, (unsigned int)s, cand, cnt, out_idx, out_val);
+    e = enqueue_select(grad, (unsigned long long)d, s, setup.sm_count, hist, cand, cnt, out_idx, out_val, cs, nullptr);
+    if (e != cudaSuccess) return (int)e;
     if (out_status) k_copy_status<<<1, 1, 0, cs>>>(cnt, out_status);
     return (int)cudaGetLastError();
 }

@@ -296,8 +296,29 @@ def test_constant_sparse_gradient_closed_form(sgc):
 
 
 def test_dependent_column_stops_like_the_oracle(sgc):
-    # k = 2: a third column is always dependent; both sides stop after two iterations
-    d, k, s = 64, 2, 2
+    # With s <= k (which sgc_create enforces) the stop needs columns that are dependent although there are at most k of
+    # them.  Seeds whose first two columns at k = 2 are exactly parallel (66855), nearly so (112200: sin^2 = 6.2e-11,
+    # under the 1e-10 pivot bound) and merely ill-conditioned (143364: sin^2 = 1.5e-9) reach it from both sides with
+    # d = 2, s = 2, where the second pick is forced.
+    d, k, s = 2, 2, 2
+    g = np.array([0.75, -1.25], dtype=np.float32)
+    for seed, want_done in ((66855, 1), (112200, 1), (143364, 2)):
+        st = sgc.Sgc(d, k, s, seed, 1e-3, 0.9, 0.999, 1e-8)
+        ref = oracle.Oracle(d, k, s, seed, 1e-3, 0.9, 0.999, 1e-8)
+        w = cuda(np.zeros(4, dtype=np.float32))
+        wr = np.zeros(d, dtype=np.float32)
+        st.step(cuda(np.concatenate([g, np.zeros(2, dtype=np.float32)])), w)
+        ref.step(g, wr)
+        for m in "MV":
+            assert st.get("done" + m) == ref.get("done" + m) == want_done, (seed, m)
+            assert np.array_equal(st.get("lam" + m), ref.get("lam" + m)), (seed, m)
+        assert bool(st.get("status") & sgc.STATUS_DEPENDENT_COLUMN) == (want_done < s)
+        assert st.status() == int(st.get("status"))
+        np.testing.assert_allclose(w.cpu().numpy()[:d], wr, rtol=1e-4, atol=1e-12)
+        st.close()
+        ref.close()
+    # the generic small case: k = 2, s = 2 among 64 columns completes both picks
+    d = 64
     g = np.random.default_rng(3).standard_normal(d).astype(np.float32)
     st = sgc.Sgc(d, k, s, 3, 1e-3, 0.9, 0.999, 1e-8)
     ref = oracle.Oracle(d, k, s, 3, 1e-3, 0.9, 0.999, 1e-8)
@@ -305,7 +326,7 @@ def test_dependent_column_stops_like_the_oracle(sgc):
     wr = np.zeros(d, dtype=np.float32)
     st.step(cuda(g), w)
     ref.step(g, wr)
-    assert st.get("doneM") == ref.get("doneM") and np.array_equal(st.get("lamM"), ref.get("lamM"))
+    assert st.get("doneM") == ref.get("doneM") == 2 and np.array_equal(st.get("lamM"), ref.get("lamM"))
     st.close()
 
 

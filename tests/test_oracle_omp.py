@@ -106,11 +106,57 @@ def test_lowest_index_wins_exact_ties_and_no_reselection():
 
 
 def test_dependent_column_stops_early():
-    # k = 2 rows: a third column is always dependent on two selected ones
-    out = oracle.omp(3, 6, 2, 2, np.array([1.0, -2.0]))
+    # k = 2 rows: two picked columns span the plane, so whichever column the third iteration picks is a combination of
+    # them.  Algorithm 3's gamma = 1/sqrt(g_ll - c^H c) would divide by ~0 there; the oracle's reading is that the
+    # recovery ends with the picks made so far.  s = 3 > k reaches that branch (s = 2 never does).
+    y = np.array([1.0, -2.0])
+    two = oracle.omp(3, 6, 2, 2, y)
+    assert two["done"] == 2
+    out = oracle.omp(3, 6, 2, 3, y)
     assert out["done"] == 2
-    st = oracle.Oracle(6, 2, 2, 3, 1e-3, 0.9, 0.999, 1e-8)
-    st.close()
+    assert out["lam"][2] == 0xFFFFFFFF and out["x"][2] == 0.0 and out["rnorm"][2] == 0.0
+    # the picks before the stop are those of the shorter run, and so is the least-squares fit
+    assert np.array_equal(out["lam"][:2], two["lam"]) and np.array_equal(out["x"][:2], two["x"])
+    # the fit on two independent columns of the plane is exact
+    A = _columns(3, 2, out["lam"][:2])
+    np.testing.assert_allclose(A @ out["x"][:2], y, atol=1e-12)
+    # the same with k = 3: three picks complete (the stop does not fire on independent columns), the fourth cannot
+    y3 = np.array([0.5, -1.0, 2.0])
+    for seed in range(5):
+        assert oracle.omp(seed, 40, 3, 3, y3)["done"] == 3
+        o4 = oracle.omp(seed, 40, 3, 4, y3)
+        assert o4["done"] == 3 and o4["lam"][3] == 0xFFFFFFFF
+        assert len(set(o4["lam"][:3].tolist())) == 3
+
+
+def _sin2_of_first_two_columns(seed):
+    Z = oracle.z_block(seed, 0, 2, 0, 2).astype(np.float64)
+    a, b = Z[:, 0], Z[:, 1]
+    return (a[0] * b[1] - a[1] * b[0]) ** 2 / ((a @ a) * (b @ b))
+
+
+def test_dependence_threshold_from_both_sides():
+    # The stop is for a column whose component outside the span of the support is below 1e-5 of its norm (1e-10 in the
+    # squared, relative pivot).  With k = 2 and d = 2 the second pick is forced, so the angle between the two columns
+    # decides: seeds found by search whose first two columns are exactly parallel, at sin^2 = 6.2e-11 (stop) and at
+    # sin^2 = 1.5e-9 (an ordinary, if ill-conditioned, pick).  A threshold off by a factor of 20 either way fails.
+    y = np.array([0.3, 1.0])
+    assert _sin2_of_first_two_columns(66855) == 0.0
+    assert oracle.omp(66855, 2, 2, 2, y)["done"] == 1
+    s2 = _sin2_of_first_two_columns(112200)
+    assert 5e-11 < s2 < 1e-10
+    out = oracle.omp(112200, 2, 2, 2, y)
+    assert out["done"] == 1 and out["lam"][1] == 0xFFFFFFFF and out["x"][1] == 0.0
+    s2 = _sin2_of_first_two_columns(143364)
+    assert 1e-9 < s2 < 2e-9
+    out = oracle.omp(143364, 2, 2, 2, y)
+    assert out["done"] == 2 and sorted(out["lam"].tolist()) == [0, 1]
+    A = _columns(143364, 2, out["lam"])
+    np.testing.assert_allclose(A @ out["x"], y, rtol=0, atol=1e-7)      # condition number ~ 5e4
+
+
+def _columns(seed, k, lam):
+    return float(oracle.sigma(k)) * np.stack([oracle.z_block(seed, 0, k, int(c), 1)[:, 0] for c in lam], axis=1).astype(np.float64)
 
 
 def test_whole_step_constant_sparse_gradient_closed_form():

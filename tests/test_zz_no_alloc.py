@@ -1,4 +1,5 @@
-"""sgc_sparsify_static: the allocation-free top-s selection must agree with the selection inside sgc_step.
+"""sgc_sparsify_static: the allocation-free top-s selection must agree with the selection inside sgc_step and with
+the CPU oracle's definition of Sparsify_s (full sort by magnitude, ties to the lower index).
 
 The entry point exists for callers that cannot call cudaMalloc when they need a selection (a framework that
 owns all device memory through its own pool, or a thread that must avoid cudaMalloc's device-wide
@@ -9,6 +10,7 @@ values are compared bit for bit, the bar the other selection tests use.  Collect
 import numpy as np
 import pytest
 
+import oracle
 from paper_2502_00311_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -45,6 +47,10 @@ def test_static_selection_matches_step_selection_twice_in_a_row():
         want_idx, want_val = reference_selection(binding, g, d, s)
         assert np.array_equal(got_idx, want_idx), (d, s)
         assert np.array_equal(got_val.view(np.uint32), want_val.view(np.uint32)), (d, s)
+        # the independent reference: the oracle sorts the whole vector
+        orc_idx, orc_val = oracle.sparsify(g.cpu().numpy(), s)
+        assert np.array_equal(got_idx, orc_idx), (d, s)
+        assert np.array_equal(got_val.view(np.uint32), orc_val.view(np.uint32)), (d, s)
         assert int(out_status.item()) == 0
         del g
     # a degenerate vector (all magnitudes equal) takes the exact fallback and says so
@@ -60,6 +66,9 @@ def test_static_selection_matches_step_selection_twice_in_a_row():
     torch.cuda.synchronize()
     want_idx, _ = reference_selection(binding, g, 200_000, 32)
     assert np.array_equal(out_idx[:32].cpu().numpy().view(np.uint32), want_idx)
+    orc_idx, orc_val = oracle.sparsify(g.cpu().numpy(), 32)
+    assert np.array_equal(out_idx[:32].cpu().numpy().view(np.uint32), orc_idx)
+    assert np.array_equal(out_val[:32].cpu().numpy().view(np.uint32), orc_val.view(np.uint32))
     assert int(out_status.item()) == 0
 
 
