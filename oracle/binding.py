@@ -22,7 +22,7 @@ def build(force=False):
     if (not force) and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC):
         return _SO
     tmp = _SO + ".tmp%d" % os.getpid()
-    cmd = ["g++", "-O2", "-std=c++17", "-fopenmp", "-ffp-contract=off", "-mfma", "-shared", "-fPIC",
+    cmd = ["g++", "-O3", "-std=c++17", "-fopenmp", "-ffp-contract=off", "-mavx2", "-mfma", "-shared", "-fPIC",
            _SRC, "-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, _SO)
@@ -61,6 +61,9 @@ def lib():
             L.orc_omp_tol.restype = C.c_int32
             L.orc_omp_tol.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32, f64p, C.c_double, u32p, f64p, f64p, f64p,
                                       f64p]
+            L.orc_select.restype = None
+            L.orc_select.argtypes = [C.c_uint64, C.c_int64, C.c_int32, C.c_int32, f64p, u32p, i32p, C.c_int32,
+                                     C.POINTER(C.c_int64), f64p, f64p]
             L.orc_least_squares.restype = C.c_int32
             L.orc_least_squares.argtypes = [C.c_uint64, C.c_int32, u32p, C.c_int32, f64p, f64p]
             L.orc_set_recovery.restype = None
@@ -160,6 +163,32 @@ def omp(seed, d, k, s, y, residual_tol=0.0):
     done = lib().orc_omp_tol(C.c_uint64(seed), d, k, s, _p(y, C.c_double), float(residual_tol), _p(lam, C.c_uint32),
                              _p(x, C.c_double), _p(t1, C.c_double), _p(t2, C.c_double), _p(rn, C.c_double))
     return dict(done=int(done), lam=lam, x=x, top1=t1, top2=t2, rnorm=rn)
+
+
+def select(seed, d, k, R, skip=None):
+    """The Select line of Algorithm 3 for a batch of residuals R [n, k] against all d columns of A(seed, k x d).
+
+    skip: optional list of n index sequences, the columns excluded for each residual (its support so far).
+    Returns dict(idx [n] int64, best [n], second [n]): argmax column (lowest index on ties) and the two largest scores."""
+    R = np.ascontiguousarray(R, dtype=np.float64)
+    n = R.shape[0]
+    assert R.shape == (n, k)
+    counts = np.zeros(n, dtype=np.int32)
+    stride = 1
+    if skip is not None:
+        assert len(skip) == n
+        counts = np.array([len(sk) for sk in skip], dtype=np.int32)
+        stride = max(1, int(counts.max()))
+    flat = np.zeros((n, stride), dtype=np.uint32)
+    if skip is not None:
+        for i, sk in enumerate(skip):
+            flat[i, :len(sk)] = np.asarray(sk, dtype=np.uint32)
+    idx = np.empty(n, dtype=np.int64)
+    best = np.empty(n, dtype=np.float64)
+    second = np.empty(n, dtype=np.float64)
+    lib().orc_select(C.c_uint64(seed), int(d), int(k), n, _p(R, C.c_double), _p(flat, C.c_uint32), _p(counts, C.c_int32),
+                     stride, _p(idx, C.c_int64), _p(best, C.c_double), _p(second, C.c_double))
+    return dict(idx=idx, best=best, second=second)
 
 
 def least_squares(seed, k, lam, y):

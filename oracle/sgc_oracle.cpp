@@ -27,7 +27,8 @@
 //   column, the treatment of Eq. (8) where the two supports differ or x^V <= 0, and the opt-in variant of
 //   orc_set_recovery (one shared support, early stop on the residual).
 //
-// Beyond the step itself: orc_reproject (SGCA, Appendix C, Algorithm 4), orc_omp_tol / orc_least_squares /
+// Beyond the step itself: orc_select (the Select line of Algorithm 3 for several residuals at once, for checking picks at
+// sizes where s full iterations are out of reach), orc_reproject (SGCA, Appendix C, Algorithm 4), orc_omp_tol / orc_least_squares /
 // orc_set_recovery (the variant built on the remark after Eq. (8)); the chunked (MESGC) and projected (CESGC) forms of
 // Section 4.4 are compositions of these states written out in oracle/binding.py (cesgc_step) and in the tests.
 //
@@ -364,6 +365,74 @@ int32_t orc_omp_tol(uint64_t seed, int64_t d, int32_t k, int32_t s, const double
 int32_t orc_omp(uint64_t seed, int64_t d, int32_t k, int32_t s, const double* y,
                 uint32_t* lam, double* x, double* top1, double* top2, double* rnorm) {
     return orc_omp_tol(seed, d, k, s, y, 0.0, lam, x, top1, top2, rnorm);
+}
+
+// The "Select" line of Algorithm 3 (Appendix B) on its own, for a batch of residuals: for every residual r_n, n < n_res,
+//   idx[n] = argmax over the columns i in [0, d) outside skip_n of |<A_:i, r_n>| / ||A_:i||_2   (lowest i on exact ties),
+// with the best and the second-best score.  skip_n (the columns already in the support of residual n) holds skip_count[n]
+// entries at skip[n * skip_stride ...].  Every residual is treated exactly as one iteration of orc_omp_tol treats its
+// residual; the batch only lets one generated column of A meet all residuals.  R is n_res x k, row-major.
+void orc_select(uint64_t seed, int64_t d, int32_t k, int32_t n_res, const double* R, const uint32_t* skip,
+                const int32_t* skip_count, int32_t skip_stride, int64_t* idx, double* best, double* second) {
+    const double sigma = (double)sigma_of_k(k);
+    std::vector<uint8_t> listed((size_t)d, 0);          // the column is in some residual's skip list
+    for (int32_t n = 0; n < n_res; ++n)
+        for (int32_t q = 0; skip && q < skip_count[n]; ++q) {
+            const uint32_t c = skip[(size_t)n * skip_stride + q];
+            if ((int64_t)c < d) listed[c] = 1;
+        }
+    std::vector<double> Rt((size_t)k * n_res);           // k x n_res: the residuals' entries of one row side by side
+    for (int32_t n = 0; n < n_res; ++n)
+        for (int32_t j = 0; j < k; ++j) Rt[(size_t)j * n_res + n] = R[(size_t)n * k + j];
+    int nthreads = 1;
+#ifdef _OPENMP
+    nthreads = omp_get_max_threads();
+#endif
+    std::vector<double> tb1((size_t)nthreads * n_res, -1.0), tb2((size_t)nthreads * n_res, -1.0);
+    std::vector<int64_t> ti1((size_t)nthreads * n_res, -1);
+#pragma omp parallel
+    {
+        int tid = 0, nt = 1;
+#ifdef _OPENMP
+        tid = omp_get_thread_num(); nt = omp_get_num_threads();
+#endif
+        const int64_t lo = d * tid / nt, hi = d * (tid + 1) / nt;
+        double* b1 = &tb1[(size_t)tid * n_res];
+        double* b2 = &tb2[(size_t)tid * n_res];
+        int64_t* i1 = &ti1[(size_t)tid * n_res];
+        std::vector<double> dot(n_res);
+        for (int64_t i = lo; i < hi; ++i) {
+            const uint32_t ck = column_key(seed, (uint32_t)i);
+            std::fill(dot.begin(), dot.end(), 0.0);
+            double n2 = 0.0;
+            for (int32_t j = 0; j < k; ++j) {
+                const double a = a_entry(ck, (uint32_t)j, sigma);
+                const double* rj = &Rt[(size_t)j * n_res];
+                for (int32_t n = 0; n < n_res; ++n) dot[n] += a * rj[n];
+                n2 += a * a;
+            }
+            const double nrm = std::sqrt(n2);
+            for (int32_t n = 0; n < n_res; ++n) {
+                if (listed[i]) {
+                    bool skipped = false;
+                    for (int32_t q = 0; q < skip_count[n]; ++q) skipped = skipped || skip[(size_t)n * skip_stride + q] == (uint32_t)i;
+                    if (skipped) continue;
+                }
+                const double c = std::fabs(dot[n]) / nrm;
+                if (c > b1[n]) { b2[n] = b1[n]; b1[n] = c; i1[n] = i; }
+                else if (c > b2[n]) { b2[n] = c; }
+            }
+        }
+    }
+    for (int32_t n = 0; n < n_res; ++n) {
+        double b1 = -1.0, b2 = -1.0; int64_t i1 = -1;
+        for (int tdx = 0; tdx < nthreads; ++tdx) {       // ascending column ranges: strict > keeps the lowest index
+            const double c1 = tb1[(size_t)tdx * n_res + n], c2 = tb2[(size_t)tdx * n_res + n];
+            if (c1 > b1) { b2 = std::max(b1, c2); b1 = c1; i1 = ti1[(size_t)tdx * n_res + n]; }
+            else { b2 = std::max(b2, c1); }
+        }
+        idx[n] = i1; best[n] = b1; second[n] = b2;
+    }
 }
 
 // Least squares of y on a given support: x = argmin ||y - A_Lambda x||_2 (the last step of every OMP iteration, on

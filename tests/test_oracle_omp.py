@@ -299,3 +299,49 @@ def test_shared_support_equals_the_printed_algorithm_when_the_supports_coincide(
         np.testing.assert_allclose(Wb, Wa, rtol=0, atol=1e-9)
     a.close()
     b.close()
+
+
+# ---- the batched Select (used to check picks at full size, where s whole iterations are out of reach) --------------
+def test_select_is_the_dense_normalised_argmax_for_every_residual():
+    seed, d, k, n = 12, 3000, 48, 7
+    rng = np.random.default_rng(0)
+    R = rng.standard_normal((n, k))
+    R[3] = 0.0                                                          # all scores tie at zero: lowest free index
+    skip = [sorted(rng.choice(d, size=q, replace=False).tolist()) for q in (0, 1, 5, 2, 0, 9, 3)]
+    skip[3] = [0, 1]
+    out = oracle.select(seed, d, k, R, skip)
+    Z = oracle.z_block(seed, 0, k, 0, d).astype(np.float64)
+    A = float(oracle.sigma(k)) * Z
+    sc = np.abs(R @ A) / np.sqrt((A * A).sum(axis=0))                   # n x d, the definition with A written out
+    for i in range(n):
+        s_i = sc[i].copy()
+        s_i[skip[i]] = -1.0
+        order = np.argsort(-s_i, kind="stable")                         # stable: ties keep the lower index first
+        assert out["idx"][i] == order[0], i
+        np.testing.assert_allclose(out["best"][i], s_i[order[0]], rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(out["second"][i], s_i[order[1]], rtol=1e-12, atol=1e-300)
+    assert out["idx"][3] == 2
+    # without skip lists
+    out0 = oracle.select(seed, d, k, R)
+    assert np.array_equal(out0["idx"], np.argmax(sc, axis=1))
+
+
+def test_select_reproduces_every_iteration_of_omp():
+    # feeding Select the residual before each iteration of a full OMP run (with the support so far excluded) must give
+    # that run's picks and scores back: the batch is s independent copies of one iteration
+    seed, d, k, s = 5, 20_000, 96, 12
+    rng = np.random.default_rng(3)
+    supp = rng.choice(d, size=s, replace=False)
+    A_s = _columns(seed, k, supp)
+    y = A_s @ rng.uniform(1.0, 2.0, size=s) + 0.05 * rng.standard_normal(k)
+    run = oracle.omp(seed, d, k, s, y)
+    R, skip = [], []
+    for j in range(s):
+        lam = run["lam"][:j]
+        r = y if j == 0 else y - _columns(seed, k, lam) @ oracle.least_squares(seed, k, lam, y)
+        R.append(r)
+        skip.append(lam.tolist())
+    out = oracle.select(seed, d, k, np.array(R), skip)
+    assert np.array_equal(out["idx"], run["lam"].astype(np.int64))
+    np.testing.assert_allclose(out["best"], run["top1"], rtol=1e-9)
+    np.testing.assert_allclose(out["second"], run["top2"], rtol=1e-9)
