@@ -1,14 +1,18 @@
 """Benchmark of one SGC optimizer step (sparsify -> project -> k-space Adam -> OMP recovery -> scatter).
 
-    python bench.py --gpus N --steps K --warmup W [--impl ours|reference] [--workload NAME]
+    python bench.py --gpus N --steps K --warmup W [--impl ours|reference] [--workload NAME] [--configs all|none|a,b,...]
 
-Workload at N = 1 (and per rank at N > 1: the path does not shard, ranks are independent replicas):
+Headline workload at N = 1 (and per rank at N > 1: the path does not shard, ranks are independent replicas):
 one fp32 4096x4096 matrix, k = 2048, s = 64, seed 1, Student-t(3)*1e-3 noise + 64 planted U(0.5,1) spikes.
-A "step" is one sgc_step call on a fresh seeded gradient (four gradients of 64 MiB rotate, 256 MiB > L2).
+A "step" is one sgc_step call on a fresh seeded gradient: every warm-up and every timed step has a buffer of its own
+(64 MiB each, never re-read, so no step finds its input in L2).
 
-Prints ONE JSON line: the step time in ms per matrix, device-timed with inputs resident in HBM (`value`), the
-same through host buffers (`e2e`), the roofline of the dominant kernel, and the CPU oracle's time for the
-same step on the host cores (`cpu_baseline`, a bounded sample scaled to the whole step).
+Prints ONE JSON line: the step time in ms per matrix, device-timed with inputs resident in HBM (`value`; median, min
+and p90 of the per-step times beside it), the same through host buffers (`e2e`), the first three steps of a fresh state
+(`cold_start_ms`), the roofline of the dominant kernel, the CPU oracle's time for the same step on the host cores
+(`cpu_baseline`, a bounded sample scaled to the whole step) and, at N = 1, `configs`: the other benchmark
+configurations (one transformer layer as same-A groups, the 32-layer stack, the (k, s) sweep, drifting supports, the
+paper's chunked variants), each with its own per-step statistics.
 `--impl reference` times the CPU oracle alone.
 """
 import argparse
@@ -33,9 +37,13 @@ WORKLOADS = {
     "c1_64x64": dict(d=64 * 64, k=256, s=16, seed=0, kind="gauss", cfg_id=1),
     "small_2M_k2048_s8": dict(d=1 << 21, k=2048, s=8, seed=1, kind="student", cfg_id=2),      # profiler-sized cases
     "small_2M_k2048_s64": dict(d=1 << 21, k=2048, s=64, seed=1, kind="student", cfg_id=2),
+    "small_2M_k2048_s128": dict(d=1 << 21, k=2048, s=128, seed=1, kind="student", cfg_id=3),
     "c5_4096x11008_k1024_s16": dict(d=4096 * 11008, k=1024, s=16, seed=1, kind="student", cfg_id=5),
 }
+EXTRA_CONFIGS = ("drift", "c3_llama7b_layer", "c5_sweep", "mesgc", "c4_llama7b_32layers")
 FP32_LANES_PER_SM = 128
+# sample of the CPU oracle that both the `cpu_baseline` leg and `--impl reference` time
+ORACLE_SAMPLE_COLS, ORACLE_SAMPLE_ITERS = 1 << 20, 8
 
 
 def peaks():
@@ -97,15 +105,23 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
-def oracle_sample(wl, grad, d_cols, iters):
+def spread(ms):
+    """median / min / p90 / mean of per-step times."""
+    a = np.asarray(ms, dtype=np.float64)
+    return dict(ms_median=float(np.median(a)), ms_min=float(a.min()), ms_p90=float(np.percentile(a, 90)),
+                ms_mean=float(a.mean()), steps=int(a.size))
+
+
+def oracle_sample(wl, grad, d_cols=ORACLE_SAMPLE_COLS, iters=ORACLE_SAMPLE_ITERS):
     """Times the CPU oracle on a bounded sample of one step and scales it to the whole step.
 
     a1-a3 run in full.  a4 runs `iters` OMP iterations for ONE of the two residuals against the first d_cols
     columns of A; its time is scaled by (d / d_cols) * (s / iters) * 2 (the oracle's OMP cost is linear in the
     number of columns, iterations and residuals; the least-squares solves are negligible beside k*d per pass).
-    Returns (ms for the whole step, seconds actually spent, threads)."""
+    Returns (ms for the whole step, seconds actually spent, threads, description of the sample)."""
     import oracle
     hp = inputs.ADAM
+    d_cols, iters = min(wl["d"], d_cols), min(wl["s"], iters)
     t0 = time.perf_counter()
     ref = oracle.Oracle(wl["d"], wl["k"], wl["s"], wl["seed"], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
     ref.step_compress(grad)
@@ -116,7 +132,9 @@ def oracle_sample(wl, grad, d_cols, iters):
     t_omp = time.perf_counter() - t0
     ref.close()
     full = t_compress + t_omp * (wl["d"] / d_cols) * (wl["s"] / iters) * 2.0
-    return full * 1e3, t_compress + t_omp, oracle.num_threads()
+    sample = ("a1-a3 in full; a4 = %d of %d OMP iterations of 1 of 2 residuals on %d of %d columns (%.1f s measured), "
+              "scaled linearly in columns*iterations*residuals" % (iters, wl["s"], d_cols, wl["d"], t_compress + t_omp))
+    return full * 1e3, t_compress + t_omp, oracle.num_threads(), sample
 
 
 def run_reference(args, wl):
@@ -124,22 +142,18 @@ def run_reference(args, wl):
     if rank != 0:
         return
     supp, sign = inputs.planted_support(wl["d"], wl["s"], inputs.support_seed(wl["cfg_id"], 0))
-    d_cols, iters = min(wl["d"], 1 << 18), min(wl["s"], 4)
-    times, threads, spent = [], 1, 0.0
+    times, threads, sample = [], 1, ""
     for step in range(args.warmup + args.steps):
         g = inputs.gradient(wl["d"], wl["kind"], supp, sign, inputs.step_seed(wl["cfg_id"], 0, step + 1))
-        ms, sec, threads = oracle_sample(wl, g, d_cols, iters)
-        spent += sec
+        ms, _, threads, sample = oracle_sample(wl, g)
         if step >= args.warmup:
             times.append(ms)
     value = float(np.mean(times))
-    sample = ("per step: a1-a3 in full; a4 = %d of %d OMP iterations of 1 of 2 residuals on %d of %d columns, "
-              "scaled linearly in columns*iterations*residuals" % (iters, wl["s"], d_cols, wl["d"]))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "ms", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": value, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic", "config": {"workload": args.workload, "d": wl["d"], "k": wl["k"], "s": wl["s"]},
-        "cpu_baseline": {"value": value, "unit": "ms", "cores": threads, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "ms", "cores": threads, "kind": "oracle", "sample": "per step: " + sample},
         "e2e": {"value": value, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -157,6 +171,258 @@ def aggregate(total_ms, e2e_ms, steps, world, device):
     return ms_per_step, ms_per_step / world, float(t[1]) / world
 
 
+# ---- timing helpers ---------------------------------------------------------------------------------------------
+def timed_steps(step_fn, n, stream, prepare=None, after=None):
+    """Runs step_fn(i) for i < n on `stream`, each bracketed by its own pair of CUDA events; prepare(i) (e.g. drawing a
+    fresh gradient on the device) runs before the start event, after(i) (e.g. reading counters back) after the end event.
+    Returns the per-step times in ms."""
+    import torch
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for i in range(n):
+        if prepare is not None:
+            prepare(i)
+        ev[i][0].record(stream)
+        step_fn(i)
+        ev[i][1].record(stream)
+        if after is not None:
+            after(i)
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def pass_width(s):
+    """Residual rows of a full-width screening pass for sparsity s (both recoveries)."""
+    return 2 * min(128, (min(s, 128) + 15) // 16 * 16)
+
+
+class SingleMatrix:
+    """One state with a device gradient that is redrawn before every step (support fixed, drifting or redrawn)."""
+
+    def __init__(self, binding, d, k, s, seed, cfg_id, matrix_id=0, drift=0):
+        import torch
+        hp = inputs.ADAM
+        self.torch, self.d, self.k, self.s, self.drift = torch, d, k, s, drift
+        self.st = binding.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+        supp, sign = inputs.planted_support(d, s, inputs.support_seed(cfg_id, matrix_id))
+        self.supp = torch.from_numpy(supp.astype(np.int64)).cuda()
+        self.sign = torch.from_numpy(sign).cuda()
+        self.grad = torch.empty(d, dtype=torch.float32, device="cuda")
+        self.weight = torch.from_numpy(inputs.weights(d, 99 + matrix_id)).cuda()
+        self.seed0 = inputs.step_seed(cfg_id, matrix_id, 0)
+        self.gen = torch.Generator(device="cuda").manual_seed(self.seed0 + 17)
+        self.n = 0
+        self.stats = []
+
+    def prepare(self, i=None):
+        torch = self.torch
+        self.n += 1
+        if self.drift:                              # `drift` of the s planted positions move every step (s = all of them)
+            where = torch.randperm(self.s, device="cuda", generator=self.gen)[:self.drift]
+            self.supp[where] = torch.randint(0, self.d, (self.drift,), device="cuda", generator=self.gen)
+        inputs.gradient_on_device(self.grad, self.supp, self.sign, self.seed0 + self.n)
+
+    def step(self, i=None):
+        self.st.step(self.grad, self.weight)
+
+    def after(self, i=None):
+        self.stats.append((int(self.st.get("rounds")), int(self.st.get("list_rounds")), int(self.st.get("pass_rows")),
+                           int(self.st.get("fallback"))))
+
+    def run(self, warmup, steps):
+        stream = self.torch.cuda.current_stream()
+        for _ in range(warmup):
+            self.prepare()
+            self.step()
+        self.stats = []
+        ms = timed_steps(self.step, steps, stream, self.prepare, self.after)
+        out = spread(ms)
+        out.update(passes_summary(self.stats, self.k, self.d, ms))
+        return out
+
+    def close(self):
+        self.st.close()
+
+
+def passes_summary(stats, k, d, ms, pk=None):
+    """stats: per step (full passes, list passes, residual rows screened by the full passes, lock-step flag)."""
+    pk = pk or peaks()
+    flops = [2.0 * k * d * rows for _, _, rows, _ in stats]
+    frac = [f / (t * 1e-3) / 1e12 / pk["bf16_tflops"] for f, t in zip(flops, ms)]
+    return dict(full_passes_per_step=[r for r, _, _, _ in stats], list_passes_per_step=[l for _, l, _, _ in stats],
+                lockstep_steps=int(sum(fb for _, _, _, fb in stats)),
+                roofline_frac=float(np.median(frac)),
+                roofline_note="2*k*d*(residual rows screened) flops of the step's screening passes / WHOLE step time / measured "
+                              "bf16 peak (%s)" % pk["source"])
+
+
+def config_drift(binding, args):
+    """The headline shape with supports that move: 2 of the 64 planted positions re-drawn per step (bounded drift, as
+    Section 3.3 assumes), and all 64 re-drawn every step (no stationarity at all)."""
+    wl = WORKLOADS["c2_4096x4096"]
+    out = {}
+    for name, drift in (("drift_2_of_64", 2), ("redrawn_support", wl["s"])):
+        m = SingleMatrix(binding, wl["d"], wl["k"], wl["s"], wl["seed"], 2, matrix_id=1, drift=drift)
+        out[name] = m.run(4, 8)
+        m.close()
+    return out
+
+
+def config_c5(binding, args):
+    out = {}
+    rows, cols = inputs.C5_SHAPE
+    for (k, s) in inputs.C5_PAIRS:
+        m = SingleMatrix(binding, rows * cols, k, s, 1, 5)
+        out["c5_k%d_s%d" % (k, s)] = m.run(3, 5)
+        m.close()
+    return out
+
+
+class Layers:
+    """n_layers transformer layers of seven projections each; same-shape matrices share A and step as one group."""
+
+    def __init__(self, binding, cfg, cfg_id, n_layers):
+        import torch
+        hp = inputs.ADAM
+        self.torch, self.binding = torch, binding
+        self.k, self.s = cfg["k"], cfg["s"]
+        shapes = cfg["shapes"][:7] * n_layers
+        self.dims = [r * c for r, c in shapes]
+        self.kinds = [("qkvo", "qkvo", "qkvo", "qkvo", "gate_up", "gate_up", "down")[i % 7] for i in range(len(shapes))]
+        self.states, self.grads, self.weights, self.supp = [], [], [], []
+        for i, d in enumerate(self.dims):
+            self.states.append(binding.Sgc(d, self.k, self.s, cfg["seed"], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"]))
+            sp, sg = inputs.planted_support(d, self.s, inputs.support_seed(cfg_id, i))
+            self.supp.append((torch.from_numpy(sp.astype(np.int64)).cuda(), torch.from_numpy(sg).cuda()))
+            self.grads.append(torch.empty(d, dtype=torch.float32, device="cuda"))
+            self.weights.append(torch.randn(d, device="cuda") * 0.02)
+        self.groups = [[i for i, kd in enumerate(self.kinds) if kd == name] for name in ("qkvo", "gate_up", "down")]
+        self.cfg_id, self.n, self.stats = cfg_id, 0, []
+
+    def prepare(self, i=None):
+        self.n += 1
+        for m, g in enumerate(self.grads):
+            inputs.gradient_on_device(g, self.supp[m][0], self.supp[m][1], inputs.step_seed(self.cfg_id, m, self.n))
+
+    def step(self, i=None):
+        for grp in self.groups:
+            if len(grp) == 1:
+                self.states[grp[0]].step(self.grads[grp[0]], self.weights[grp[0]])
+            else:
+                self.binding.step_group([self.states[m] for m in grp], [self.grads[m] for m in grp],
+                                        [self.weights[m] for m in grp])
+
+    def after(self, i=None):
+        # passes are booked on the state that leads each batch; summing over all states counts each pass once
+        self.stats.append(tuple(int(sum(int(st.get(name)) for st in self.states)) for name in ("rounds", "list_rounds"))
+                          + (int(sum(int(st.get("fallback")) for st in self.states)),))
+
+    def run(self, warmup, steps):
+        stream = self.torch.cuda.current_stream()
+        for _ in range(warmup):
+            self.prepare()
+            self.step()
+        self.stats = []
+        ms = timed_steps(self.step, steps, stream, self.prepare, self.after)
+        out = spread(ms)
+        out.update(matrices=len(self.dims), params=int(sum(self.dims)), ms_per_matrix_median=out["ms_median"] / len(self.dims),
+                   full_passes_per_step=[a for a, _, _ in self.stats], list_passes_per_step=[b for _, b, _ in self.stats],
+                   lockstep_states=[c for _, _, c in self.stats], k=self.k, s=self.s,
+                   groups={"qkvo": len(self.groups[0]), "gate_up": len(self.groups[1]), "down": len(self.groups[2])})
+        return out
+
+    def close(self):
+        for st in self.states:
+            st.close()
+        self.states, self.grads, self.weights = [], [], []
+        self.torch.cuda.empty_cache()
+
+
+def config_c3(binding, args):
+    L = Layers(binding, inputs.CONFIGS["c3_llama7b_layer"], 3, 1)
+    out = L.run(3, 5)
+    L.close()
+    return {"c3_llama7b_layer": out}
+
+
+def config_c4(binding, args):
+    """The whole 32-layer stack (224 matrices, 6.5e9 parameters): one optimizer step for the model on one GPU.  When the
+    stack does not fit beside what else is on the device, two layers are timed and the figure scaled, labelled so."""
+    import torch
+    cfg = inputs.CONFIGS["c4_llama7b_32layers"]
+    for n_layers in (32, 2):
+        try:
+            L = Layers(binding, cfg, 4, n_layers)
+        except (binding.SgcError, torch.OutOfMemoryError, RuntimeError) as e:      # not enough memory: the smaller stack
+            err = str(e).splitlines()[0][:120]
+            import gc
+            gc.collect()
+            torch.cuda.empty_cache()
+            continue
+        out = L.run(3, 3)
+        L.close()
+        if n_layers < 32:
+            out["extrapolated"] = "measured on %d layers, ms figures multiplied by %d (%s)" % (n_layers, 32 // n_layers, err)
+            for key in ("ms_median", "ms_min", "ms_p90", "ms_mean"):
+                out[key] *= 32 // n_layers
+        return {"c4_llama7b_32layers": out}
+    return {"c4_llama7b_32layers": {"unavailable": err}}
+
+
+def config_mesgc(binding, args):
+    """The paper's chunked variants (Section 4.4) on one 4096 x 4096 gradient: MESGC at the paper's setting (256 chunks,
+    one kept entry, eight rows of A per chunk) and at two corners of its chunk study, CESGC at rank 32 with 64 chunks."""
+    import torch
+    hp = inputs.ADAM
+    d = 4096 * 4096
+    out = {}
+    grad = torch.empty(d, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    for (c, k, sc) in ((256, 8, 1), (1024, 28, 4), (256, 112, 16)):
+        me = binding.Mesgc(d, c, k, sc, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0)
+        sp, sg = inputs.planted_support(d, c * sc, 100 + c)
+        sp, sg = torch.from_numpy(sp.astype(np.int64)).cuda(), torch.from_numpy(sg).cuda()
+        w = torch.randn(d, device="cuda") * 0.02
+        count = [0]
+
+        def prepare(i=None):
+            count[0] += 1
+            inputs.gradient_on_device(grad, sp, sg, 7000 + count[0])
+
+        for _ in range(3):
+            prepare()
+            me.step(grad, w)
+        res = spread(timed_steps(lambda i: me.step(grad, w), 10, stream, prepare))
+        res.update(chunks=c, k_c=k, s_c=sc, launches=me.chunks[0].last_launches(),
+                   gradient_GBps=4.0 * d / res["ms_median"] / 1e6)
+        out["mesgc_c%d_k%d_s%d" % (c, k, sc)] = res
+        me.close()
+    m = n = 4096
+    r, c, k, sc = 32, 64, 217, 31
+    ce = binding.Cesgc(m, n, r, c, k, sc, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], alpha=2.0)
+    q, _ = torch.linalg.qr(torch.randn(m, r, device="cuda"))                   # any orthonormal B serves the timing
+    ce.set_projection(q.t().contiguous())
+    w = torch.zeros(m, n, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    g2 = grad.view(m, n)
+
+    def prepare_ce(i=None):
+        torch.randn(m, n, device="cuda", generator=gen, out=g2)
+        g2.mul_(1e-3)
+
+    for _ in range(3):
+        prepare_ce()
+        ce.step(g2, w)
+    res = spread(timed_steps(lambda i: ce.step(g2, w), 10, stream, prepare_ce))
+    res.update(rank=r, chunks=c, k_c=k, s_c=sc, gradient_GBps=4.0 * d / res["ms_median"] / 1e6)
+    out["cesgc_r32_c64_k217_s31"] = res
+    ce.close()
+    return out
+
+
+CONFIG_RUNNERS = {"drift": config_drift, "c3_llama7b_layer": config_c3, "c5_sweep": config_c5, "mesgc": config_mesgc,
+                  "c4_llama7b_32layers": config_c4}
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -170,12 +436,18 @@ def run_ours(args, wl):
     binding.lib()
     d, k, s = wl["d"], wl["k"], wl["s"]
     hp = inputs.ADAM
-    ring = 4 if d * 4 * 4 > 200e6 else max(4, int(300e6 // (d * 4)) + 1)
-    ring = min(ring, 64)
+    # one buffer per step: warm-up, timed, and the instrumented repeat share nothing with their neighbours in time
+    n_bufs = args.warmup + args.steps
+    if n_bufs * d * 4 > 40e9:
+        n_bufs = max(8, int(40e9 // (d * 4)))
     supp, sign = inputs.planted_support(d, s, inputs.support_seed(wl["cfg_id"], rank))
-    host_grads = [torch.from_numpy(inputs.gradient(d, wl["kind"], supp, sign, inputs.step_seed(wl["cfg_id"], rank, i + 1)))
-                  .pin_memory() for i in range(ring)]
-    dev_grads = [g.cuda() for g in host_grads]
+    e2e_steps = max(1, min(args.steps, 10))
+    host_grads, dev_grads = [], []
+    for i in range(n_bufs):
+        g = torch.from_numpy(inputs.gradient(d, wl["kind"], supp, sign, inputs.step_seed(wl["cfg_id"], rank, i + 1)))
+        dev_grads.append(g.cuda())
+        if i < e2e_steps:
+            host_grads.append(g.pin_memory())
     weight = torch.from_numpy(inputs.weights(d, 99 + rank)).cuda()
     st = binding.Sgc(d, k, s, wl["seed"], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
     st.set_mode(args.mode)
@@ -186,33 +458,36 @@ def run_ours(args, wl):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing (value) ---------------------------------------------------------------
-    for i in range(args.warmup):
-        st.step(dev_grads[i % ring], weight, stream)
+    # ---- warm-up; its first three steps are the cold start of a fresh state ---------------------------------------
+    cold_rounds = []
+    cold = timed_steps(lambda i: st.step(dev_grads[i % n_bufs], weight, stream), args.warmup, stream,
+                       after=lambda i: cold_rounds.append(int(st.get("rounds"))))
+    # ---- device-resident timing (value): K steps between two events, profiling off --------------------------------
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    st.set_profile(True)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    e0.record(stream)
     launches = 0
+    marks[0].record(stream)
     for i in range(args.steps):
-        st.step(dev_grads[(args.warmup + i) % ring], weight, stream)
+        st.step(dev_grads[(args.warmup + i) % n_bufs], weight, stream)
+        marks[i + 1].record(stream)
         launches += st.last_launches()
-    e1.record(stream)
     barrier()
-    total_ms = e0.elapsed_time(e1)
+    total_ms = marks[0].elapsed_time(marks[-1])
+    per_step = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
     clocks = sampler.stop()
     status = int(st.get("status"))
-    st.set_profile(False)
-    # per-kernel times and the number of screening passes that did work, from a second, instrumented run of the
-    # same steps (event pairs around every launch and a read-back of the round counter perturb the step time)
+    # ---- per-kernel times and pass counts from a second, instrumented run on the same gradients (event pairs around
+    # every launch and read-backs of the counters perturb the step time, so none of it is part of `value`) --------------
     st.set_profile(True)
-    rounds = []
-    for i in range(args.steps):
-        st.step(dev_grads[(args.warmup + i) % ring], weight, stream)
+    rounds, rows = [], []
+    n_inst = min(args.steps, 10)
+    for i in range(n_inst):
+        st.step(dev_grads[(args.warmup + i) % n_bufs], weight, stream)
         rounds.append(int(st.get("rounds")))
+        rows.append(int(st.get("pass_rows")))
     prof = st.get_profile()
     st.set_profile(False)
     lockstep = int(st.get("fallback"))
@@ -225,12 +500,11 @@ def run_ours(args, wl):
     copied = [torch.cuda.Event(), torch.cuda.Event()]
     consumed = [torch.cuda.Event(), torch.cuda.Event()]
     out_idx = np.empty(s, dtype=np.uint32)
-    e2e_steps = max(1, min(args.steps, 10))
 
     def upload(i):
         with torch.cuda.stream(copy_stream):
             copy_stream.wait_event(consumed[i % 2])            # the step that last read this buffer has finished
-            stages[i % 2].copy_(host_grads[i % ring], non_blocking=True)
+            stages[i % 2].copy_(host_grads[i % len(host_grads)], non_blocking=True)
             copied[i % 2].record(copy_stream)
 
     barrier()
@@ -256,30 +530,33 @@ def run_ours(args, wl):
 
     if rank == 0:
         pk = peaks()
-        n_pass = 2 * min(128, (min(s, 128) + 15) // 16 * 16)     # residuals per screening pass (both recoveries)
+        n_pass = pass_width(s)
         pass_ms, _ = prof["pass"]
-        working = max(sum(rounds), 1)
         if sum(rounds) > 0:
             # dominant kernel: the tensor-core screening pass, C = A^T R with A generated on the fly
-            pass_avg_s = pass_ms / working * 1e-3
-            achieved = 2.0 * k * d * n_pass / pass_avg_s / 1e12
+            pass_avg_s = pass_ms / sum(rounds) * 1e-3
+            n_avg = sum(rows) / sum(rounds)                       # residual rows per pass (narrower once a recovery is complete)
+            achieved = 2.0 * k * d * n_avg / pass_avg_s / 1e12
             roof = {"kernel": "k_pass", "bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
                     "frac": achieved / pk["bf16_tflops"], "traffic": 2.0 * d + 0.56e6, "peak_source": pk["source"],
                     "traffic_note": "DRAM bytes per launch: 2 bytes per column of the 1/norm table plus R^T (0.56 MB); ncu "
-                                    "measured 4.75 MB at d = 2^21 (profiles/k_pass_small_2M_k2048_s64.md), scaled by d",
-                    "note": "2*k*d*N flops per pass (N = %d residuals, f16 x f16 -> fp32 on tcgen05); the operand A is "
-                            "regenerated by the CUDA cores (k*d entries per pass), which is what limits the pass" % n_pass,
+                                    "measured 4.75 MB at d = 2^21 on the small_2M_k2048_s64 workload, scaled by d",
+                    "note": "2*k*d*N flops per pass (N = %.0f residual rows on average, full width %d; f16 x f16 -> fp32 on "
+                            "tcgen05); the operand A is regenerated by the CUDA cores (k*d entries per pass), which is what "
+                            "limits the pass" % (n_avg, n_pass),
                     "avg_launch_ms": pass_avg_s * 1e3, "launches": sum(rounds),
                     "generated_entries_per_s": k * d / pass_avg_s}
         else:
             omp_ms, omp_n = prof["omp"]
-            it_s = omp_ms / max(args.steps * s, 1) * 1e-3
+            it_s = omp_ms / max(n_inst * s, 1) * 1e-3
             alu_peak = 148 * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
             achieved = 2.0 * k * d * 2 / it_s / 1e12
             roof = {"kernel": "k_omp (lock-step)", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
                     "frac": achieved / alu_peak, "traffic": None,
                     "note": "useful fp32 FMA flops 2*k*d*2 per OMP iteration; peak = 148 SM * 128 lanes * 2 * sm_max_mhz",
                     "avg_launch_ms": it_s * 1e3, "launches": omp_n}
+        sel_ms = sum(prof[name][0] for name in ("select_sample", "select_filter", "select_pick")) / n_inst
+        sel_gbs = 4.0 * d / (sel_ms * 1e-3) / 1e9
         filt_ms, filt_n = prof["select_filter"]
         filt_gbs = 4.0 * d / (filt_ms / max(filt_n, 1) * 1e-3) / 1e9
         line = {
@@ -287,28 +564,48 @@ def run_ours(args, wl):
             "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "d": d, "k": k, "s": s, "seed_A": wl["seed"],
-                       "l2": "%d rotating gradients of %.0f MiB (> 126 MB L2)" % (ring, d * 4 / 2 ** 20),
+                       "l2": "a fresh gradient buffer of %.0f MiB for every step (%d buffers): no input is ever found in L2"
+                             % (d * 4 / 2 ** 20, n_bufs),
                        "replicas": world, "status_word": status, "recovery": "lock-step" if lockstep else "speculative",
                        "screening_passes_per_step": rounds},
+            "per_step": spread(per_step),
+            "cold_start_ms": [round(v, 3) for v in cold[:3]], "cold_start_passes": cold_rounds[:3],
             "roofline": roof,
-            "roofline_select": {"kernel": "k_filter", "bound": "hbm", "achieved": filt_gbs, "peak": pk["hbm_gbs"],
-                                "unit": "GB/s", "frac": filt_gbs / pk["hbm_gbs"], "peak_source": pk["source"],
-                                "avg_launch_ms": filt_ms / max(filt_n, 1)},
-            "phases_ms_per_step": {kname: v[0] / args.steps for kname, v in prof.items()},
+            "roofline_select": {"kernel": "a1: k_sample + k_filter + k_pick", "bound": "hbm", "achieved": sel_gbs,
+                                "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": sel_gbs / pk["hbm_gbs"],
+                                "peak_source": pk["source"], "avg_ms": sel_ms,
+                                "note": "4*d bytes (one read of the gradient) over the time of all launches of the selection",
+                                "filter_alone_gbs": filt_gbs, "filter_alone_frac": filt_gbs / pk["hbm_gbs"]},
+            "phases_ms_per_step": {kname: v[0] / n_inst for kname, v in prof.items()},
             "e2e": {"value": e2e_value, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": launches, "clocks": clocks,
         }
         if world == 1 and not args.no_cpu_baseline:
-            g = host_grads[0].numpy()
-            d_cols, iters = min(d, 1 << 21), min(s, 8)
-            ms, spent, threads = oracle_sample(wl, g, d_cols, iters)
-            line["cpu_baseline"] = {"value": ms, "unit": "ms", "cores": threads, "kind": "oracle",
-                                    "sample": "a1-a3 in full; a4 = %d of %d OMP iterations of 1 of 2 residuals on %d of %d "
-                                              "columns (%.1f s measured), scaled linearly in columns*iterations*residuals"
-                                              % (iters, s, d_cols, d, spent)}
-        print(json.dumps(line))
+            runs = [oracle_sample(wl, host_grads[i].numpy()) for i in range(min(3, len(host_grads)))]
+            line["cpu_baseline"] = {"value": float(np.mean([r[0] for r in runs])), "unit": "ms", "cores": runs[0][2],
+                                    "kind": "oracle", "sample": "mean over %d steps, each: %s" % (len(runs), runs[0][3])}
     st.close()
+    del dev_grads, host_grads, stages
+    torch.cuda.empty_cache()
+    if rank == 0:
+        if world == 1 and args.configs != "none":
+            wanted = EXTRA_CONFIGS if args.configs == "all" else tuple(args.configs.split(","))
+            configs = {args.workload: dict(spread(per_step), full_passes_per_step=rounds, roofline_frac=line["roofline"]["frac"])}
+            for name in wanted:
+                t0 = time.perf_counter()
+                try:
+                    res = CONFIG_RUNNERS[name](binding, args)
+                except Exception as e:                               # a failed extra configuration must not cost the headline
+                    res = {name: {"error": "%s: %s" % (type(e).__name__, str(e).splitlines()[0][:200])}}
+                    torch.cuda.empty_cache()
+                for key, val in res.items():
+                    val["wall_s"] = round(time.perf_counter() - t0, 1)
+                    configs[key] = val
+            line["configs"] = configs
+            if "redrawn_support" in configs and "ms_median" in configs["redrawn_support"]:
+                line["redrawn_support_ms"] = configs["redrawn_support"]["ms_median"]
+        print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
@@ -320,10 +617,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_4096x4096", choices=sorted(WORKLOADS))
+    ap.add_argument("--configs", default="all", help="extra configurations at N = 1: all, none, or a comma-separated "
+                    "subset of " + ",".join(EXTRA_CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--mode", type=int, default=0, choices=[0, 1, 2], help="recovery: 0 auto, 1 lock-step, 2 speculative")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.workload != "c2_4096x4096" and args.configs == "all":
+        args.configs = "none"                  # the extra configurations accompany the headline workload only
     wl = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)

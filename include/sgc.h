@@ -96,6 +96,8 @@ enum {
     SGC_GET_FALLBACK = 22,  /* int32      1 when the last step finished (or ran entirely) in lock-step  */
     SGC_GET_N_CAND = 23,    /* int32      length of the candidate list kept for the next step           */
     SGC_GET_LIST_ROUNDS = 25, /* int32     list passes (screening passes over the wide lists only) that the last step resolved */
+    SGC_GET_PASS_ROWS = 26, /* int32       residual rows screened by the passes over all d columns of the last step, summed over
+                               those passes (a state stepped alone; 2 k d flops of contraction per row)       */
     SGC_GET_ROUND_TRACE = 24 /* int32[24][3] per screening pass of the last step: picks of M^ confirmed so far, picks of V^ confirmed so
                                 far, length of the candidate list after it (rows past SGC_GET_ROUNDS are zero)               */
 };

@@ -25,7 +25,8 @@ RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, 
                status=(14, np.uint32, None), mismatch=(15, np.int32, None), negv=(16, np.int32, None),
                doneM=(17, np.int32, None), doneV=(18, np.int32, None), rnormM=(19, np.float64, "s"),
                rnormV=(20, np.float64, "s"), rounds=(21, np.int32, None), fallback=(22, np.int32, None),
-               n_cand=(23, np.int32, None), round_trace=(24, np.int32, 72), list_rounds=(25, np.int32, None))
+               n_cand=(23, np.int32, None), round_trace=(24, np.int32, 72), list_rounds=(25, np.int32, None),
+               pass_rows=(26, np.int32, None))
 
 MODE_AUTO, MODE_LOCKSTEP, MODE_SPECULATIVE = 0, 1, 2
 
@@ -290,7 +291,8 @@ class Mesgc:
 
 class Cesgc:
     """Compute-efficient SGC (Section 4.4): SGC, chunked, on the projected gradient B G of an m x n matrix; the update
-    returns through B^T (sgc_cesgc_step).  B (r x m, float32, CUDA) is the caller's: set_projection() stores it."""
+    returns through B^T (sgc_cesgc_step).  B (r x m, float32, CUDA, orthonormal rows: the paper takes the leading left-singular
+    vectors of a gradient and renews them every fixed number of iterations) is the caller's: set_projection() stores it."""
 
     def __init__(self, m, n, r, c, k, s_c, seed, lr, beta1, beta2, eps, alpha=None):
         import torch
@@ -305,14 +307,6 @@ class Cesgc:
         if B.shape != (self.r, self.m) or not B.is_cuda or not B.is_contiguous() or B.element_size() != 4:
             raise TypeError("B must be a contiguous float32 CUDA tensor of shape (r, m)")
         self.B = B
-
-    def refresh_projection(self, grad):
-        """B <- the first r left-singular vectors of grad (m x n), transposed: what the paper renews every fixed number
-        of iterations.  The SVD is torch's (a library routine outside the per-step path)."""
-        import torch
-        U, _, _ = torch.linalg.svd(grad.reshape(self.m, self.n).float(), full_matrices=False)
-        Q, _ = torch.linalg.qr(U[:, :self.r].double())          # fp32 singular vectors are orthonormal to ~1e-4 only
-        self.set_projection(Q.t().float().contiguous())
 
     def step(self, grad, weight, stream=None):
         if self.B is None:

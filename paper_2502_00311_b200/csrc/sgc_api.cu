@@ -346,6 +346,7 @@ SGC_API int sgc_get(sgc_state* st, int32_t what, void* dst, size_t bytes) {
         case SGC_GET_FALLBACK: src = &st->ctl->fallback; n = 4; break;
         case SGC_GET_N_CAND: src = &st->ctl->n_cand; n = 4; break;
         case SGC_GET_LIST_ROUNDS: src = &st->ctl->list_rounds; n = 4; break;
+        case SGC_GET_PASS_ROWS: src = &st->ctl->pass_rows; n = 4; break;
         case SGC_GET_ROUND_TRACE: src = &st->ctl->trace[0][0]; n = 4 * 3 * sgc::kMaxRounds; break;
         default: return SGC_ERR_WHAT;
     }

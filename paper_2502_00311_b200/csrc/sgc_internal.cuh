@@ -28,8 +28,6 @@ constexpr uint32_t kGolden = 0x9E3779B9u;
 constexpr uint32_t kMulEntry = 0x85EBCA6Bu;
 constexpr uint32_t kStrideSalt = 0x5BD1E995u;
 constexpr uint32_t kC0x2 = 0x40c240c2u, kC1x2 = 0xbad9bad9u, kC2x2 = 0x3f893f89u;   // C0, C1, C2 in both halves
-constexpr uint32_t kInv256x2 = 0x1c001c00u;          // 2^-8
-constexpr uint32_t kCentrex2 = 0xc4ffc4ffu;          // -(1024 + 255)/256
 
 __host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
     x ^= x >> 16; x *= 0x7feb352du;
@@ -58,15 +56,22 @@ __device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
     return d;
 }
 
+__device__ __forceinline__ uint32_t hsub2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
 // h0 = ck + p*mk (the caller advances it by mk per row pair).  Returns Z of rows 2p (low half) and 2p+1 (high
 // half) as two binary16 bit patterns.
 __device__ __forceinline__ uint32_t z_pair_from_word(uint32_t h0) {
     uint32_t h = h0;
-    h ^= h >> 16; h *= kMulEntry; h ^= h >> 15;
-    // byte pair sums straight into the significand of the half 1024: the halves 1024 + S (exact, S <= 510)
-    // (bytes 0 and 2) + (bytes 1 and 3) as two 16-bit fields: byte permutes and one add, all on the integer pipe
-    const uint32_t s2 = __byte_perm(h, 0u, 0x4240) + __byte_perm(h, 0u, 0x4341) + 0x64006400u;
-    const uint32_t x = hfma2(s2, kInv256x2, kCentrex2);        // (S - 255)/256, exact
+    h ^= h >> 16; h *= kMulEntry;
+    // x = (b0 + b1 - 255)/256 (even row; b2, b3 for the odd row) as a difference of two halves that are planted by byte
+    // permutes alone: the half 0x4400 | b is 4 + b/256, so (4 + b0/256) - (4 + (255 - b1)/256) = x, exactly.  The
+    // complement of bytes 1 and 3 rides along in the three-input logic operation of the last mixing step.
+    h = h ^ (h >> 15) ^ 0xFF00FF00u;
+    const uint32_t x = hsub2(__byte_perm(h, 0x44444444u, 0x4240), __byte_perm(h, 0x44444444u, 0x4341));
     const uint32_t w = hmul2(x, x);
     uint32_t q = hfma2(w, kC2x2, kC1x2);
     q = hfma2(q, w, kC0x2);
@@ -180,6 +185,7 @@ struct SpecCtl {
     int mini_done;          // 1: list passes rest until the next full pass
     int list_rounds;        // list passes of the last step that were resolved
     int list_refuted;       // picks that those list passes refuted
+    int pass_rows;          // residual rows that the full passes of the last step screened, summed over the passes
     int hist_count, hist_next;  // ring of the kept index sets of the last steps: valid slots, slot of the next step
     int trace[kMaxRounds][3];   // per round: confirmed picks of both streams and the list length after it
     double ynorm[2];        // ||y|| per residual

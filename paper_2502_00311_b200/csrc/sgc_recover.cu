@@ -1191,7 +1191,11 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
     if (threadIdx.x == 0) {
         give_up = 0; any_failed = 0;
         if (mini) ctl->list_rounds = ctl->list_rounds + 1;
-        else ctl->rounds = ctl->rounds + 1;
+        else {
+            ctl->rounds = ctl->rounds + 1;
+            // width of the pass whose reports are being resolved (ctl->narrow still names it)
+            ctl->pass_rows = ctl->pass_rows + (ctl->narrow ? ((a.half_n + 31) / 32) * 32 : 2 * a.half_n);
+        }
     }
     for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = 0;
     __syncthreads();
@@ -1360,7 +1364,7 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau, int sh
         ctl->finished[1] = shared ? 1 : 0;          // shared support: the second stream makes no picks of its own
         ctl->narrow = shared ? 1 : 0;
         ctl->stop[0] = ctl->stop[1] = 0;
-        ctl->rounds = 0; ctl->pass_error = 0;
+        ctl->rounds = 0; ctl->pass_error = 0; ctl->pass_rows = 0;
         for (int r = 0; r < kMaxRounds; ++r) ctl->trace[r][0] = ctl->trace[r][1] = ctl->trace[r][2] = 0;
         ctl->gram_ok = 1;
         if (ctl->list_version == 0) ctl->list_version = 1;      // a fresh state: no Gram matrix yet
@@ -1720,7 +1724,7 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
                     const bool two_widths = st->pass_n_half < st->pass_n;       // the width that ctl->narrow names runs
                     e = launch_pass(st->tmap[0], st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale,
                                     st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp,
-                                    two_widths ? &st->ctl->narrow : nullptr, 0);
+                                    two_widths ? &st->ctl->narrow : nullptr, 0, st->wait_limit_ns);
                     if (two_widths && e == cudaSuccess) {
                         e = launch_pass(st->tmap_half, st->seed, (uint64_t)st->d, st->k, st->pass_n_half, st->tau,
                                         st->inv_scale, st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors,

@@ -76,3 +76,22 @@ def support_seed(cfg_id, matrix_id):
 
 def step_seed(cfg_id, matrix_id, step):
     return 1_000_000 * cfg_id + 1000 * matrix_id + step
+
+
+def gradient_on_device(out, support, sign, seed, chunk=1 << 24):
+    """Fills the float32 CUDA tensor `out` with a "student" gradient drawn on the device (torch's generator): the same law
+    as gradient(kind="student") -- 1e-3 * Student-t(3) noise, planted entries sign * U(0.5, 1) at `support` (CUDA int64
+    tensor) -- but not the same numbers.  For workloads too large to draw on the host (the whole-model configurations);
+    nothing that is compared with the oracle uses it."""
+    import torch
+    gen = torch.Generator(device=out.device)
+    gen.manual_seed(int(seed))
+    d = out.numel()
+    for lo in range(0, d, chunk):
+        n = min(chunk, d - lo)
+        z = torch.randn(4, n, device=out.device, generator=gen)
+        chi = (z[1] * z[1] + z[2] * z[2] + z[3] * z[3]) * (1.0 / 3.0)          # chi^2_3 / 3
+        out[lo:lo + n] = z[0] * torch.rsqrt(chi) * 1e-3
+    mag = torch.rand(support.numel(), device=out.device, generator=gen) * 0.5 + 0.5
+    out[support] = sign * mag
+    return out

@@ -629,20 +629,6 @@ def test_cesgc_step_matches_its_oracle(sgc, m, n, r, c, k, sc):
         rf.close()
 
 
-def test_cesgc_refresh_projection_spans_the_leading_singular_vectors(sgc):
-    import torch
-    m, n, r = 300, 200, 5
-    rng = np.random.default_rng(4)
-    G = (rng.standard_normal((m, r)) * np.array([9.0, 7.0, 5.0, 3.0, 2.0])) @ rng.standard_normal((r, n)) + 0.01 * rng.standard_normal((m, n))
-    ce = sgc.Cesgc(m, n, r, 2, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
-    ce.refresh_projection(cuda(G.astype(np.float32)))
-    B = ce.B.cpu().numpy().astype(np.float64)
-    U, _, _ = np.linalg.svd(G, full_matrices=False)
-    np.testing.assert_allclose(B @ B.T, np.eye(r), atol=1e-5)                       # orthonormal rows
-    np.testing.assert_allclose(B.T @ B, U[:, :r] @ U[:, :r].T, atol=1e-3)           # the same subspace (signs are free)
-    ce.close()
-
-
 def test_cesgc_step_rejects_bad_shapes(sgc):
     import torch
     ce = sgc.Cesgc(64, 32, 4, 2, 16, 2, 1, 1e-3, 0.9, 0.999, 1e-8)
