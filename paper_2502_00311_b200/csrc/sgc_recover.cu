@@ -1651,7 +1651,7 @@ cudaError_t finish_recover_setup(sgc_state* st) {
 // Recovery (a4 + a5) of n states that share (d, k, s, seed), hence A.  The states' screened residuals are laid out side by
 // side in the screening buffers of the first state of each batch (a batch = as many states as fit kPassMaxN columns), so
 // one pass over A serves a whole batch; everything else runs per state.  n = 1 is the plain sgc_step.
-cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches) {
+static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches) {
     sgc_state* st0 = sts[0];
     bool speculate = true;
     for (int i = 0; i < n; ++i)
@@ -1823,8 +1823,31 @@ cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, i
     return cudaGetLastError();
 }
 
+// Which states of a group share passes.  One pass serves a batch of states only while it has room for all their residuals
+// (kPassMaxN rows), and the two-level screening -- what keeps the number of passes over all d columns down when the
+// recovery picks columns outside the kept sets -- is a single-state scheme.  So a state goes alone when a batch could hold
+// nothing beside it, or when its last step needed three or more passes over all columns (the same signal that switches
+// its two-level screening on); the others are batched.  The result does not depend on the split.
+cudaError_t launch_recover_group(sgc_state* const* sts, float* const* weights, int n, cudaStream_t stream, int* launches) {
+    if (n == 1) return recover_batches(sts, weights, 1, stream, launches);
+    std::vector<sgc_state*> together;
+    std::vector<float*> together_w;
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < n && e == cudaSuccess; ++i) {
+        sgc_state* st = sts[i];
+        const bool speculates = st->spec_ok && st->spec_ready && (st->mode == 2 || (st->mode == 0 && st->d >= (1ll << 16)));
+        const int last = speculates ? (*reinterpret_cast<volatile int*>(st->h_rounds) & 255) : 0;
+        const bool alone = speculates && (kPassMaxN / st->pass_n < 2 || st->two_level || last >= 3);
+        if (alone) e = recover_batches(&sts[i], &weights[i], 1, stream, launches);
+        else { together.push_back(st); together_w.push_back(weights[i]); }
+    }
+    if (e == cudaSuccess && !together.empty())
+        e = recover_batches(together.data(), together_w.data(), (int)together.size(), stream, launches);
+    return e;
+}
+
 cudaError_t launch_recover(sgc_state* st, float* weight, cudaStream_t stream, int* launches) {
-    return launch_recover_group(&st, &weight, 1, stream, launches);
+    return recover_batches(&st, &weight, 1, stream, launches);
 }
 
 }  // namespace sgc
