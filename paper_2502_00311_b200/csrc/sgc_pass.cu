@@ -43,7 +43,7 @@ struct PassArgs {
     uint32_t seed_lo, seed_hi;
     unsigned long long d;
     int k, n;                    // n: residuals per pass (multiple of 32, <= 256)
-    int stages, bufs;            // pipeline depth; accumulator buffers in tensor memory (2 when n <= 128)
+    int stages, bufs;            // slots of the ring; accumulator buffers in tensor memory (2 when n <= 128)
     unsigned int num_super;      // ceil(d / 256)
     const float* tau;            // [n] thresholds (+inf = unused residual), in the units of the (scaled) rows of R^T
     const float* inv_scale;      // [n] factor that turns a score back into the caller's units, or nullptr for 1
@@ -174,7 +174,9 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 //   tau    float[256], 1 / tau float[256]
 //   mbarriers: full[stages], empty[stages], acc_full[2], acc_empty[2], drain;  tensor-memory base;  abort flag
 // WIDE: the two-level screening code (wide-list harvest, list passes) is compiled in
-template <bool TABLE, bool WIDE>
+// SUB: 64-row chunks of A per slot of the ring, i.e. per hand-off between generators, TMA and MMA issuer (2 when the
+// residual block is narrow enough for two slots of 128 rows: half as many barrier rounds per generated entry)
+template <bool TABLE, bool WIDE, int SUB>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
     if (a.gate[0] != nullptr) {
         bool any = false;
@@ -200,7 +202,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const int stage_bytes = 2 * kTileBytes + a.n * 128;
+    const int sub_bytes = 2 * kTileBytes + a.n * 128;      // one 64-row chunk: two tiles of A and the chunk of R^T
+    const int stage_bytes = SUB * sub_bytes;
     const uint32_t norms_off = (uint32_t)a.stages * stage_bytes;
     float* norms = reinterpret_cast<float*>(gen_base + norms_off);
     float* tau_s = norms + kNormRing * kSuperCols * 2;
@@ -250,10 +253,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             uint32_t st = 0, ph = 0;
             bool ok = true;
             for (unsigned int sweep = blockIdx.x; ok && sweep < num_super; sweep += gridDim.x) {
-                for (int kc = 0; kc < kc_count; ++kc) {
+                for (int kc = 0; kc < kc_count; kc += SUB) {
                     if (!mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 256, a.wait_limit_ns)) { ok = false; break; }
-                    mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u);
-                    tma_load_2d(base + st * stage_bytes + 2 * kTileBytes, &tmap, kc * kChunkRows, 0, bar_full + 8u * st);
+                    mbar_arrive_expect_tx(bar_full + 8u * st, (uint32_t)a.n * 128u * SUB);
+#pragma unroll
+                    for (int u = 0; u < SUB; ++u)
+                        tma_load_2d(base + st * stage_bytes + u * sub_bytes + 2 * kTileBytes, &tmap, (kc + u) * kChunkRows, 0,
+                                    bar_full + 8u * st);
                     if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
                 }
             }
@@ -273,16 +279,19 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                 if (!mbar_wait(bar_acce + 8u * buf, (use & 1u) ^ 1u, abort_flag, 32, a.wait_limit_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t acc0 = tmem_base + buf * acc_cols, acc1 = acc0 + a.n;
-                for (int kc = 0; kc < kc_count; ++kc) {
+                for (int kc = 0; kc < kc_count; kc += SUB) {
                     if (!mbar_wait(bar_full + 8u * st, ph, abort_flag, 0, a.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t lo = desc_lo0 + st * stage_step;
-                    const uint32_t first = kc != 0 ? 1u : 0u;
 #pragma unroll
-                    for (int kk = 0; kk < kChunkRows / 16; ++kk) {
-                        const uint64_t bdesc = desc_hi | (uint64_t)(lo + (2 * kTileBytes >> 4) + 2 * kk);
-                        umma_f16(acc0, desc_hi | (uint64_t)(lo + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
-                        umma_f16(acc1, desc_hi | (uint64_t)(lo + (kTileBytes >> 4) + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                    for (int u = 0; u < SUB; ++u) {
+                        const uint32_t lo = desc_lo0 + st * stage_step + u * ((uint32_t)sub_bytes >> 4);
+                        const uint32_t first = (kc + u) != 0 ? 1u : 0u;
+#pragma unroll
+                        for (int kk = 0; kk < kChunkRows / 16; ++kk) {
+                            const uint64_t bdesc = desc_hi | (uint64_t)(lo + (2 * kTileBytes >> 4) + 2 * kk);
+                            umma_f16(acc0, desc_hi | (uint64_t)(lo + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                            umma_f16(acc1, desc_hi | (uint64_t)(lo + (kTileBytes >> 4) + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                        }
                     }
                     umma_commit(bar_empty + 8u * st);        // frees the stage once these MMAs have read it
                     if (++st == (uint32_t)a.stages) { st = 0; ph ^= 1u; }
@@ -383,9 +392,11 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             float norm = 0.0f;
             uint32_t h = key.ck + (uint32_t)(half * 16) * key.mk;   // one word per row pair
             const uint32_t skip = 16u * key.mk;                  // the other generator thread of this column owns the next 32 rows
-            for (int kc = 0; kc < kc_count; ++kc) {
+            for (int kc = 0; kc < kc_count; kc += SUB) {
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * st, ph ^ 1u, abort_flag, 0, a.wait_limit_ns))) { ok = false; break; }
-                const uint32_t dst = base + st * stage_bytes;
+#pragma unroll
+                for (int u = 0; u < SUB; ++u) {
+                const uint32_t dst = base + st * stage_bytes + u * sub_bytes;
 #pragma unroll
                 for (int c = 0; c < 4; c += 2) {
                     uint32_t w[8];
@@ -404,7 +415,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                     }
                 }
                 h += skip;
-                if (!TABLE && kc == kc_count - 1) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
+                }
+                if (!TABLE && kc + SUB >= kc_count) norms[((size_t)(sweep_i % kNormRing) * kSuperCols + col_local) * 2 + half] = norm;
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_full + 8u * st);
@@ -479,14 +491,16 @@ cudaError_t get_encoder(EncodeTiledFn* out) {
     return cudaSuccess;
 }
 
-size_t pass_smem_bytes(int n, int stages) {
-    return 1024 + (size_t)stages * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 512) +
-           8 * (2 * (size_t)stages + 5) + 16;
+size_t pass_smem_bytes(int n, int slots, int sub) {
+    return 1024 + (size_t)slots * sub * (2 * kTileBytes + (size_t)n * 128) + sizeof(float) * (kNormRing * kSuperCols * 2 + 512) +
+           8 * (2 * (size_t)slots + 5) + 16;
 }
 
 }  // namespace
 
-int pass_stages(int n) { return n <= 128 ? 4 : 3; }
+// 64-row chunks per slot and slots of the ring: four chunks fit beside a residual block of up to 128 rows, three beyond
+int pass_sub(int n, int k) { return (n <= 128 && k % (2 * kChunkRows) == 0) ? 2 : 1; }
+int pass_slots(int n, int k) { return (n <= 128 ? 4 : 3) / pass_sub(n, k); }
 
 cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
     EncodeTiledFn enc = nullptr;
@@ -502,18 +516,26 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+template <bool TABLE, bool WIDE, int SUB>
+cudaError_t pass_opt_in(int need) {
+    return cudaFuncSetAttribute(k_pass<TABLE, WIDE, SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, need);
+}
+
 cudaError_t pass_configure(int) {
     static_assert(sizeof(CUtensorMap) == kTensorMapBytes, "tensor map storage");
     size_t need = 0;                              // one setting that serves every width the kernel is launched with
-    for (int n = 32; n <= kPassMaxN; n += 32) {
-        const size_t b = pass_smem_bytes(n, pass_stages(n));
-        if (b > need) need = b;
-    }
-    cudaError_t e = cudaFuncSetAttribute(k_pass<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_pass<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_pass<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    for (int n = 32; n <= kPassMaxN; n += 32)
+        for (int sub = 1; sub <= 2; ++sub) {
+            const size_t b = pass_smem_bytes(n, (n <= 128 ? 4 : 3) / sub, sub);
+            if ((n <= 128 || sub == 1) && b > need) need = b;
+        }
+    cudaError_t e = pass_opt_in<false, false, 1>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<false, false, 2>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, true, 1>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, true, 2>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, false, 1>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, false, 2>((int)need);
+    return e;
 }
 
 cudaError_t launch_inv_norms(uint64_t seed, uint64_t d, int k, uint16_t* out, cudaStream_t stream) {
@@ -530,7 +552,8 @@ cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int 
     a.sel = sel; a.sel_value = sel_value;
     a.seed_lo = (uint32_t)(seed & 0xFFFFFFFFu); a.seed_hi = (uint32_t)(seed >> 32);
     a.d = d; a.k = k; a.n = n;
-    a.stages = pass_stages(n); a.bufs = n <= 128 ? 2 : 1;
+    const int sub = pass_sub(n, k);
+    a.stages = pass_slots(n, k); a.bufs = n <= 128 ? 2 : 1;
     a.num_super = (unsigned int)((d + kSuperCols - 1) / kSuperCols);
     a.tau = tau; a.inv_scale = inv_scale; a.inv_norm = inv_norm; a.rep_count = rep_count; a.rep = rep; a.rep_cap = rep_cap;
     for (int q = 0; q < kPassMaxBatch; ++q) { a.gate[q] = gates ? gates[q] : nullptr; a.error[q] = errors ? errors[q] : nullptr; }
@@ -545,9 +568,16 @@ cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int 
     if (grid > a.num_super) grid = a.num_super;
     CUtensorMap map;
     memcpy(&map, tmap, sizeof(map));
-    if (inv_norm && wide) k_pass<true, true><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
-    else if (inv_norm) k_pass<true, false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
-    else k_pass<false, false><<<grid, kPassThreads, pass_smem_bytes(n, a.stages), stream>>>(map, a);
+    const size_t smem = pass_smem_bytes(n, a.stages, sub);
+    if (sub == 2) {
+        if (inv_norm && wide) k_pass<true, true, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm) k_pass<true, false, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else k_pass<false, false, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
+    } else {
+        if (inv_norm && wide) k_pass<true, true, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm) k_pass<true, false, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else k_pass<false, false, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
+    }
     return cudaGetLastError();
 }
 
