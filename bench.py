@@ -571,7 +571,7 @@ def run_ours(args, wl):
             "per_step": spread(per_step),
             "cold_start_ms": [round(v, 3) for v in cold[:3]], "cold_start_passes": cold_rounds[:3],
             "roofline": roof,
-            "roofline_select": {"kernel": "a1: k_sample + k_filter + k_pick", "bound": "hbm", "achieved": sel_gbs,
+            "roofline_select": {"kernel": "a1: k_select_fast (one launch: stream with the carried threshold, exact pick in its last block)", "bound": "hbm", "achieved": sel_gbs,
                                 "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": sel_gbs / pk["hbm_gbs"],
                                 "peak_source": pk["source"], "avg_ms": sel_ms,
                                 "note": "4*d bytes (one read of the gradient) over the time of all launches of the selection",

@@ -200,6 +200,8 @@ struct Counters {
     int done[2];                // completed OMP iterations per residual (M^, V^)
     int stopped[2];             // 1 once a residual's OMP has stopped early
     int n_upd, mismatch, negv, pad;
+    unsigned int sel_tau_next;  // threshold carried to the next step's one-kernel selection (0: none yet)
+    unsigned int sel_ticket2;   // blocks of the one-kernel selection that have finished
 };
 
 // Batched chunk path (sgc_chunked.cu): the records of one chunk's state, as the batched kernels address them
@@ -241,6 +243,7 @@ struct sgc_state {
     int device; int sm_count;
     cudaStream_t last_stream; bool has_stream;
     int32_t last_launches; bool stepped;
+    bool sel_warm;              // a top-s threshold from the previous step is on the device (one-kernel selection)
     int corr_grid, corr_smem;
     int mode;                   // 0 auto, 1 lock-step only, 2 speculative whenever k allows it
     int shared_support;         // 1: OMP(M^) alone selects, V^ is fitted on its support (sgc_set_recovery)

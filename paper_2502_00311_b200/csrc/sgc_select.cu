@@ -132,10 +132,10 @@ struct GradSource {
     }
 };
 
-// Returns (in every thread) the s-th largest key of src[0..n).  hist: kDigits words of shared memory.
-template <class Src>
+// Returns (in every thread) the s-th largest key of src[0..n).  hist: kDigits words of shared memory.  NT: threads of the block.
+template <int NT, class Src>
 __device__ unsigned long long block_kth_largest(Src src, unsigned long long n, unsigned int s, unsigned int* hist,
-                                                unsigned int* scan, unsigned long long* bcast) {
+                                                unsigned int* scan, unsigned long long* bcast) {      // bcast: 3 words
     unsigned long long prefix = 0ull, mask = 0ull;
     unsigned int need = s;
     int shift = 64;
@@ -143,93 +143,267 @@ __device__ unsigned long long block_kth_largest(Src src, unsigned long long n, u
         const int bits = shift >= kDigitBits ? kDigitBits : shift;
         shift -= bits;
         const unsigned int dm = (1u << bits) - 1u;
-        for (int b = threadIdx.x; b < kDigits; b += kPickThreads) hist[b] = 0u;
+        for (int b = threadIdx.x; b < kDigits; b += NT) hist[b] = 0u;
         __syncthreads();
-        for (unsigned long long i = threadIdx.x; i < n; i += kPickThreads) {
+        for (unsigned long long i = threadIdx.x; i < n; i += NT) {
             const unsigned long long key = src(i);
             if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & dm], 1u);
         }
         __syncthreads();
-        // scan from the top digit: thread t owns reversed bins 2t, 2t+1
-        const unsigned int r0 = hist[kDigits - 1 - 2 * threadIdx.x], r1 = hist[kDigits - 2 - 2 * threadIdx.x];
-        unsigned int v = r0 + r1;
+        // scan from the top digit: thread t owns the reversed bins B t .. B t + B - 1
+        constexpr int B = kDigits / NT;
+        unsigned int r[B];
+        unsigned int v = 0;
+#pragma unroll
+        for (int u = 0; u < B; ++u) { r[u] = hist[kDigits - 1 - (B * (int)threadIdx.x + u)]; v += r[u]; }
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         unsigned int incl = v;
         for (int o = 1; o < 32; o <<= 1) { const unsigned int t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
         if (lane == 31) scan[warp] = incl;
         __syncthreads();
         if (warp == 0) {
-            unsigned int w = scan[lane], wi = w;
+            unsigned int w = lane < NT / 32 ? scan[lane] : 0u, wi = w;
             for (int o = 1; o < 32; o <<= 1) { const unsigned int t = __shfl_up_sync(0xffffffffu, wi, o); if (lane >= o) wi += t; }
             scan[lane] = wi - w;                            // exclusive offset of each warp
         }
         __syncthreads();
         const unsigned int excl = scan[warp] + incl - v;    // keys in strictly higher bins than mine
         if (excl < need && need <= excl + v) {              // exactly one thread
-            unsigned int digit, used;
-            if (need <= excl + r0) { digit = kDigits - 1 - 2 * threadIdx.x; used = excl; }
-            else { digit = kDigits - 2 - 2 * threadIdx.x; used = excl + r0; }
+            unsigned int used = excl, digit = 0, in_bin = 0;
+#pragma unroll
+            for (int u = 0; u < B; ++u) {
+                if (in_bin == 0u && need <= used + r[u]) { digit = kDigits - 1 - (B * threadIdx.x + u); in_bin = r[u]; }
+                else if (in_bin == 0u) used += r[u];
+            }
             bcast[0] = (unsigned long long)digit;
             bcast[1] = (unsigned long long)(need - used);
+            bcast[2] = (unsigned long long)in_bin;
         }
         __syncthreads();
         prefix |= bcast[0] << shift;
         mask |= (unsigned long long)dm << shift;
         need = (unsigned int)bcast[1];
-        __syncthreads();
+        const bool whole_bin = bcast[2] == bcast[1];        // every key of the boundary bin is wanted: its lowest possible
+        __syncthreads();                                    // key (remaining digits zero) is a valid threshold
+        if (whole_bin) break;
     }
     return prefix;
 }
 
-__global__ void __launch_bounds__(kPickThreads)
-k_pick(const float* __restrict__ grad, unsigned long long d, unsigned int s, const unsigned long long* __restrict__ cand,
-       Counters* __restrict__ cnt, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val) {
-    __shared__ unsigned int hist[kDigits];
-    __shared__ unsigned int scan[32];
-    __shared__ unsigned long long bcast[2];
-    __shared__ uint32_t picked[kMaxS];
-    __shared__ unsigned int n_out;
-    const unsigned int count = cnt->sel_count;
+// shared memory of the exact selection (one block)
+struct PickSmem {
+    unsigned int hist[kDigits];
+    unsigned int scan[32];
+    unsigned long long bcast[3];
+    uint32_t picked[kMaxS];
+    unsigned int n_out;
+};
+
+// The s largest keys among `count` candidates (or, when the candidate list cannot serve -- fewer than s entries or an
+// overflow -- among all d entries of the gradient: slow, exact, flagged), sorted by index, with their values.
+template <int NT>
+__device__ void pick_block(PickSmem& sm, const float* __restrict__ grad, unsigned long long d, unsigned int s,
+                           const unsigned long long* __restrict__ cand, unsigned int count, Counters* __restrict__ cnt,
+                           uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val) {
     const bool use_cand = (count >= s) && (count <= (unsigned int)kSelCap);
-    if (threadIdx.x == 0) n_out = 0u;
-    for (int i = threadIdx.x; i < kMaxS; i += kPickThreads) picked[i] = 0xFFFFFFFFu;
+    if (threadIdx.x == 0) sm.n_out = 0u;
+    for (int i = threadIdx.x; i < kMaxS; i += NT) sm.picked[i] = 0xFFFFFFFFu;
     __syncthreads();
     if (use_cand) {
         CandSource src{cand};
-        const unsigned long long kth = block_kth_largest(src, count, s, hist, scan, bcast);
-        for (unsigned int i = threadIdx.x; i < count; i += kPickThreads) {
+        const unsigned long long kth = block_kth_largest<NT>(src, count, s, sm.hist, sm.scan, sm.bcast);
+        for (unsigned int i = threadIdx.x; i < count; i += NT) {
             const unsigned long long key = cand[i];
-            if (key >= kth) picked[atomicAdd(&n_out, 1u)] = ~(uint32_t)key;
+            if (key >= kth) sm.picked[atomicAdd(&sm.n_out, 1u)] = ~(uint32_t)key;
         }
     } else {
         if (threadIdx.x == 0) atomicOr(&cnt->status, (unsigned int)SGC_STATUS_SELECT_FALLBACK);
         GradSource src{grad};
-        const unsigned long long kth = block_kth_largest(src, d, s, hist, scan, bcast);
-        for (unsigned long long i = threadIdx.x; i < d; i += kPickThreads) {
+        const unsigned long long kth = block_kth_largest<NT>(src, d, s, sm.hist, sm.scan, sm.bcast);
+        for (unsigned long long i = threadIdx.x; i < d; i += NT) {
             const unsigned long long key = src(i);
             if (key >= kth) {
                 if ((key >> 32) >= 0x7F800000ull) atomicOr(&cnt->status, (unsigned int)SGC_STATUS_NONFINITE_INPUT);
-                picked[atomicAdd(&n_out, 1u)] = (uint32_t)i;
+                sm.picked[atomicAdd(&sm.n_out, 1u)] = (uint32_t)i;
             }
         }
     }
     __syncthreads();
-    // ascending index order: bitonic sort of 1024 slots (unused slots hold 0xFFFFFFFF and sink to the end)
-    for (unsigned int size = 2; size <= (unsigned int)kMaxS; size <<= 1) {
+    // ascending index order: bitonic sort of the slots in use, rounded up to a power of two (unused slots hold
+    // 0xFFFFFFFF and sink to the end)
+    unsigned int span = 2;
+    while (span < s) span <<= 1;
+    for (unsigned int size = 2; size <= span; size <<= 1) {
         for (unsigned int stride = size >> 1; stride > 0; stride >>= 1) {
-            const unsigned int i = threadIdx.x, j = i ^ stride;
-            if (j > i) {
-                const uint32_t a = picked[i], b = picked[j];
-                const bool up = ((i & size) == 0);
-                if ((a > b) == up) { picked[i] = b; picked[j] = a; }
+            for (unsigned int i = threadIdx.x; i < span; i += NT) {
+                const unsigned int j = i ^ stride;
+                if (j > i && j < span) {
+                    const uint32_t a = sm.picked[i], b = sm.picked[j];
+                    const bool up = ((i & size) == 0);
+                    if ((a > b) == up) { sm.picked[i] = b; sm.picked[j] = a; }
+                }
             }
             __syncthreads();
         }
     }
-    if (threadIdx.x < s) {
-        const uint32_t idx = picked[threadIdx.x];
-        sel_idx[threadIdx.x] = idx;
-        sel_val[threadIdx.x] = grad[idx];
+    for (unsigned int i = threadIdx.x; i < s; i += NT) {
+        const uint32_t idx = sm.picked[i];
+        sel_idx[i] = idx;
+        sel_val[i] = grad[idx];
+    }
+}
+
+// carry_out: the sampled threshold is left for the next call's one-kernel selection, which appends to an empty list
+__global__ void __launch_bounds__(kPickThreads)
+k_pick(const float* __restrict__ grad, unsigned long long d, unsigned int s, const unsigned long long* __restrict__ cand,
+       Counters* __restrict__ cnt, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, int carry_out) {
+    __shared__ PickSmem sm;
+    pick_block<kPickThreads>(sm, grad, d, s, cand, cnt->sel_count, cnt, sel_idx, sel_val);
+    if (carry_out && threadIdx.x == 0) {
+        cnt->sel_tau_next = cnt->sel_tau;
+        cnt->sel_count = 0u;
+    }
+}
+
+// ---- the one-kernel selection of a warm state ---------------------------------------------------------------
+// Gradients of consecutive steps follow nearly the same law, so the threshold tau that left a few thousand survivors
+// in one step serves the next: one kernel streams the gradient with the carried tau (one read of d floats, the only
+// HBM traffic of a1), counts what lies in the 8 magnitude bins below tau as well (a bin is 1/16 of an octave, so the
+// histogram reaches a factor 1.41 below tau), and the block that finishes last derives the next step's tau from that
+// histogram and makes the exact pick.  A miss (fewer than s survivors, or more than the list holds: the law moved by
+// a factor of several from one step to the next) is served by the same block with the exact selection over the whole
+// gradient -- milliseconds instead of microseconds, flagged SGC_STATUS_SELECT_FALLBACK -- which also yields the next tau.
+// The first step of a state has no tau and takes the sampled path (k_sample, k_filter, k_pick) instead.
+constexpr int kFastLoads = 4;                       // 128-bit loads in flight per thread
+constexpr int kFastThreads = 512;                   // three blocks per SM, four loads each: 96 KB in flight per SM
+constexpr int kTailBins = 8;                        // histogram bins kept below tau
+
+__device__ __forceinline__ void tail_count(float g, unsigned int floor_key, unsigned int* sh_hist) {
+    const uint32_t key = mag_bits(g);
+    if (key >= floor_key) atomicAdd(&sh_hist[key >> 19], 1u);
+}
+
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_select_fast(const float* __restrict__ grad, unsigned long long d, unsigned int s, unsigned int want,
+              unsigned long long* __restrict__ cand, unsigned int* __restrict__ hist, Counters* __restrict__ cnt,
+              uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val) {
+    __shared__ __align__(16) unsigned int sh_hist[kSelBins];
+    __shared__ PickSmem sm;
+    __shared__ unsigned int part[kFastThreads];
+    __shared__ unsigned int next_bin;
+    __shared__ bool last;
+    unsigned int tau = cnt->sel_tau_next;
+    if (tau == 0u) tau = 0x7F800000u;                // nothing usable carried: only non-finite entries pass; the exact path serves
+    const unsigned int tau_bin = tau >> 19;
+    const unsigned int floor_bin = tau_bin > (unsigned int)kTailBins ? tau_bin - kTailBins : 0u;
+    const unsigned int floor_key = floor_bin << 19;
+    for (int b = threadIdx.x; b < kSelBins; b += kFastThreads) sh_hist[b] = 0u;
+    __syncthreads();
+    const unsigned long long n4 = d >> 2;
+    const float4* g4 = reinterpret_cast<const float4*>(grad);
+    const unsigned long long stride = (unsigned long long)gridDim.x * kFastThreads;
+    unsigned long long i = (unsigned long long)blockIdx.x * kFastThreads + threadIdx.x;
+    for (; i + (kFastLoads - 1) * stride < n4; i += kFastLoads * stride) {
+        float4 v[kFastLoads];
+#pragma unroll
+        for (int u = 0; u < kFastLoads; ++u) v[u] = __ldcs(g4 + i + u * stride);
+        uint32_t m = 0u;
+#pragma unroll
+        for (int u = 0; u < kFastLoads; ++u)
+            m = max(m, max(max(mag_bits(v[u].x), mag_bits(v[u].y)), max(mag_bits(v[u].z), mag_bits(v[u].w))));
+        if (m >= floor_key) {
+#pragma unroll
+            for (int u = 0; u < kFastLoads; ++u) {
+                const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    tail_count(e[c], floor_key, sh_hist);
+                    consider(e[c], (i + u * stride) * 4 + c, tau, cand, cnt);
+                }
+            }
+        }
+    }
+    for (; i < n4; i += stride) {
+        const float4 a = __ldcs(g4 + i);
+        const float e[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            tail_count(e[c], floor_key, sh_hist);
+            consider(e[c], i * 4 + c, tau, cand, cnt);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (d & 3ull)) {       // ragged tail
+        const unsigned long long t = (n4 << 2) + threadIdx.x;
+        tail_count(grad[t], floor_key, sh_hist);
+        consider(grad[t], t, tau, cand, cnt);
+    }
+    __syncthreads();
+    for (int b = floor_bin + threadIdx.x; b < kSelBins; b += kFastThreads)
+        if (sh_hist[b]) atomicAdd(&hist[b], sh_hist[b]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = (atomicAdd(&cnt->sel_ticket2, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    // ---- last block: next threshold from the histogram, then the exact pick --------------------------------------
+    // the histogram comes into shared memory in one parallel read; thread t sums its bins, a block-wide suffix scan finds
+    // the thread whose bins hold the crossing, and that thread walks them
+    constexpr int per = kSelBins / kFastThreads;        // 8 bins per thread
+    unsigned int mine = 0;
+    for (int u = 0; u < per; ++u) { const unsigned int c = __ldcg(&hist[threadIdx.x * per + u]); sh_hist[threadIdx.x * per + u] = c; mine += c; }
+    const unsigned int count = __ldcg(&cnt->sel_count);
+    const bool hit = count >= s && count <= (unsigned int)kSelCap;
+    part[threadIdx.x] = mine;
+    if (threadIdx.x == 0) next_bin = floor_bin;         // when even the whole histogram holds fewer than `want`: its floor
+    __syncthreads();
+    {
+        // keys in the bins of higher threads: suffix sum by a Hillis-Steele scan over the reversed order
+        const int rt = kFastThreads - 1 - threadIdx.x;
+        unsigned int incl = mine;
+        for (int o = 1; o < kFastThreads; o <<= 1) {
+            __syncthreads();
+            const unsigned int add = (rt >= o) ? part[threadIdx.x + o] : 0u;
+            __syncthreads();
+            incl += add;
+            part[threadIdx.x] = incl;
+        }
+        const unsigned int above = incl - mine;
+        if (above < want && want <= incl) {              // exactly one thread
+            unsigned int acc = above;
+            for (int u = per - 1; u >= 0; --u) {
+                acc += sh_hist[threadIdx.x * per + u];
+                if (acc >= want) { next_bin = threadIdx.x * per + u; break; }
+            }
+        }
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kSelBins; b += kFastThreads) hist[b] = 0u;    // the next step starts from zero
+    const unsigned long long* src = cand;
+    if (hit && count <= (unsigned int)(kSelBins / 2)) {
+        // a short candidate list is staged in shared memory (the histogram has served its purpose): the digit passes of
+        // the exact pick then read it from there
+        __syncthreads();
+        unsigned long long* staged = reinterpret_cast<unsigned long long*>(sh_hist);
+        for (unsigned int e = threadIdx.x; e < count; e += kFastThreads) staged[e] = __ldcg(cand + e);
+        __syncthreads();
+        src = staged;
+    }
+    // a miss hands pick_block an empty list: it then selects exactly over the whole gradient and flags the fallback
+    pick_block<kFastThreads>(sm, grad, d, s, src, hit ? count : 0u, cnt, sel_idx, sel_val);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int nb = next_bin;
+        if (!hit) {
+            // next threshold from the result itself: a quarter octave below the smallest kept magnitude
+            uint32_t lo = 0xFFFFFFFFu;
+            for (unsigned int e = 0; e < s; ++e) lo = min(lo, mag_bits(sel_val[e]));
+            nb = (lo >> 19) > 4u ? (lo >> 19) - 4u : 1u;
+        }
+        if (nb < 1u) nb = 1u;
+        cnt->sel_tau_next = nb << 19;
+        cnt->sel_count = 0u;
+        cnt->sel_ticket2 = 0u;
     }
 }
 
@@ -240,6 +414,7 @@ struct SelectPlan {
     unsigned int target;        // rank in the sample that corresponds to max(2048, 8 s) survivors in the vector
     int sample_grid;
     unsigned int filter_blocks;
+    unsigned int want;          // survivors aimed at: max(2048, 8 s)
 };
 
 SelectPlan plan_select(unsigned long long d, int s, int sm_count) {
@@ -254,6 +429,7 @@ SelectPlan plan_select(unsigned long long d, int s, int sm_count) {
     if (want < 2048ull) want = 2048ull;
     unsigned long long target = (want * n_sample + d - 1) / d;       // rank in the sample
     if (target < 32ull) target = 32ull;
+    p.want = (unsigned int)want;
     p.n_chunks = (unsigned int)n_chunks;
     p.target = (unsigned int)target;
     p.sample_grid = (int)(n_chunks < 4096ull ? n_chunks / 8 : 512);
@@ -267,12 +443,20 @@ SelectPlan plan_select(unsigned long long d, int s, int sm_count) {
     return p;
 }
 
-// The three launches of the selection on `stream`; hist and the counters must be zero on entry (k_sample leaves them
-// so for the next call).  `timed` (may be null) receives the per-kernel timing when profiling is on.
+// The launches of the selection on `stream`; hist and the counters must be zero on entry (the kernels leave them so for
+// the next call).  warm: a threshold carried from the previous call exists, and the one-kernel selection runs; otherwise
+// the sampled path (sample, filter, pick), which leaves its threshold behind when carry_out is set.  `timed` (may be null)
+// receives the per-kernel timing when profiling is on.
 cudaError_t enqueue_select(const float* grad, unsigned long long d, int s, int sm_count, unsigned int* hist,
                            unsigned long long* cand, Counters* cnt, uint32_t* out_idx, float* out_val, cudaStream_t stream,
-                           sgc_state* timed) {
+                           sgc_state* timed, bool warm, bool carry_out, int* launches) {
     const SelectPlan p = plan_select(d, s, sm_count);
+    if (warm && !p.direct) {
+        PhaseTimer timer(timed, stream, kPhaseFilter, 1);
+        k_select_fast<<<3 * sm_count, kFastThreads, 0, stream>>>(grad, d, (unsigned int)s, p.want, cand, hist, cnt, out_idx, out_val);
+        *launches += 1;
+        return cudaGetLastError();
+    }
     {
         PhaseTimer timer(timed, stream, kPhaseSample, 1);
         k_sample<<<p.direct ? 1 : p.sample_grid, kSampleThreads, 0, stream>>>(grad, d, p.n_chunks, p.target, hist, cnt, p.direct);
@@ -283,17 +467,20 @@ cudaError_t enqueue_select(const float* grad, unsigned long long d, int s, int s
     }
     {
         PhaseTimer timer(timed, stream, kPhasePick, 1);
-        k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)s, cand, cnt, out_idx, out_val);
+        k_pick<<<1, kPickThreads, 0, stream>>>(grad, d, (unsigned int)s, cand, cnt, out_idx, out_val, carry_out && !p.direct ? 1 : 0);
     }
+    *launches += 3;
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_select(sgc_state* st, const float* grad, cudaStream_t stream, int* launches) {
-    *launches += 3;
-    return enqueue_select(grad, (unsigned long long)st->d, st->s, st->sm_count, st->sel_hist, st->sel_cand, st->cnt,
-                          st->sel_idx, st->sel_val, stream, st);
+    // the first selection of a state samples its threshold; every later one carries it
+    const cudaError_t e = enqueue_select(grad, (unsigned long long)st->d, st->s, st->sm_count, st->sel_hist, st->sel_cand,
+                                         st->cnt, st->sel_idx, st->sel_val, stream, st, st->sel_warm, true, launches);
+    if (e == cudaSuccess) st->sel_warm = true;
+    return e;
 }
 
 }  // namespace sgc
@@ -370,7 +557,9 @@ extern "C" SGC_API int sgc_sparsify_static(const float* grad, int64_t d, int32_t
     // counters and histogram must start at zero; the candidate list is overwritten before it is read
     e = cudaMemsetAsync(setup.ptr, 0, kStaticCandOff, cs);
     if (e != cudaSuccess) return (int)e;
-    e = enqueue_select(grad, (unsigned long long)d, s, setup.sm_count, hist, cand, cnt, out_idx, out_val, cs, nullptr);
+    int launches = 0;
+    e = enqueue_select(grad, (unsigned long long)d, s, setup.sm_count, hist, cand, cnt, out_idx, out_val, cs, nullptr, false, false,
+                       &launches);
     if (e != cudaSuccess) return (int)e;
     if (out_status) k_copy_status<<<1, 1, 0, cs>>>(cnt, out_status);
     return (int)cudaGetLastError();
