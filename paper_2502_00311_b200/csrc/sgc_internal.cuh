@@ -106,7 +106,7 @@ constexpr int kSelCap = 32768;          // candidate slots of the top-s filter
 constexpr int kSelBins = 4096;          // 12-bit magnitude histogram of the sample
 constexpr int kCorrThreads = 512;       // threads per block of the correlation pass
 constexpr int kCorrCols = 2;            // columns per thread and tile
-constexpr int kCorrTop = 2;             // candidates kept per block and residual
+constexpr int kCorrTop = 3;             // slots per block and residual: its best two columns, and the score of its third best
 constexpr int kRescoreCap = 16;         // candidates rescored in fp64 per iteration and residual
 constexpr int kBookThreads = 1024;
 constexpr int kOmpThreads = 1024;       // threads per block of the cooperative OMP kernel

@@ -64,13 +64,16 @@ __device__ __forceinline__ bool better(float sa, uint32_t ia, float sb, uint32_t
     return (sa > sb) || (sa == sb && ia < ib);
 }
 
+// the best two columns seen, and the largest score among all others (what is dropped: the caller can tell whether a
+// dropped column could still have mattered)
 struct Top2 {
-    float s1, s2; uint32_t i1, i2;
-    __device__ __forceinline__ void init() { s1 = s2 = -1.0f; i1 = i2 = kNoColumn; }
+    float s1, s2, s3; uint32_t i1, i2;
+    __device__ __forceinline__ void init() { s1 = s2 = s3 = -1.0f; i1 = i2 = kNoColumn; }
     __device__ __forceinline__ void push(float s, uint32_t i) {
         if (i == i1 || i == i2) return;
-        if (better(s, i, s1, i1)) { s2 = s1; i2 = i1; s1 = s; i1 = i; }
-        else if (better(s, i, s2, i2)) { s2 = s; i2 = i; }
+        if (better(s, i, s1, i1)) { s3 = fmaxf(s3, s2); s2 = s1; i2 = i1; s1 = s; i1 = i; }
+        else if (better(s, i, s2, i2)) { s3 = fmaxf(s3, s2); s2 = s; i2 = i; }
+        else s3 = fmaxf(s3, s);
     }
 };
 
@@ -78,8 +81,10 @@ __device__ __forceinline__ void warp_merge(Top2& t) {
     for (int o = 16; o > 0; o >>= 1) {
         const float a1 = __shfl_xor_sync(0xffffffffu, t.s1, o), a2 = __shfl_xor_sync(0xffffffffu, t.s2, o);
         const uint32_t j1 = __shfl_xor_sync(0xffffffffu, t.i1, o), j2 = __shfl_xor_sync(0xffffffffu, t.i2, o);
+        const float a3 = __shfl_xor_sync(0xffffffffu, t.s3, o);
         if (j1 != kNoColumn) t.push(a1, j1);
         if (j2 != kNoColumn) t.push(a2, j2);
+        t.s3 = fmaxf(t.s3, a3);
     }
 }
 
@@ -277,6 +282,7 @@ __device__ void corr_all_columns(const OmpArgs& a, float2* sr, uint32_t (*mask_i
             Cand* o = a.corr_cand + ((size_t)warp * gridDim.x + blockIdx.x) * kCorrTop;
             o[0].score = t.s1; o[0].idx = t.i1;
             o[1].score = t.s2; o[1].idx = t.i2;
+            o[2].score = t.s3; o[2].idx = kNoColumn;        // score of the best column this block did not forward
         }
     }
 }
@@ -331,6 +337,7 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
             Cand* o = a.corr_cand + ((size_t)warp * gridDim.x + blockIdx.x) * kCorrTop;
             o[0].score = t.s1; o[0].idx = t.i1;
             o[1].score = t.s2; o[1].idx = t.i2;
+            o[2].score = -1.0f; o[2].idx = kNoColumn;       // a speculation: the screening pass judges what was left out
         }
     }
 }
@@ -376,6 +383,9 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
             if (c.idx != kNoColumn && c.score >= 0.0f && c.score >= thr) {
                 const int slot = atomicAdd(&sh.n_cand, 1);
                 if (slot < kRescoreCap) sh.cand_idx[slot] = c.idx;
+            } else if (c.idx == kNoColumn && c.score >= 0.0f && c.score >= thr) {
+                // a block kept a third column inside the rescoring window to itself: it never reaches the fp64 decision
+                atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
             }
         }
         __syncthreads();
