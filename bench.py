@@ -40,7 +40,7 @@ WORKLOADS = {
     "small_2M_k2048_s128": dict(d=1 << 21, k=2048, s=128, seed=1, kind="student", cfg_id=3),
     "c5_4096x11008_k1024_s16": dict(d=4096 * 11008, k=1024, s=16, seed=1, kind="student", cfg_id=5),
 }
-EXTRA_CONFIGS = ("drift", "c3_llama7b_layer", "c5_sweep", "mesgc", "c4_llama7b_32layers")
+EXTRA_CONFIGS = ("drift", "lockstep", "c3_llama7b_layer", "c5_sweep", "mesgc", "c4_llama7b_32layers")
 FP32_LANES_PER_SM = 128
 # sample of the CPU oracle that both the `cpu_baseline` leg and `--impl reference` time
 ORACLE_SAMPLE_COLS, ORACLE_SAMPLE_ITERS = 1 << 20, 8
@@ -267,6 +267,26 @@ def config_drift(binding, args):
     return out
 
 
+def config_lockstep(binding, args):
+    """The headline shape in lock-step mode (one pass over all columns per OMP iteration on the CUDA cores: the exact path that
+    the speculative recovery falls back to).  Useful flops = 2*k*d per column-residual product, 2 residuals, s iterations."""
+    wl = WORKLOADS["c2_4096x4096"]
+    m = SingleMatrix(binding, wl["d"], wl["k"], wl["s"], wl["seed"], 2, matrix_id=2)
+    m.st.set_mode(binding.MODE_LOCKSTEP)
+    out = m.run(1, 2)
+    m.close()
+    pk = peaks()
+    alu_peak = 148 * FP32_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6 / 1e12
+    achieved = 2.0 * wl["k"] * wl["d"] * 2 * wl["s"] / (out["ms_median"] * 1e-3) / 1e12
+    out.update(roofline={"kernel": "k_omp (lock-step)", "bound": "alu", "achieved": achieved, "peak": alu_peak, "unit": "TFLOP/s",
+                         "frac": achieved / alu_peak,
+                         "note": "useful fp32 FMA flops 2*k*d*2*s per step over the whole step time; peak = 148 SM * 128 lanes * 2 * "
+                                 "sm_max_mhz.  Each generated entry (6.5 instructions) serves only two multiply-adds here, which "
+                                 "caps the useful fraction near 2/(2 + 6.5) of the issue rate"})
+    out.pop("roofline_frac", None)
+    return {"lockstep_c2_4096x4096": out}
+
+
 def config_c5(binding, args):
     out = {}
     rows, cols = inputs.C5_SHAPE
@@ -419,7 +439,7 @@ def config_mesgc(binding, args):
     return out
 
 
-CONFIG_RUNNERS = {"drift": config_drift, "c3_llama7b_layer": config_c3, "c5_sweep": config_c5, "mesgc": config_mesgc,
+CONFIG_RUNNERS = {"drift": config_drift, "lockstep": config_lockstep, "c3_llama7b_layer": config_c3, "c5_sweep": config_c5, "mesgc": config_mesgc,
                   "c4_llama7b_32layers": config_c4}
 
 
