@@ -64,10 +64,10 @@ enum {
     SGC_STATUS_NEGATIVE_V = 1u << 3,       /* a recovered second-moment entry was <= 0; skipped   */
     SGC_STATUS_CANDIDATE_OVERFLOW = 1u << 4, /* a bounded candidate buffer overflowed.  In the speculative recovery the
                                                 step then fell back to its slower exact path (result unaffected).  In the
-                                                lock-step recovery more near-maximal columns (within 2e-3 of the best fp32
-                                                score) met than reach the fp64 decision -- more than 16 in all, or three in
-                                                one block's range: the pick may then differ from the exact argmax by such a
-                                                near-tie                                                            */
+                                                lock-step recovery more than 16 columns came within 2e-3 of the best fp32
+                                                score of one pick (a block that keeps such a column beyond the two it
+                                                forwards has its range screened again, so up to 16 always reach the fp64
+                                                decision): the pick may then differ from the exact argmax by a near-tie */
     SGC_STATUS_SELECT_FALLBACK = 1u << 5,  /* the sampled top-s threshold missed; exact fallback ran */
     SGC_STATUS_TIMEOUT = 1u << 6           /* a bounded wait inside a tensor-core screening pass ran out; the pass's
                                               reports were discarded and the step finished on its slower exact path */

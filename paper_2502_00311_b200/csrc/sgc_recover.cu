@@ -127,6 +127,7 @@ struct BookSmem {
     uint32_t best_idx;
     uint32_t cand_idx[kRescoreCap];
     int n_cand;
+    int rescan_n; int rescan_blk[8];  // blocks of the lock-step screen that kept a near-maximal column to themselves
     int hi, extra, dep, stop;         // speculation record of this block's stream
     unsigned int smax_bits;
 };
@@ -342,6 +343,51 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
     }
 }
 
+__device__ __forceinline__ bool in_support_list(const uint32_t* lam, int n, uint32_t col) {
+    for (int q = 0; q < n; ++q) if (lam[q] == col) return true;
+    return false;
+}
+
+// Lock-step only.  Block `blk` of the screen forwarded its best two columns for residual m, but a third scored inside the
+// rescoring window as well (score >= thr).  The bookkeeping block walks that block's tiles again with the arithmetic of
+// corr_all_columns (same operations in the same order, hence the same fp32 scores) and appends every free column with
+// score >= thr that was not forwarded, so that all of them reach the fp64 decision.  Costs about one screen of a block
+// (a 1/gridDim share of the columns), only when it happens.
+__device__ void rescan_block(const OmpArgs& a, BookSmem& sh, int m, int j, int blk, float thr, const float2* sr,
+                             const Cand* fwd) {
+    const int k = a.k;
+    const uint32_t f0 = fwd[0].idx, f1 = fwd[1].idx;
+    const uint32_t* lam = a.lam + (size_t)m * a.s;
+    constexpr unsigned int kTileCols = kOmpThreads * kCorrCols;
+    for (unsigned int tile = (unsigned int)blk; tile < a.num_tiles; tile += gridDim.x) {
+        const unsigned long long col_base = (unsigned long long)tile * kTileCols;
+#pragma unroll 1
+        for (int c = 0; c < kCorrCols; ++c) {
+            const unsigned long long col = col_base + c * kOmpThreads + threadIdx.x;
+            const ColKey key = column_key(a.seed_lo, a.seed_hi, (uint32_t)col);
+            uint32_t h = key.ck;
+            float acc = 0.0f, an = 0.0f;
+            for (int row = 0; row < k; row += 2) {
+                const float2 r0 = sr[row], r1 = sr[row + 1];
+                const float2 z = half2_bits_to_float2(z_pair_from_word(h));
+                h += key.mk;
+                acc = __fmaf_rn(z.x, m ? r0.y : r0.x, acc);
+                an = __fmaf_rn(z.x, z.x, an);
+                acc = __fmaf_rn(z.y, m ? r1.y : r1.x, acc);
+                if (row + 1 < k) an = __fmaf_rn(z.y, z.y, an);
+            }
+            if (col >= a.d) continue;
+            const float inv = an > 0.0f ? 1.0f / an : 0.0f;
+            const float sc = acc * acc * inv;
+            if (sc >= thr && (uint32_t)col != f0 && (uint32_t)col != f1 && !in_support_list(lam, j, (uint32_t)col)) {
+                const int slot = atomicAdd(&sh.n_cand, 1);
+                if (slot < kRescoreCap) sh.cand_idx[slot] = (uint32_t)col;
+            }
+        }
+    }
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------------------
 // phase B: one pick of Algorithm 3 for residual m (whole block).  The pick is `forced` when given, otherwise
 // the fp64 argmax among the screened candidates of phase A.
@@ -350,7 +396,7 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
 // recorded); spec_next >= 0: the new residual becomes row spec_next of the screened batch.
 // ------------------------------------------------------------------------------------------------
 __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t forced, int spec_c, int spec_next,
-                         bool final_pick, const Cand* cc, int n_entries) {
+                         bool final_pick, const Cand* cc, int n_entries, const float2* sr_lock = nullptr) {
     const int k = a.k, s = a.s;
     const double* y = a.y64 + (size_t)m * k;
     double* r = a.r64 + (size_t)m * k;
@@ -372,7 +418,7 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
             if (c.idx != kNoColumn) mx = fmaxf(mx, c.score);
         }
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if (threadIdx.x == 0) sh.n_cand = 0;
+        if (threadIdx.x == 0) { sh.n_cand = 0; sh.rescan_n = 0; }
         if (lane == 0) sh.fred[warp] = mx;
         __syncthreads();
         mx = sh.fred[lane];
@@ -384,11 +430,19 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
                 const int slot = atomicAdd(&sh.n_cand, 1);
                 if (slot < kRescoreCap) sh.cand_idx[slot] = c.idx;
             } else if (c.idx == kNoColumn && c.score >= 0.0f && c.score >= thr) {
-                // a block kept a third column inside the rescoring window to itself: it never reaches the fp64 decision
-                atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
+                // a block of the lock-step screen kept a third column inside the rescoring window to itself: its range is
+                // screened again below so that the column reaches the fp64 decision (flagged only when that cannot be done)
+                const int slot = sr_lock != nullptr ? atomicAdd(&sh.rescan_n, 1) : 8;
+                if (slot < 8) sh.rescan_blk[slot] = e / kCorrTop;
+                else atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
             }
         }
         __syncthreads();
+        if (sr_lock != nullptr) {
+            const int n_rescan = sh.rescan_n < 8 ? sh.rescan_n : 8;
+            for (int q = 0; q < n_rescan; ++q)
+                rescan_block(a, sh, m, j, sh.rescan_blk[q], thr, sr_lock, cc + (size_t)sh.rescan_blk[q] * kCorrTop);
+        }
         nc = sh.n_cand;
         if (nc > kRescoreCap) {
             if (threadIdx.x == 0) atomicOr(&a.cnt->status, (unsigned int)SGC_STATUS_CANDIDATE_OVERFLOW);
@@ -595,7 +649,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
             const int c = j - base[m];                            // -1 for a confirmed prescribed pick
             const int next = (mode == 0 && c + 1 < a.half_n && j + 1 < a.s) ? c + 1 : -1;
             const int rc = book_pick(a, sh, m, j, forced, speculative ? c : -1, next, !speculative,
-                                     a.corr_cand + (size_t)m * gridDim.x * kCorrTop, (int)gridDim.x * kCorrTop);
+                                     a.corr_cand + (size_t)m * gridDim.x * kCorrTop, (int)gridDim.x * kCorrTop,
+                                     mode == 1 ? sr : nullptr);
             if (threadIdx.x == 0) {
                 if (rc == 0) {
                     sh.hi = j + 1;

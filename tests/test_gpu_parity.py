@@ -330,6 +330,37 @@ def test_dependent_column_stops_like_the_oracle(sgc):
     st.close()
 
 
+def test_lockstep_three_near_tied_columns_in_one_block(sgc):
+    # The lock-step screen runs in fp32 and every block forwards only its best two columns per residual to the fp64
+    # decision.  Three columns of one block's range whose scores agree to ~1e-7 (far inside the 2e-3 rescoring window, far
+    # above fp64 noise) must still be ordered as the oracle orders them: the block reports that it kept a third one back and
+    # its range is screened again.  M^ = a_c1 x1 + a_c2 x2 + a_c3 x3 with x solving "equal normalised correlations".
+    d, k, s = 4096, 256, 3
+    hp = inputs.ADAM
+    rng = np.random.default_rng(17)
+    for trial in range(12):
+        seed = 100 + trial
+        cols = np.sort(rng.choice(2048, size=3, replace=False))              # one tile of the screen: one block
+        A = float(oracle.sigma(k)) * np.stack([oracle.z_block(seed, 0, k, int(c), 1)[:, 0] for c in cols], axis=1).astype(np.float64)
+        G = (A.T @ A) / np.sqrt((A * A).sum(axis=0))[:, None]
+        x = np.linalg.solve(G, np.ones(3))
+        g = np.zeros(d, dtype=np.float32)
+        g[cols] = x.astype(np.float32)
+        st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+        ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+        w, wr = cuda(np.zeros(d, dtype=np.float32)), np.zeros(d, dtype=np.float32)
+        st.step(cuda(g), w)
+        ref.step(g, wr)
+        assert int(st.get("fallback")) == 1                                   # d < 65536: lock-step
+        top = ref.get("top1M")[0], ref.get("top2M")[0]
+        assert abs(top[0] - top[1]) < 1e-5 * top[0]                           # the premise: a near-tie at the first pick
+        assert np.array_equal(st.get("lamM"), ref.get("lamM")), (trial, st.get("lamM"), ref.get("lamM"))
+        assert np.array_equal(st.get("lamV"), ref.get("lamV")), trial
+        assert not int(st.get("status")) & sgc.STATUS_CANDIDATE_OVERFLOW
+        st.close()
+        ref.close()
+
+
 def test_state_set_get_roundtrip_and_resume(sgc):
     d, k, s = 30_000, 128, 6
     hp = inputs.ADAM
