@@ -37,6 +37,10 @@ constexpr int kSuperCols = 2 * kTileCols;                    // columns of A per
 constexpr int kChunkRows = 64;                               // rows of A per pipeline stage (128 B of binary16)
 constexpr int kTileBytes = kTileCols * kChunkRows * 2;       // 16384
 constexpr int kNormRing = 8;
+#ifndef SGC_PASS_SWAP
+#define SGC_PASS_SWAP 1
+#endif
+constexpr bool kPassSwap = SGC_PASS_SWAP != 0;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default bound of every mbarrier wait
 
 struct PassArgs {
@@ -176,7 +180,10 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // WIDE: the two-level screening code (wide-list harvest, list passes) is compiled in
 // SUB: 64-row chunks of A per slot of the ring, i.e. per hand-off between generators, TMA and MMA issuer (2 when the
 // residual block is narrow enough for two slots of 128 rows: half as many barrier rounds per generated entry)
-template <bool TABLE, bool WIDE, int SUB>
+// SWAP (128 residual rows, table of norms, no wide lists): the residual chunk is the M operand and all 256 generated columns
+// the N operand of one MMA per 16 rows (instead of two MMAs of N = 128 that both read the residual chunk); the accumulator then
+// holds residuals along the lanes and columns of A along the tensor-memory columns
+template <bool TABLE, bool WIDE, int SUB, bool SWAP>
 __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant__ CUtensorMap tmap, PassArgs a) {
     if (a.gate[0] != nullptr) {
         bool any = false;
@@ -268,6 +275,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
         // ---------------- MMA issuer ----------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(a.n);
+            const uint32_t idesc_swap = umma_idesc(kSuperCols);      // M = 128 residual rows, N = 256 columns of A
             // descriptors differ only in their start-address field (units of 16 bytes): keep that word per stage
             const uint64_t desc_hi = umma_desc(0) & 0xFFFFFFFF00000000ull;
             const uint32_t desc_lo0 = (uint32_t)(umma_desc(base) & 0xFFFFFFFFull);
@@ -289,8 +297,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
 #pragma unroll
                         for (int kk = 0; kk < kChunkRows / 16; ++kk) {
                             const uint64_t bdesc = desc_hi | (uint64_t)(lo + (2 * kTileBytes >> 4) + 2 * kk);
-                            umma_f16(acc0, desc_hi | (uint64_t)(lo + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
-                            umma_f16(acc1, desc_hi | (uint64_t)(lo + (kTileBytes >> 4) + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                            if (SWAP) {
+                                // D[residual][column] += R_chunk (128 x 16) * Z (256 x 16)^T: both tiles of A are one N operand
+                                umma_f16(acc0, bdesc, desc_hi | (uint64_t)(lo + 2 * kk), idesc_swap, kk != 0 ? 1u : first);
+                            } else {
+                                umma_f16(acc0, desc_hi | (uint64_t)(lo + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                                umma_f16(acc1, desc_hi | (uint64_t)(lo + (kTileBytes >> 4) + 2 * kk), bdesc, idesc, kk != 0 ? 1u : first);
+                            }
                         }
                     }
                     umma_commit(bar_empty + 8u * st);        // frees the stage once these MMAs have read it
@@ -308,6 +321,79 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
             const uint32_t buf = sweep_i % a.bufs, use = sweep_i / a.bufs;
             if (!__all_sync(0xffffffffu, mbar_wait(bar_accf + 8u * buf, use & 1u, abort_flag, 512, a.wait_limit_ns))) { ok = false; break; }
             tc_fence_after();
+            if (SWAP) {
+                // this thread owns residual n_res; the 256 columns of the sweep run along the tensor-memory columns.  Each
+                // epilogue warp keeps its own copy of the sweep's 1 / ||Z_i|| as floats (no barrier between the warps)
+                const int n_res = quad * 32 + lane;
+                const float tau_n = tau_s[n_res];
+                float* inv_w = norms + (size_t)quad * kSuperCols;
+                uint32_t* col_w = reinterpret_cast<uint32_t*>(norms + (size_t)(4 + quad) * kSuperCols);   // list pass: the columns
+                __syncwarp();
+#pragma unroll
+                for (int q = 0; q < kSuperCols / 32; ++q) {
+                    unsigned long long col = (unsigned long long)sweep * kSuperCols + q * 32 + lane;
+                    if (listed) {
+                        const unsigned int idx = (unsigned int)col;
+                        col = idx < list_n0 ? a.big_list[idx] : (idx < list_n ? a.big_list[(size_t)a.big_cap + idx - list_n0] : a.d);
+                        col_w[q * 32 + lane] = (uint32_t)col;
+                    }
+                    inv_w[q * 32 + lane] = col < a.d ? half_bits_to_float(a.inv_norm[col]) : 0.0f;
+                }
+                __syncwarp();
+                // every 8th residual feeds the wide list of its stream (full passes of the two-level screening)
+                const bool feeds = WIDE && a.big_tau != nullptr && !listed && (n_res & 7) == 0;
+                const float wide_tau_n = feeds ? a.big_tau[n_res >> 3] : 0.0f;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kSuperCols; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * acc_cols + c0, v);
+                    float peak = 0.0f;
+                    const float4* in4 = reinterpret_cast<const float4*>(inv_w + c0);
+#pragma unroll
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 w = in4[i4];
+                        peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4])) * w.x);
+                        peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 1])) * w.y);
+                        peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 2])) * w.z);
+                        peak = fmaxf(peak, fabsf(__uint_as_float(v[4 * i4 + 3])) * w.w);
+                    }
+                    if (feeds && peak >= wide_tau_n) {
+                        const int m = n_res >= a.big_half ? 1 : 0;
+                        unsigned int hits = 0u;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            hits |= (fabsf(__uint_as_float(v[i])) * inv_w[c0 + i] >= wide_tau_n ? 1u : 0u) << i;
+                        while (hits) {
+                            const int i = __ffs(hits) - 1;
+                            hits &= hits - 1u;
+                            const unsigned long long col = (unsigned long long)sweep * kSuperCols + c0 + i;
+                            const unsigned int bit = 1u << ((unsigned int)col & 31u);
+                            if (!(atomicOr(&a.big_bits[(size_t)m * ((a.d + 31) >> 5) + (col >> 5)], bit) & bit)) {
+                                const unsigned int slot = atomicAdd(&a.big_count[m], 1u);
+                                if (slot < (unsigned int)a.big_cap) a.big_list[(size_t)m * a.big_cap + slot] = (uint32_t)col;
+                            }
+                        }
+                    }
+                    if (!(peak >= tau_n)) continue;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float inv = inv_w[c0 + i];
+                        const float sc = fabsf(__uint_as_float(v[i])) * inv;
+                        if (sc >= tau_n && inv > 0.0f) {
+                            const unsigned int slot = atomicAdd(&a.rep_count[n_res], 1u);
+                            if (slot < (unsigned int)a.rep_cap) {
+                                const float out = a.inv_scale ? sc * a.inv_scale[n_res] : sc;
+                                const uint32_t col = listed ? col_w[c0 + i] : (uint32_t)((unsigned long long)sweep * kSuperCols + c0 + i);
+                                a.rep[(size_t)n_res * a.rep_cap + slot] = make_uint2(col, __float_as_uint(out));
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+                continue;
+            }
             const float* nr = norms + (size_t)(sweep_i % kNormRing) * kSuperCols * 2;
 #pragma unroll 1
             for (int t = 0; t < 2; ++t) {
@@ -516,9 +602,9 @@ cudaError_t pass_encode_map(void* tmap_out, const void* rt, int n, int k) {
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <bool TABLE, bool WIDE, int SUB>
+template <bool TABLE, bool WIDE, int SUB, bool SWAP = false>
 cudaError_t pass_opt_in(int need) {
-    return cudaFuncSetAttribute(k_pass<TABLE, WIDE, SUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, need);
+    return cudaFuncSetAttribute(k_pass<TABLE, WIDE, SUB, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, need);
 }
 
 cudaError_t pass_configure(int) {
@@ -535,6 +621,8 @@ cudaError_t pass_configure(int) {
     if (e == cudaSuccess) e = pass_opt_in<true, true, 2>((int)need);
     if (e == cudaSuccess) e = pass_opt_in<true, false, 1>((int)need);
     if (e == cudaSuccess) e = pass_opt_in<true, false, 2>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, false, 2, true>((int)need);
+    if (e == cudaSuccess) e = pass_opt_in<true, true, 2, true>((int)need);
     return e;
 }
 
@@ -570,13 +658,15 @@ cudaError_t launch_pass(const void* tmap, uint64_t seed, uint64_t d, int k, int 
     memcpy(&map, tmap, sizeof(map));
     const size_t smem = pass_smem_bytes(n, a.stages, sub);
     if (sub == 2) {
-        if (inv_norm && wide) k_pass<true, true, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
-        else if (inv_norm) k_pass<true, false, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
-        else k_pass<false, false, 2><<<grid, kPassThreads, smem, stream>>>(map, a);
+        if (inv_norm && wide && n == kTileCols && kPassSwap) k_pass<true, true, 2, true><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm && wide) k_pass<true, true, 2, false><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm && n == kTileCols && kPassSwap) k_pass<true, false, 2, true><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm) k_pass<true, false, 2, false><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else k_pass<false, false, 2, false><<<grid, kPassThreads, smem, stream>>>(map, a);
     } else {
-        if (inv_norm && wide) k_pass<true, true, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
-        else if (inv_norm) k_pass<true, false, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
-        else k_pass<false, false, 1><<<grid, kPassThreads, smem, stream>>>(map, a);
+        if (inv_norm && wide) k_pass<true, true, 1, false><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else if (inv_norm) k_pass<true, false, 1, false><<<grid, kPassThreads, smem, stream>>>(map, a);
+        else k_pass<false, false, 1, false><<<grid, kPassThreads, smem, stream>>>(map, a);
     }
     return cudaGetLastError();
 }
