@@ -15,7 +15,7 @@ _lib = None
 EXPORTS = ["sgc_create", "sgc_step", "sgc_step_group", "sgc_step_chunked", "sgc_cesgc_step", "sgc_destroy", "sgc_set_alpha", "sgc_get", "sgc_set_state",
            "sgc_clear_status", "sgc_last_launches", "sgc_set_profile", "sgc_get_profile", "sgc_sparsify_static", "sgc_z_block",
            "sgc_set_mode", "sgc_set_recovery", "sgc_screen", "sgc_reproject", "sgc_strerror", "sgc_version", "sgc_status",
-           "sgc_set_wait_limit"]
+           "sgc_set_wait_limit", "sgc_set_max_rounds"]
 
 # selectors of sgc_get: name -> (code, dtype, length attribute or None for a scalar)
 RECORDS = dict(t=(0, np.int64, None), M=(1, np.float32, "k"), V=(2, np.float32, "k"), sel_idx=(3, np.uint32, "s"),
@@ -79,6 +79,8 @@ def lib():
         L.sgc_status.argtypes = [vp, C.POINTER(C.c_uint32)]
         L.sgc_set_wait_limit.restype = C.c_int
         L.sgc_set_wait_limit.argtypes = [vp, C.c_uint64]
+        L.sgc_set_max_rounds.restype = C.c_int
+        L.sgc_set_max_rounds.argtypes = [vp, C.c_int32]
         L.sgc_last_launches.restype = C.c_int
         L.sgc_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
         L.sgc_set_profile.restype = C.c_int
@@ -237,6 +239,10 @@ class Sgc:
     def set_wait_limit(self, ns):
         """Bound (ns) of the waits inside this state's screening passes; 0 restores the default."""
         _check(lib().sgc_set_wait_limit(self._h, C.c_uint64(int(ns))), "sgc_set_wait_limit")
+
+    def set_max_rounds(self, rounds):
+        """Most speculation rounds a step enqueues (what they leave open is finished in lock-step); 0 = automatic."""
+        _check(lib().sgc_set_max_rounds(self._h, C.c_int32(int(rounds))), "sgc_set_max_rounds")
 
     def clear_status(self):
         _check(lib().sgc_clear_status(self._h), "sgc_clear_status")

@@ -391,6 +391,13 @@ SGC_API int sgc_set_wait_limit(sgc_state* st, uint64_t ns) {
     return SGC_OK;
 }
 
+SGC_API int sgc_set_max_rounds(sgc_state* st, int32_t rounds) {
+    if (!st) return SGC_ERR_NULL;
+    if (rounds < 0) return SGC_ERR_DIM;
+    st->max_rounds = rounds;
+    return SGC_OK;
+}
+
 SGC_API int sgc_last_launches(sgc_state* st, int32_t* out) {
     if (!st || !out) return SGC_ERR_NULL;
     *out = st->last_launches;

@@ -300,6 +300,7 @@ struct sgc_state {
     unsigned int* wide_count;   // [2]
     unsigned int* wide_bits;    // [2] bitmaps over [0, d): the column is in the stream's wide list
     unsigned long long wait_limit_ns;   // bound of the waits inside this state's screening passes; 0 = the default
+    int max_rounds;             // host: most speculation rounds a step may enqueue; 0 = chosen from the last step's count
     int* h_rounds;              // pinned, device-mapped: rounds the last finished step needed (read without synchronising)
     int* d_rounds;              // device alias of h_rounds
 };

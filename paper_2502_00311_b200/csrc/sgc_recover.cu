@@ -1067,7 +1067,13 @@ __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
         li[i] = a.pick_li[(size_t)m * s + i];
     }
     __syncthreads();
-    // the picked column of pick j, for the kernels that rebuild residuals from the stored columns
+    // the picked column of pick j, for the kernels that rebuild residuals from the stored columns; the block of the first
+    // state also stores the column of pick base - 1, which may be a prescribed one that no earlier round has stored
+    if (c == 0 && base > 0) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(a.zlist + (size_t)li[base - 1] * k);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(a.zsel + ((size_t)m * s + base - 1) * k);
+        for (int pr = t; pr < (k >> 1); pr += kGramThreads) dst[pr] = src[pr];
+    }
     if (j < hi) {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(a.zlist + (size_t)a.pick_li[(size_t)m * s + j] * k);
         uint32_t* dst = reinterpret_cast<uint32_t*>(a.zsel + ((size_t)m * s + j) * k);
@@ -1751,7 +1757,8 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
         // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
         const int hint = speculate ? *reinterpret_cast<volatile int*>(st->h_rounds) : 0;
         const int last = hint & 255;
-        const int want = last <= 0 ? 8 : 2 * last + 4;
+        int want = last <= 0 ? 8 : 2 * last + 4;
+        if (st->max_rounds > 0 && want > st->max_rounds) want = st->max_rounds;
         if (want > n_rounds) n_rounds = want;
         // two-level screening pays where steps need several full passes (recovery picks columns outside the kept sets);
         // it is dropped again when a step needed one pass and its list passes refuted nothing

@@ -193,6 +193,39 @@ def test_speculative_recovery_with_redrawn_supports_and_alpha(sgc):
     assert all(fb == 0 for _, fb, _ in stats), stats
 
 
+@pytest.mark.parametrize("max_rounds", [1, 2, 3])
+def test_lockstep_finishes_what_a_bounded_number_of_rounds_leaves_open(sgc, max_rounds):
+    # Two steady steps, then a new support every step, so that every later step needs several rounds of speculation and
+    # its first refuted pick gets a prescribed column.  With the rounds bounded, the lock-step path takes over from a
+    # state that the Gram-matrix speculation left behind -- stored columns, F, coefficients and the prescribed pick
+    # included -- and must still end with Algorithm 3's supports and update.
+    d, k, s, seed = 150_000, 256, 32, 3
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    st.set_mode(sgc.MODE_SPECULATIVE)
+    st.set_max_rounds(max_rounds)
+    ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    w0 = inputs.weights(d, 99)
+    w_gpu, w_ref = cuda(w0.copy()), w0.copy()
+    open_steps = 0
+    for step in range(1, 6):
+        supp, sign = inputs.planted_support(d, s, 1000 * seed + (0 if step <= 2 else step))
+        g = inputs.gradient(d, "student", supp, sign, 50 * seed + step)
+        st.step(cuda(g), w_gpu)
+        ref.step(g, w_ref)
+        assert np.array_equal(st.get("lamM"), ref.get("lamM")), step
+        assert np.array_equal(st.get("lamV"), ref.get("lamV")), step
+        assert int(st.get("rounds")) <= max_rounds
+        trace = st.get("round_trace").reshape(-1, 3)
+        open_steps += int(trace[int(st.get("rounds")) - 1, 0] < s or trace[int(st.get("rounds")) - 1, 1] < s)
+        np.testing.assert_allclose(w_gpu.cpu().numpy(), w_ref, rtol=0, atol=1e-6)
+    assert open_steps >= 1, open_steps              # the bound really cut a step short
+    with pytest.raises(sgc.SgcError):
+        st.set_max_rounds(-1)
+    st.close()
+    ref.close()
+
+
 @pytest.mark.parametrize("d,k,s,steps", [(400_000, 256, 48, 7), (1_000_000, 512, 100, 4)])
 def test_two_level_screening_matches_the_oracle(sgc, d, k, s, steps):
     # inexact regime (supports redrawn every step, k small): steps need several passes over all columns, which switches
