@@ -43,6 +43,7 @@ struct OmpArgs {
     unsigned int num_tiles;            // lock-step tiles of kOmpThreads * kCorrCols columns
     double sigma;
     int half_n;                        // residuals per stream in one screening pass
+    int rows_wide, rows_narrow;        // rows of the pass that serves both streams / the first stream alone
     double z_harvest, z_floor;         // screening thresholds in units of ||r|| / sqrt(k)
     Cand* corr_cand;                   // [2][grid][kCorrTop]
     const double* y64; double* r64; float* r32;      // r32 viewed as float[2k] (interleaved pairs)
@@ -1265,7 +1266,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
         else {
             ctl->rounds = ctl->rounds + 1;
             // width of the pass whose reports are being resolved (ctl->narrow still names it)
-            ctl->pass_rows = ctl->pass_rows + (ctl->narrow ? ((a.half_n + 31) / 32) * 32 : 2 * a.half_n);
+            ctl->pass_rows = ctl->pass_rows + (ctl->narrow ? a.rows_narrow : a.rows_wide);
         }
     }
     for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = 0;
@@ -1323,6 +1324,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             rescore_candidates(a, sh, nc, ra.rtmp);
             if (sh.best_idx == pick) { v = j + 1; continue; }
             forced = sh.best_idx; v = j; failed = true;
+            if (!mini && threadIdx.x == 0) ctl->refuted = ctl->refuted + 1;
             make_room(ra, (int)count + 1 + ((hi - j) / kLookAhead) * 1024);
             harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
             // look ahead: the later residuals of this speculation are off the true path by a pick or a few, yet close
@@ -1425,7 +1427,7 @@ __global__ void k_spec_init(SpecCtl* ctl, int speculate, float* wide_tau, int sh
     if (threadIdx.x == 0) {
         ctl->tv[0] = ctl->tv[1] = 0;
         ctl->tforced[0] = ctl->tforced[1] = kNoColumn;
-        ctl->mini_done = 0; ctl->list_rounds = 0; ctl->list_refuted = 0;
+        ctl->mini_done = 0; ctl->list_rounds = 0; ctl->list_refuted = 0; ctl->refuted = 0;
         // no wide list unless a long-list speculation asks for one
         if (wide_tau != nullptr) for (int g = 0; g < kPassMaxN / 8; ++g) wide_tau[g] = __int_as_float(0x7f800000);
         ctl->round_active = speculate; ctl->fallback = speculate ? 0 : 1;
@@ -1469,8 +1471,9 @@ k_cand_update(SpecCtl* ctl, const Counters* cnt, const uint32_t* lam, int s, uin
               const uint32_t* kept_ring, int* rounds_out) {
     __shared__ int n_s;
     // how many rounds this step took (the enqueued rounds if even they were not enough): sizes the next step's launches
-    // bit 8: a list pass refuted a pick (the wide lists earned their keep)
-    if (threadIdx.x == 0) *rounds_out = (ctl->fallback ? kMaxRounds : ctl->rounds) | (ctl->list_refuted > 0 ? 256 : 0);
+    // bit 8: a list pass refuted a pick (the wide lists earned their keep); bit 9: a full pass refuted a pick
+    if (threadIdx.x == 0)
+        *rounds_out = (ctl->fallback ? kMaxRounds : ctl->rounds) | (ctl->list_refuted > 0 ? 256 : 0) | (ctl->refuted > 0 ? 512 : 0);
     int n = ctl->n_cand;
     // rebuild from the supports and the ring of kept index sets when the list has outgrown its bound, or when it holds
     // far more than those although a single round confirmed every pick (harvested columns of an earlier cold start)
@@ -1643,6 +1646,7 @@ OmpArgs make_args(const sgc_state* st) {
     a.num_tiles = (unsigned int)(((unsigned long long)st->d + tile_cols - 1) / tile_cols);
     a.sigma = (double)(float)(1.0 / sqrt((double)st->k));
     a.half_n = st->pass_n / 2;
+    a.rows_wide = st->pass_n; a.rows_narrow = st->pass_n_half;
     a.z_harvest = st->z_harvest; a.z_floor = st->z_floor;
     a.corr_cand = st->corr_cand; a.y64 = st->y64; a.r64 = st->r64; a.r32 = reinterpret_cast<float*>(st->r32);
     a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
@@ -1767,11 +1771,22 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
     }
     if (n_rounds > kMaxRounds) n_rounds = kMaxRounds;
     const bool two_level = speculate && n == 1 && st0->two_level;
+    // A state whose two streams fill a pass of more than kPassFastRows rows, and whose last step had a pick refuted: the
+    // refuted stream needs several rounds anyway, and the rows of a speculation beyond its first refuted pick are wasted.
+    // Such a step screens half as many residuals per stream and round, in the pass of half the width at half the cost;
+    // the stream that is confirmed without contest rides along in two rounds instead of one.
+    const bool compact = speculate && n == 1 && st0->pass_n > kPassFastRows && st0->pass_n_half <= kPassFastRows &&
+                         (*reinterpret_cast<volatile int*>(st0->h_rounds) & 512) != 0;
+    if (compact) {
+        args[0].half_n = st0->pass_n_half / 2;
+        args[0].rows_wide = args[0].rows_narrow = st0->pass_n_half;
+        n_rounds = n_rounds + 1 < kMaxRounds ? n_rounds + 1 : kMaxRounds;
+    }
     PassWide wide;
     if (two_level) {
         args[0].wide_count = st0->wide_count;
         wide.tau = st0->wide_tau; wide.list = st0->wide_list; wide.count = st0->wide_count; wide.bits = st0->wide_bits;
-        wide.cap = kWideCap; wide.half_n = st0->pass_n / 2; wide.ctl = st0->ctl; wide.list_pass = false;
+        wide.cap = kWideCap; wide.half_n = args[0].half_n; wide.ctl = st0->ctl; wide.list_pass = false;
     }
     if (speculate) {
         for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
@@ -1793,7 +1808,12 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
                     int* errors[kPassMaxBatch] = {&st->ctl->pass_error};
                     PassWide lp = wide;
                     lp.list_pass = true;
-                    const bool two_widths = st->pass_n_half < st->pass_n;       // the width that ctl->narrow names runs
+                    const bool two_widths = !compact && st->pass_n_half < st->pass_n;   // the width that ctl->narrow names runs
+                    if (compact)
+                        e = launch_pass(st->tmap_half, st->seed, (uint64_t)st->d, st->k, st->pass_n_half, st->tau, st->inv_scale,
+                                        st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp,
+                                        nullptr, 0, st->wait_limit_ns);
+                    else
                     e = launch_pass(st->tmap[0], st->seed, (uint64_t)st->d, st->k, st->pass_n, st->tau, st->inv_scale,
                                     st->inv_norm, st->rep_count, st->rep, kRepCap, gates, errors, st->sm_count, stream, &lp,
                                     two_widths ? &st->ctl->narrow : nullptr, 0, st->wait_limit_ns);
@@ -1840,7 +1860,12 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
                     }
                     // a state on its own: once only its first stream has residuals left (the second recovery is complete, or
                     // the shared-support variant is on), the pass half as wide serves the round; ctl->narrow names the width
-                    const bool two_widths = n == 1 && lead->pass_n_half < lead->pass_n;
+                    const bool two_widths = n == 1 && !compact && lead->pass_n_half < lead->pass_n;
+                    if (compact)
+                        e = launch_pass(lead->tmap_half, lead->seed, (uint64_t)lead->d, lead->k, lead->pass_n_half, lead->tau,
+                                        lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
+                                        lead->sm_count, stream, two_level ? &wide : nullptr, nullptr, 0, lead->wait_limit_ns);
+                    else
                     e = launch_pass(lead->tmap[nb - 1], lead->seed, (uint64_t)lead->d, lead->k, nb * lead->pass_n, lead->tau,
                                     lead->inv_scale, lead->inv_norm, lead->rep_count, lead->rep, kRepCap, gates, errors,
                                     lead->sm_count, stream, two_level ? &wide : nullptr,

@@ -226,6 +226,34 @@ def test_lockstep_finishes_what_a_bounded_number_of_rounds_leaves_open(sgc, max_
     ref.close()
 
 
+def test_steps_after_a_refuted_pick_screen_in_passes_of_half_the_width(sgc):
+    # s = 96: both streams fill a pass of 192 residual rows.  After a step in which a full pass refuted a pick, the
+    # next step screens 48 residuals per stream and round in the 96-row pass (half the cost per round); the supports
+    # must not depend on which width a step used.
+    d, k, s, seed = 100_000, 768, 96, 5
+    hp = inputs.ADAM
+    st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    st.set_mode(sgc.MODE_SPECULATIVE)
+    ref = oracle.Oracle(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
+    w0 = inputs.weights(d, 99)
+    w_gpu, w_ref = cuda(w0.copy()), w0.copy()
+    widths = []
+    for step in range(1, 7):
+        supp, sign = inputs.planted_support(d, s, 77 + (0 if step <= 2 else step))      # new supports from step 3 on
+        g = inputs.gradient(d, "student", supp, sign, 900 + step)
+        st.step(cuda(g), w_gpu)
+        ref.step(g, w_ref)
+        assert np.array_equal(st.get("lamM"), ref.get("lamM")), step
+        assert np.array_equal(st.get("lamV"), ref.get("lamV")), step
+        np.testing.assert_allclose(w_gpu.cpu().numpy(), w_ref, rtol=0, atol=1e-6)
+        assert int(st.get("fallback")) == 0
+        widths.append((int(st.get("rounds")), int(st.get("pass_rows"))))
+    assert widths[0][1] >= 192, widths                                    # a fresh state starts with the pass over all 192 rows
+    assert any(r >= 2 and rows == 96 * r for r, rows in widths[1:]), widths
+    st.close()
+    ref.close()
+
+
 @pytest.mark.parametrize("d,k,s,steps", [(400_000, 256, 48, 7), (1_000_000, 512, 100, 4)])
 def test_two_level_screening_matches_the_oracle(sgc, d, k, s, steps):
     # inexact regime (supports redrawn every step, k small): steps need several passes over all columns, which switches
