@@ -292,18 +292,27 @@ __device__ void corr_all_columns(const OmpArgs& a, float2* sr, uint32_t (*mask_i
 // ------------------------------------------------------------------------------------------------
 // phase A, restricted: the candidate list against both residuals (warp = one column, lanes over rows)
 // ------------------------------------------------------------------------------------------------
-__device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], const int* picks) {
+__device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], const int* picks, float2* sr,
+                                uint32_t (*sup)[kMaxS]) {
     const int k = a.k, s = a.s;
-    const float2* r32 = reinterpret_cast<const float2*>(a.r32);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // the residual pair and both supports, once per call, in shared memory: every candidate reads them
+    {
+        const float2* r32 = reinterpret_cast<const float2*>(a.r32);
+        for (int row = threadIdx.x; row < k; row += kOmpThreads) sr[row] = r32[row];
+        for (int q = threadIdx.x; q < picks[0]; q += kOmpThreads) sup[0][q] = a.lam[q];
+        for (int q = threadIdx.x; q < picks[1]; q += kOmpThreads) sup[1][q] = a.lam[s + q];
+    }
+    __syncthreads();
+    const float2* r32 = sr;
     Top2 best[2];
     best[0].init(); best[1].init();
     const int stride = gridDim.x * (kOmpThreads / 32);
     for (int e = warp * gridDim.x + blockIdx.x; e < n_cand; e += stride) {        // neighbours go to different blocks
         const uint32_t col = a.cand_list[e];
         bool t0 = false, t1 = false;
-        for (int q = lane; q < picks[0]; q += 32) t0 |= (a.lam[q] == col);
-        for (int q = lane; q < picks[1]; q += 32) t1 |= (a.lam[s + q] == col);
+        for (int q = lane; q < picks[0]; q += 32) t0 |= (sup[0][q] == col);
+        for (int q = lane; q < picks[1]; q += 32) t1 |= (sup[1][q] == col);
         t0 = __any_sync(0xffffffffu, t0);
         t1 = __any_sync(0xffffffffu, t1);
         const ColKey key = column_key(a.seed_lo, a.seed_hi, col);
@@ -480,47 +489,62 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     }
     __syncthreads();
     // ---- 4. g = A_Lambda^T a_new  (Gram column; "g_{:,lambda_k}" restricted to the support) --------------
+    // warp = one stored column; eight binary16 entries per load when the rows allow it
     const double sig2 = a.sigma * a.sigma;
     {
         const uint16_t* znew = zs + (size_t)j * k;
+        const bool vec = (k & 7) == 0;
         for (int l = warp; l < j; l += kOmpThreads / 32) {
             const uint16_t* zl = zs + (size_t)l * k;
             double acc = 0.0;
+            if (vec) {
+                const uint4* pl = reinterpret_cast<const uint4*>(zl);
+                const uint4* pn = reinterpret_cast<const uint4*>(znew);
+#pragma unroll 4
+                for (int v = lane; v < (k >> 3); v += 32) {
+                    const uint4 xa = pl[v], xb = pn[v];
+                    const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {                          // products of two binary16 numbers are exact in fp32
+                        const float2 fa = half2_bits_to_float2(wa[e]), fb = half2_bits_to_float2(wb[e]);
+                        acc += (double)(fa.x * fb.x);
+                        acc += (double)(fa.y * fb.y);
+                    }
+                }
+            } else {
 #pragma unroll 8
-            for (int row = lane; row < k; row += 32)
-                acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));   // product exact in fp32
+                for (int row = lane; row < k; row += 32)
+                    acc += (double)(half_bits_to_float(zl[row]) * half_bits_to_float(znew[row]));
+            }
             acc = warp_sum(acc);
             if (lane == 0) sh.gvec[l] = sig2 * acc;
         }
     }
     __syncthreads();
-    // ---- 5. c = F^T g ;  F is upper triangular, F(l,i) stored at F[l*s + i] ----------------------------
-    double csq = 0.0;
-    if ((int)threadIdx.x < j) {
-        const int i = threadIdx.x;
+    // ---- 5. c = F^T g ;  F is upper triangular, F(l,i) stored at F[l*s + i]; warp = one entry of c -------
+    for (int i = warp; i < j; i += kOmpThreads / 32) {
         double acc = 0.0;
-#pragma unroll 8
-        for (int l = 0; l <= i; ++l) acc += F[(size_t)l * s + i] * sh.gvec[l];
-        sh.cvec[i] = acc;
-        csq = acc * acc;
+        for (int l = lane; l <= i; l += 32) acc += F[(size_t)l * s + i] * sh.gvec[l];
+        acc = warp_sum(acc);
+        if (lane == 0) sh.cvec[i] = acc;
     }
+    __syncthreads();
+    double csq = 0.0;
+    if ((int)threadIdx.x < j) csq = sh.cvec[threadIdx.x] * sh.cvec[threadIdx.x];
     csq = block_sum(csq, sh.red);
     // ---- 6. gamma = 1/sqrt(g_ll - c^T c); a dependent column stops this recovery --------------------------
     const double gnn = sig2 * n2_new;
     const double piv = gnn - csq;
     if (!(piv > 1e-10 * gnn)) return 2;
     const double gamma = 1.0 / sqrt(piv);
-    // ---- 7. new column of F: [-gamma F c ; gamma] ------------------------------------------------------
-    __syncthreads();
-    if ((int)threadIdx.x < j) {
-        const int i = threadIdx.x;
+    // ---- 7. new column of F: [-gamma F c ; gamma]; warp = one row of F ------------------------------------
+    for (int i = warp; i < j; i += kOmpThreads / 32) {
         double acc = 0.0;
-#pragma unroll 8
-        for (int l = i; l < j; ++l) acc += F[(size_t)i * s + l] * sh.cvec[l];
-        F[(size_t)i * s + j] = -gamma * acc;
-    } else if ((int)threadIdx.x == j) {
-        F[(size_t)j * s + j] = gamma;
+        for (int l = i + lane; l < j; l += 32) acc += F[(size_t)i * s + l] * sh.cvec[l];
+        acc = warp_sum(acc);
+        if (lane == 0) F[(size_t)i * s + j] = -gamma * acc;
     }
+    if (threadIdx.x == 0) F[(size_t)j * s + j] = gamma;
     // ---- 8. a_j = gamma <a_new, r> ;  x = F a  grows by a_j * F(:, j) -------------------------------------
     const double aj = gamma * a.sigma * dot_r;
     __syncthreads();
@@ -536,10 +560,18 @@ __device__ int book_pick(const OmpArgs& a, BookSmem& sh, int m, int j, uint32_t 
     // ---- 9. r = y - A_Lambda x ---------------------------------------------------------------------------
     double rn2 = 0.0;
     for (int row = threadIdx.x; row < k; row += kOmpThreads) {
-        double acc = 0.0;
+        double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;     // four chains: the loads of 32 columns are in flight together
+        int l = 0;
 #pragma unroll 8
-        for (int l = 0; l <= j; ++l) acc += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
-        const double rv = y[row] - a.sigma * acc;
+        for (; l + 3 <= j; l += 4) {
+            acc0 += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
+            acc1 += sh.xs[l + 1] * (double)half_bits_to_float(zs[(size_t)(l + 1) * k + row]);
+            acc2 += sh.xs[l + 2] * (double)half_bits_to_float(zs[(size_t)(l + 2) * k + row]);
+            acc3 += sh.xs[l + 3] * (double)half_bits_to_float(zs[(size_t)(l + 3) * k + row]);
+        }
+        for (; l <= j; ++l) acc0 += sh.xs[l] * (double)half_bits_to_float(zs[(size_t)l * k + row]);
+        acc0 += acc2; acc1 += acc3;
+        const double rv = y[row] - a.sigma * (acc0 + acc1);
         r[row] = rv;
         a.r32[2 * row + m] = (float)rv;
         rn2 += rv * rv;
@@ -639,7 +671,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_omp(OmpArgs a, int mode) {
         }
         if (!act[0] && !act[1]) break;
         if (need_corr) {
-            if (mode == 0) corr_candidates(a, n_cand, wtop, picks);
+            if (mode == 0) corr_candidates(a, n_cand, wtop, picks, sr, mask_idx);
             else corr_all_columns(a, sr, mask_idx, mask_n, wtop, picks);
         }
         grid.sync();
@@ -1736,6 +1768,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
     std::vector<OmpArgs> args((size_t)n);
     cudaError_t e = cudaSuccess;
     int n_rounds = 0;
+    int mini_rounds = 0;          // rounds that get list passes: the likely ones; the spare rounds behind them stay cheap to enqueue
     for (int i = 0; i < n; ++i) {
         sgc_state* st = sts[i];
         sgc_state* lead = sts[i - i % per_batch];
@@ -1761,7 +1794,9 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
         // synchronising; a stale value only changes how much is enqueued); what they leave open is done in lock-step
         const int hint = speculate ? *reinterpret_cast<volatile int*>(st->h_rounds) : 0;
         const int last = hint & 255;
-        int want = last <= 0 ? 8 : 2 * last + 4;
+        int want = last <= 0 ? 8 : 2 * last + 3;
+        if (last > 0 && last + 2 > mini_rounds) mini_rounds = last + 2;
+        if (last <= 0) mini_rounds = kMaxRounds;
         if (st->max_rounds > 0 && want > st->max_rounds) want = st->max_rounds;
         if (want > n_rounds) n_rounds = want;
         // two-level screening pays where steps need several full passes (recovery picks columns outside the kept sets);
@@ -1792,7 +1827,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
         for (int round = 0; round < n_rounds && e == cudaSuccess; ++round) {
             // list passes first: speculate a few picks ahead, screen the wide lists only, keep what they confirm as
             // tentative picks; every kernel of this loop returns at once when there is nothing (more) to do
-            for (int mini = 0; two_level && mini < kMiniRounds && e == cudaSuccess; ++mini) {
+            for (int mini = 0; two_level && round < mini_rounds && mini < kMiniRounds && e == cudaSuccess; ++mini) {
                 sgc_state* st = st0;
                 {
                     PhaseTimer timer(st, stream, kPhaseCorr, 1);
