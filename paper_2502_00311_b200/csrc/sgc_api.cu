@@ -71,6 +71,7 @@ size_t layout_spec(sgc_state* st, unsigned char* base) {
         st->cand_list = carve<uint32_t>(base, off, sgc::kCandCap);
         st->cand_bits = carve<unsigned int>(base, off, ((size_t)st->d + 31) / 32);
         st->rtmp = carve<double>(base, off, k);
+        st->rhist = carve<double>(base, off, (size_t)st->pass_n * k);
         st->inv_norm = carve<uint16_t>(base, off, (size_t)st->d);
         st->zlist = carve<uint16_t>(base, off, (size_t)sgc::kGramList * k);
         st->gram = carve<double>(base, off, (size_t)sgc::kGramList * sgc::kGramList);

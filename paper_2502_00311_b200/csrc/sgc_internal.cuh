@@ -288,6 +288,7 @@ struct sgc_state {
     uint32_t* cand_list;        // [kCandCap]
     unsigned int* cand_bits;    // bitmap over [0, d): membership in cand_list
     double* rtmp;               // [k] scratch residual of the resolve kernel
+    double* rhist;              // [pass_n][k] the screened residuals of this state in fp64 (row = stream * rows per stream + position)
     uint16_t* inv_norm;         // [d] 1 / ||Z_i|| as binary16, filled once at creation (the screening pass reads it)
     uint16_t* zlist;            // [kGramList][k] the candidate columns as binary16 (Gram path)
     double* gram;               // [kGramList][kGramList] Z_C^T Z_C

@@ -50,6 +50,7 @@ struct OmpArgs {
     uint16_t* zsel; uint32_t* lam; double* F; double* acoef; double* x; double* rnorm;
     Counters* cnt; SpecCtl* ctl;
     uint16_t* rt; float* tau; float* inv_scale; unsigned int* rep_count; double* pick_score;
+    double* rhist;                     // fp64 copies of the screened residuals (row = m * half_n + position), for the resolve kernel
     // two-level screening
     float* wide_tau; double z_wide; unsigned int* wide_count; unsigned int* wide_bits;
     int mini;                          // 1: speculation ahead of a list pass (at most `depth` picks)
@@ -206,7 +207,12 @@ __device__ void write_rt_row(const OmpArgs& a, int m, int c, const double* r, do
     const int n = m * a.half_n + c;
     uint16_t* dst = a.rt + (size_t)n * a.k;
     const double sc = residual_scale(rn);
-    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) dst[row] = half_rn_bits(r[row] * sc);
+    double* keep = a.rhist + (size_t)n * a.k;
+    for (int row = threadIdx.x; row < a.k; row += kOmpThreads) {
+        const double rv = r[row];
+        dst[row] = half_rn_bits(rv * sc);
+        keep[row] = rv;
+    }
     if (threadIdx.x == 0) a.inv_scale[n] = (float)(1.0 / sc);
 }
 
@@ -1132,11 +1138,14 @@ __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
     const int nrow = m * a.half_n + c;
     const double sc = residual_scale(rn);
     uint16_t* dst = a.rt + (size_t)nrow * k;
+    double* keep = a.rhist + (size_t)nrow * k;
     for (int row = t; row < k; row += kGramThreads) {
         double acc = 0.0;
 #pragma unroll 8
         for (int l = 0; l < n_coef; ++l) acc += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
-        dst[row] = half_rn_bits((y[row] - a.sigma * acc) * sc);
+        const double rv = y[row] - a.sigma * acc;
+        dst[row] = half_rn_bits(rv * sc);
+        keep[row] = rv;
     }
     if (t == 0) {
         a.inv_scale[nrow] = (float)(1.0 / sc);
@@ -1352,8 +1361,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                                                2.0f * margin, 1);
             if (nc < 0) { bad = true; break; }
             if (nc == 1) { v = j + 1; continue; }                 // nobody comes close: the pick is the argmax
-            rebuild_prefix(a, sh, m, j, ra.rtmp, nullptr, nullptr);
-            rescore_candidates(a, sh, nc, ra.rtmp);
+            rescore_candidates(a, sh, nc, a.rhist + (size_t)n * a.k);       // the residual this pick was made from
             if (sh.best_idx == pick) { v = j + 1; continue; }
             forced = sh.best_idx; v = j; failed = true;
             if (!mini && threadIdx.x == 0) ctl->refuted = ctl->refuted + 1;
@@ -1405,8 +1413,7 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                     nc = collect_challengers(sh, ra.rep + (size_t)n * ra.rep_cap, count, lam, hi, kNoColumn, 0.0f, 2.0f * margin, 0);
                 if (nc <= 0) bad = true;
                 else {
-                    rebuild_prefix(a, sh, m, hi, ra.rtmp, nullptr, nullptr);
-                    rescore_candidates(a, sh, nc, ra.rtmp);
+                    rescore_candidates(a, sh, nc, a.rhist + (size_t)n * a.k);
                     forced = sh.best_idx; v = hi;
                     make_room(ra, (int)count + 1);
                     harvest(ra, sh, ra.rep + (size_t)n * ra.rep_cap, count, forced);
@@ -1684,6 +1691,7 @@ OmpArgs make_args(const sgc_state* st) {
     a.zsel = st->zsel; a.lam = st->lam; a.F = st->F; a.acoef = st->acoef; a.x = st->x; a.rnorm = st->rnorm;
     a.cnt = st->cnt; a.ctl = st->ctl;
     a.rt = st->rt; a.tau = st->tau; a.inv_scale = st->inv_scale; a.rep_count = st->rep_count; a.pick_score = st->pick_score;
+    a.rhist = st->rhist;
     a.cand_list = st->cand_list;
     a.zlist = st->zlist; a.gram = st->gram; a.p0 = st->p0; a.pick_li = st->pick_li;
     a.wide_tau = st->wide_tau; a.z_wide = st->z_wide; a.wide_count = nullptr; a.wide_bits = st->wide_bits; a.mini = 0;
