@@ -118,6 +118,7 @@ constexpr int kHistColumns = 8192;      // ... as long as they are at most this 
 constexpr int kLookAhead = 12;          // after a refuted pick, every kLookAhead-th later residual is harvested too
 constexpr double kLookAheadShare = 0.78; // ... as far as its columns reach this share of the residual's pick score
 constexpr int kWideCap = 2097152;       // columns per wide list (two-level screening)
+constexpr int kResolveBlocks = 16;        // blocks of the resolve kernel: all sweep the report lists, the last to finish walks the picks
 constexpr int kPassFastRows = 128;      // a pass over up to this many residual rows costs half of a wider one (A is generated once either way)
 constexpr int kMiniRounds = 8;          // list passes between two full passes, at most
 constexpr int kMiniDepth = 32;          // picks speculated ahead of one list pass
@@ -187,6 +188,8 @@ struct SpecCtl {
     int list_rounds;        // list passes of the last step that were resolved
     int list_refuted;       // picks that those list passes refuted
     int refuted;            // picks that the full passes of this step refuted
+    unsigned int resolve_ticket;   // blocks of the resolve kernel that have finished their share of the sweep
+    int contested[kPassMaxN];      // per screened residual: some report comes within the margin of its pick (sweep result)
     int pass_rows;          // residual rows that the full passes of the last step screened, summed over the passes
     int hist_count, hist_next;  // ring of the kept index sets of the last steps: valid slots, slot of the next step
     int trace[kMaxRounds][3];   // per round: confirmed picks of both streams and the list length after it

@@ -325,6 +325,7 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
         float dm = 0.0f, dv = 0.0f, n2 = 0.0f;
         uint32_t h = key.ck + (uint32_t)lane * key.mk;
         const uint32_t step = 32u * key.mk;
+#pragma unroll 4
         for (int row = 2 * lane; row < k; row += 64) {              // one generated word = two rows
             const float2 z = half2_bits_to_float2(z_pair_from_word(h));
             h += step;
@@ -1119,13 +1120,23 @@ __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
         for (int pr = t; pr < (k >> 1); pr += kGramThreads) dst[pr] = src[pr];
     }
     const bool screened = c < a.half_n && (j < hi || (j == hi && extra));
-    // r_j = y - sigma * Z_Lambda x_j: first its norm, then (for a screened state) the scaled binary16 row
+    // r_j = y - sigma * Z_Lambda x_j in fp64 (kept for the resolve kernel) and its norm, then (for a screened state) the
+    // scaled binary16 row
+    const bool has_row = c < a.half_n;
+    const int nrow = m * a.half_n + (has_row ? c : 0);
+    double* keep = a.rhist + (size_t)nrow * k;
     double rn2 = 0.0;
     for (int row = t; row < k; row += kGramThreads) {
-        double acc = 0.0;
-#pragma unroll 8
-        for (int l = 0; l < n_coef; ++l) acc += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
-        const double r1 = y[row] - a.sigma * acc;
+        double acc0 = 0.0, acc1 = 0.0;
+        int l = 0;
+#pragma unroll 4
+        for (; l + 1 < n_coef; l += 2) {
+            acc0 += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
+            acc1 += xs[l + 1] * (double)half_bits_to_float(a.zlist[(size_t)li[l + 1] * k + row]);
+        }
+        if (l < n_coef) acc0 += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
+        const double r1 = y[row] - a.sigma * (acc0 + acc1);
+        if (has_row) keep[row] = r1;
         rn2 += r1 * r1;
     }
     rn2 = block_sum_256(rn2, red);
@@ -1135,18 +1146,9 @@ __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
         else a.rnorm[(size_t)m * s + j - 1] = rn;            // ||r|| after pick j-1 (verified entries are rewritten with equal values)
     }
     if (!screened) return;
-    const int nrow = m * a.half_n + c;
     const double sc = residual_scale(rn);
     uint16_t* dst = a.rt + (size_t)nrow * k;
-    double* keep = a.rhist + (size_t)nrow * k;
-    for (int row = t; row < k; row += kGramThreads) {
-        double acc = 0.0;
-#pragma unroll 8
-        for (int l = 0; l < n_coef; ++l) acc += xs[l] * (double)half_bits_to_float(a.zlist[(size_t)li[l] * k + row]);
-        const double rv = y[row] - a.sigma * acc;
-        dst[row] = half_rn_bits(rv * sc);
-        keep[row] = rv;
-    }
+    for (int row = t; row < k; row += kGramThreads) dst[row] = half_rn_bits(keep[row] * sc);    // each thread re-reads its own rows
     if (t == 0) {
         a.inv_scale[nrow] = (float)(1.0 / sc);
         const double unit = rn / sqrt((double)k);
@@ -1300,7 +1302,52 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             return;
         }
     }
-    __shared__ int contested[kPassMaxN];        // per screened residual: some report comes within the margin of its pick
+    const int s = a.s;
+    // Sweep: every block takes its share of the report lists (warp per residual) and notes which picks have a challenger
+    // within the margin; the walk below only stops at those.  Nothing of the control block changes before the walk.
+    {
+        const int gw = blockIdx.x * (kOmpThreads / 32) + (threadIdx.x >> 5), nw = gridDim.x * (kOmpThreads / 32);
+        for (int m = 0; m < 2; ++m) {
+            if (ctl->finished[m]) continue;
+            const int base = ctl->base[m], hi = ctl->hi[m];
+            const int lo = (mini && ctl->tv[m] > base) ? ctl->tv[m] : base;
+            for (int j = lo + gw; j < hi; j += nw) {
+                const int n = m * a.half_n + (j - base);
+                const unsigned int count = a.rep_count[n];
+                bool hit = count > (unsigned int)ra.rep_cap;             // an overflowed list: the walk gives up there
+                if (!hit) {
+                    const uint32_t pick = a.lam[(size_t)m * s + j];
+                    const double ps = a.pick_score[(size_t)m * s + j];
+                    const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
+                    const float floor_sc = (float)ps - (float)screen_margin(rn, ps, a.k);
+                    const bool skip_members = ctl->list_exact[m] != 0;
+                    for (unsigned int e = threadIdx.x & 31; e < count; e += 32) {
+                        const uint2 rp = ra.rep[(size_t)n * ra.rep_cap + e];
+                        if (__uint_as_float(rp.y) < floor_sc || rp.x == pick) continue;
+                        // a list member lost the exact comparison against the pick during the speculation (or is in the support)
+                        if (skip_members && ((ra.cand_bits[rp.x >> 5] >> (rp.x & 31u)) & 1u)) continue;
+                        if (!in_support(a.lam + (size_t)m * s, j, rp.x)) hit = true;
+                    }
+                    hit = __any_sync(0xffffffffu, hit);
+                }
+                if ((threadIdx.x & 31) == 0) a.ctl->contested[n] = hit ? 1 : 0;
+            }
+        }
+    }
+    // the block that finishes its share last walks the picks (ticket counter, nobody waits)
+    __shared__ int last_block;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int ticket = atomicAdd(&a.ctl->resolve_ticket, 1u);
+        last_block = ticket == gridDim.x - 1 ? 1 : 0;
+        if (last_block) a.ctl->resolve_ticket = 0u;
+    }
+    __syncthreads();
+    if (!last_block) return;
+    __threadfence();
+    __shared__ int contested[kPassMaxN];
+    for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = ctl->contested[n];
     if (threadIdx.x == 0) {
         give_up = 0; any_failed = 0;
         if (mini) ctl->list_rounds = ctl->list_rounds + 1;
@@ -1308,34 +1355,6 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
             ctl->rounds = ctl->rounds + 1;
             // width of the pass whose reports are being resolved (ctl->narrow still names it)
             ctl->pass_rows = ctl->pass_rows + (ctl->narrow ? a.rows_narrow : a.rows_wide);
-        }
-    }
-    for (int n = threadIdx.x; n < kPassMaxN; n += kOmpThreads) contested[n] = 0;
-    __syncthreads();
-    const int s = a.s;
-    // one parallel sweep over all report lists; the walk below only stops at contested picks
-    for (int m = 0; m < 2; ++m) {
-        if (ctl->finished[m]) continue;
-        const int base = ctl->base[m], hi = ctl->hi[m];
-        const int lo = (mini && ctl->tv[m] > base) ? ctl->tv[m] : base;
-        for (int j = lo + (threadIdx.x >> 5); j < hi; j += kOmpThreads / 32) {         // warp per residual
-            const int n = m * a.half_n + (j - base);
-            const unsigned int count = a.rep_count[n];
-            if (count > (unsigned int)ra.rep_cap) { if ((threadIdx.x & 31) == 0) contested[n] = 1; continue; }
-            const uint32_t pick = a.lam[(size_t)m * s + j];
-            const double ps = a.pick_score[(size_t)m * s + j];
-            const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
-            const float floor_sc = (float)ps - (float)screen_margin(rn, ps, a.k);
-            const bool skip_members = ctl->list_exact[m] != 0;
-            bool hit = false;
-            for (unsigned int e = threadIdx.x & 31; e < count; e += 32) {
-                const uint2 rp = ra.rep[(size_t)n * ra.rep_cap + e];
-                if (__uint_as_float(rp.y) < floor_sc || rp.x == pick) continue;
-                // a list member lost the exact comparison against the pick during the speculation (or is in the support)
-                if (skip_members && ((ra.cand_bits[rp.x >> 5] >> (rp.x & 31u)) & 1u)) continue;
-                if (!in_support(a.lam + (size_t)m * s, j, rp.x)) hit = true;
-            }
-            if (__any_sync(0xffffffffu, hit) && (threadIdx.x & 31) == 0) contested[n] = 1;
         }
     }
     __syncthreads();
@@ -1874,7 +1893,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
                 ra.rep = st->rep; ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list;
                 ra.rtmp = st->rtmp; ra.kept_ring = st->kept_ring; ra.mini = 1; ra.wide_count = st->wide_count;
                 PhaseTimer timer(st, stream, kPhaseBook, 1);
-                k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
+                k_resolve<<<kResolveBlocks, kOmpThreads, 0, stream>>>(ra);
                 *launches += 1;
             }
             for (int b0 = 0; b0 < n && e == cudaSuccess; b0 += per_batch) {
@@ -1930,7 +1949,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
                     ra.rep_cap = kRepCap; ra.cand_bits = st->cand_bits; ra.cand_list = st->cand_list; ra.rtmp = st->rtmp;
                     ra.kept_ring = st->kept_ring; ra.mini = 0; ra.wide_count = st->wide_count;
                     PhaseTimer timer(st, stream, kPhaseBook, 1);
-                    k_resolve<<<1, kOmpThreads, 0, stream>>>(ra);
+                    k_resolve<<<kResolveBlocks, kOmpThreads, 0, stream>>>(ra);
                     *launches += 1;
                 }
             }

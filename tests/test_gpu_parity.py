@@ -254,7 +254,7 @@ def test_steps_after_a_refuted_pick_screen_in_passes_of_half_the_width(sgc):
     ref.close()
 
 
-@pytest.mark.parametrize("d,k,s,steps", [(400_000, 256, 48, 7), (1_000_000, 512, 100, 4)])
+@pytest.mark.parametrize("d,k,s,steps", [(400_000, 256, 48, 7), (500_000, 512, 100, 4)])
 def test_two_level_screening_matches_the_oracle(sgc, d, k, s, steps):
     # inexact regime (supports redrawn every step, k small): steps need several passes over all columns, which switches
     # on the wide lists and the list passes between full passes; the picks must not depend on any of that
