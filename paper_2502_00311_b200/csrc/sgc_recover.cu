@@ -1321,12 +1321,22 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_resolve(ResolveArgs ra) {
                     const double rn = j == 0 ? ctl->ynorm[m] : a.rnorm[(size_t)m * s + j - 1];
                     const float floor_sc = (float)ps - (float)screen_margin(rn, ps, a.k);
                     const bool skip_members = ctl->list_exact[m] != 0;
-                    for (unsigned int e = threadIdx.x & 31; e < count; e += 32) {
-                        const uint2 rp = ra.rep[(size_t)n * ra.rep_cap + e];
-                        if (__uint_as_float(rp.y) < floor_sc || rp.x == pick) continue;
-                        // a list member lost the exact comparison against the pick during the speculation (or is in the support)
-                        if (skip_members && ((ra.cand_bits[rp.x >> 5] >> (rp.x & 31u)) & 1u)) continue;
-                        if (!in_support(a.lam + (size_t)m * s, j, rp.x)) hit = true;
+                    const uint2* list = ra.rep + (size_t)n * ra.rep_cap;
+                    for (unsigned int e0 = threadIdx.x & 31; e0 < count; e0 += 8 * 32) {
+                        uint2 rp8[8];                                    // eight reports in flight per lane
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const unsigned int e = e0 + 32u * u;
+                            rp8[u] = e < count ? list[e] : make_uint2(pick, 0u);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const uint2 rp = rp8[u];
+                            if (__uint_as_float(rp.y) < floor_sc || rp.x == pick) continue;
+                            // a list member lost the exact comparison against the pick during the speculation (or is in the support)
+                            if (skip_members && ((ra.cand_bits[rp.x >> 5] >> (rp.x & 31u)) & 1u)) continue;
+                            if (!in_support(a.lam + (size_t)m * s, j, rp.x)) hit = true;
+                        }
                     }
                     hit = __any_sync(0xffffffffu, hit);
                 }
