@@ -845,6 +845,8 @@ __global__ void __launch_bounds__(kOmpThreads, 1) k_spec_small(OmpArgs a) {
 // challenger and k_resolve decides with the directly computed scores.
 // ------------------------------------------------------------------------------------------------
 constexpr int kGramThreads = 256;
+constexpr int kGramSmemN = 96, kGramSmemS = 64;       // list length and support size up to which k_omp_gram stages G and F
+constexpr size_t kGramSmemBytes = sizeof(double) * ((size_t)kGramSmemN * kGramSmemN + (size_t)kGramSmemS * kGramSmemS);
 
 __device__ __forceinline__ bool gram_round(volatile SpecCtl* ctl) {
     return ctl->round_active && !ctl->fallback && ctl->gram_ok && ctl->n_cand <= kGramList;
@@ -942,6 +944,16 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
     const double sigma = a.sigma, sig2 = sigma * sigma;
     const double* G = a.gram;
     double* F = a.F + (size_t)m * s * s;
+    // short lists and supports (the steady state) keep G and F in shared memory: every pick is a chain of a dozen dependent
+    // reads of them, each an L2 round trip otherwise.  F is written through to global memory, where later kernels read it.
+    extern __shared__ double gram_sm[];
+    double* Gs = gram_sm;
+    double* Fs = gram_sm + kGramSmemN * kGramSmemN;
+    const bool g_sm = n <= kGramSmemN, f_sm = s <= kGramSmemS;
+    if (g_sm) for (int e = t; e < n * n; e += kGramThreads) Gs[e] = G[(size_t)(e / n) * kGramList + (e % n)];
+    if (f_sm) for (int e = t; e < s * s; e += kGramThreads) Fs[e] = F[e];
+#define GRAM_G(r, c) (g_sm ? Gs[(r) * n + (c)] : G[(size_t)(r) * kGramList + (c)])
+#define GRAM_F(r, c) (f_sm ? Fs[(r) * s + (c)] : F[(size_t)(r) * s + (c)])
     double* ac = a.acoef + (size_t)m * s;
     uint32_t* lam = a.lam + (size_t)m * s;
     const uint32_t my_col = t < n ? a.cand_list[t] : kNoColumn;
@@ -951,7 +963,7 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
     __syncthreads();
     int forced_li = -1;
     if (t < n) {
-        gdiag[t] = G[(size_t)t * kGramList + t];
+        gdiag[t] = G[(size_t)t * kGramList + t];          // (global: the staged copy is not yet synchronised)
         for (int l = 0; l < v0; ++l) if (lam[l] == my_col) { li[l] = t; taken[t] = 1; atomicAdd(&found, 1); }
         if (forced0 != kNoColumn && my_col == forced0) { li[v0] = t; atomicAdd(&found, 1); }
     }
@@ -963,7 +975,7 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
     if (forced0 != kNoColumn) forced_li = li[v0];
     for (int i = t; i < v0; i += kGramThreads) {
         double acc = 0.0;
-        for (int l = i; l < v0; ++l) acc = acc + ac[l] * F[(size_t)i * s + l];
+        for (int l = i; l < v0; ++l) acc = acc + ac[l] * GRAM_F(i, l);
         xs[i] = acc;
         a.x[(size_t)m * s + i] = acc;
         a.pick_li[(size_t)m * s + i] = li[i];
@@ -977,7 +989,7 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
         if (t < n) {
             double acc = 0.0;
 #pragma unroll 8
-            for (int l = 0; l < j; ++l) acc += G[(size_t)li[l] * kGramList + t] * xs[l];
+            for (int l = 0; l < j; ++l) acc += GRAM_G(li[l], t) * xs[l];
             pi = a.p0[m * kGramList + t] - sigma * acc;
             p[t] = pi;
         }
@@ -1022,14 +1034,14 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
             if (!forced) a.pick_score[(size_t)m * s + j] = fabs(pq) / sqrt(gqq);
         }
         // Gram column of the pick restricted to the support, c = F^T g, pivot
-        for (int l = t; l < j; l += kGramThreads) gvec[l] = sig2 * G[(size_t)li[l] * kGramList + q];
+        for (int l = t; l < j; l += kGramThreads) gvec[l] = sig2 * GRAM_G(li[l], q);
         __syncthreads();
         double csq = 0.0;
         for (int i0 = 0; i0 < j; i0 += kGramThreads / 16) {
             const int i = i0 + (t >> 4), sub = t & 15;
             double acc = 0.0;
             if (i < j)
-                for (int l = sub; l <= i; l += 16) acc += F[(size_t)l * s + i] * gvec[l];
+                for (int l = sub; l <= i; l += 16) acc += GRAM_F(l, i) * gvec[l];
             for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
             if (i < j && sub == 0) { cvec[i] = acc; csq += acc * acc; }
         }
@@ -1053,16 +1065,16 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
             const int i = i0 + (t >> 4), sub = t & 15;
             double acc = 0.0;
             if (i < j)
-                for (int l = i + sub; l < j; l += 16) acc += F[(size_t)i * s + l] * cvec[l];
+                for (int l = i + sub; l < j; l += 16) acc += GRAM_F(i, l) * cvec[l];
             for (int o = 8; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (i < j && sub == 0) F[(size_t)i * s + j] = -gamma * acc;
+            if (i < j && sub == 0) { F[(size_t)i * s + j] = -gamma * acc; if (f_sm) Fs[i * s + j] = -gamma * acc; }
         }
-        if (t == 0) F[(size_t)j * s + j] = gamma;
+        if (t == 0) { F[(size_t)j * s + j] = gamma; if (f_sm) Fs[j * s + j] = gamma; }
         const double aj = gamma * sigma * pq;
         __syncthreads();
         for (int i = t; i <= j; i += kGramThreads) {
             const double xo = (i < j) ? xs[i] : 0.0;
-            const double xn = xo + aj * F[(size_t)i * s + j];
+            const double xn = xo + aj * GRAM_F(i, j);
             xs[i] = xn;
             a.x[(size_t)m * s + i] = xn;
         }
@@ -1082,6 +1094,8 @@ __global__ void __launch_bounds__(kGramThreads, 1) k_omp_gram(OmpArgs a) {
         a.ctl->list_exact[m] = 1;
     }
 }
+#undef GRAM_G
+#undef GRAM_F
 
 // block (m, c): the state after j = base + c picks of residual m
 __global__ void __launch_bounds__(kGramThreads) k_spec_rows(OmpArgs a) {
@@ -1752,6 +1766,8 @@ cudaError_t configure_recover(sgc_state* st) {
     int occ = 0;
     e = cudaFuncSetAttribute(k_spec_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_omp_gram, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGramSmemBytes);
+    if (e != cudaSuccess) return e;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_omp, kOmpThreads, smem);
     if (e != cudaSuccess) return e;
     if (occ < 1) return cudaErrorInvalidConfiguration;
@@ -1914,7 +1930,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
                     PhaseTimer timer(st, stream, kPhaseCorr, 6);
                     k_gram_prepare<<<kGramList, kGramThreads, 0, stream>>>(a);       // very short list: Gram-matrix OMP
                     k_gram_matrix<<<kGramList, kGramThreads, (size_t)st->k * 2, stream>>>(a);
-                    k_omp_gram<<<2, kGramThreads, 0, stream>>>(a);
+                    k_omp_gram<<<2, kGramThreads, kGramSmemBytes, stream>>>(a);
                     k_spec_rows<<<2 * (a.half_n + 1), kGramThreads, 0, stream>>>(a);
                     k_spec_small<<<2, kOmpThreads, st->corr_smem, stream>>>(a);      // short candidate list
                     e = launch_omp(st, a, 0, stream);                                // long candidate list
