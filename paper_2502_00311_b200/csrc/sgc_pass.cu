@@ -343,6 +343,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                 // every 8th residual feeds the wide list of its stream (full passes of the two-level screening)
                 const bool feeds = WIDE && a.big_tau != nullptr && !listed && (n_res & 7) == 0;
                 const float wide_tau_n = feeds ? a.big_tau[n_res >> 3] : 0.0f;
+                // wide-list hits of this warp are queued in shared memory and appended after the sweep, all at once: the two
+                // dependent global atomics of an append then cost the warp two round trips per sweep instead of two per hit
+                // (the warp's 32 residuals belong to one stream whenever the streams' blocks are multiples of 32 rows)
+                uint32_t* queue = reinterpret_cast<uint32_t*>(norms + (size_t)(8 + quad) * kSuperCols);
+                const bool queued = WIDE && (a.big_half & 31) == 0;
+                if (WIDE && lane == 0) queue[0] = 0u;
+                if (WIDE) __syncwarp();
 #pragma unroll 1
                 for (int c0 = 0; c0 < kSuperCols; c0 += 16) {
                     uint32_t v[16];
@@ -367,6 +374,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                             const int i = __ffs(hits) - 1;
                             hits &= hits - 1u;
                             const unsigned long long col = (unsigned long long)sweep * kSuperCols + c0 + i;
+                            if (queued) {
+                                const unsigned int qs = atomicAdd(&queue[0], 1u) + 1u;
+                                if (qs < (unsigned int)kSuperCols) { queue[qs] = (uint32_t)col; continue; }
+                            }
                             const unsigned int bit = 1u << ((unsigned int)col & 31u);
                             if (!(atomicOr(&a.big_bits[(size_t)m * ((a.d + 31) >> 5) + (col >> 5)], bit) & bit)) {
                                 const unsigned int slot = atomicAdd(&a.big_count[m], 1u);
@@ -391,7 +402,21 @@ __global__ void __launch_bounds__(kPassThreads, 1) k_pass(const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acce + 8u * buf);
+                if (lane == 0) mbar_arrive(bar_acce + 8u * buf);     // the accumulator is free; the queued appends follow
+                if (WIDE && queued) {
+                    unsigned int qn = queue[0];
+                    if (qn > (unsigned int)kSuperCols - 1u) qn = (unsigned int)kSuperCols - 1u;
+                    const int m = quad * 32 >= a.big_half ? 1 : 0;
+                    for (unsigned int e = 1u + lane; e <= qn; e += 32u) {
+                        const unsigned long long col = queue[e];
+                        const unsigned int bit = 1u << ((unsigned int)col & 31u);
+                        if (!(atomicOr(&a.big_bits[(size_t)m * ((a.d + 31) >> 5) + (col >> 5)], bit) & bit)) {
+                            const unsigned int slot = atomicAdd(&a.big_count[m], 1u);
+                            if (slot < (unsigned int)a.big_cap) a.big_list[(size_t)m * a.big_cap + slot] = (uint32_t)col;
+                        }
+                    }
+                    __syncwarp();
+                }
                 continue;
             }
             const float* nr = norms + (size_t)(sweep_i % kNormRing) * kSuperCols * 2;
