@@ -231,7 +231,7 @@ SGC_API int sgc_set_wait_limit(sgc_state* st, uint64_t ns);
  * enqueues; the picks that the rounds leave open are made on the exact lock-step path, so the result is Algorithm 3's
  * (Appendix B) for every bound.  The paper has no counterpart: the bound caps the work a step enqueues ahead of time.
  *   rounds   0 (the default) lets the library choose from the number of rounds the last finished step needed (twice that
- *            plus four, at most 24); negative: SGC_ERR_DIM.  In a group (sgc_step_group) the largest bound of a batch holds. */
+ *            plus three, at most 24); negative: SGC_ERR_DIM.  In a group (sgc_step_group) the largest bound of a batch holds. */
 SGC_API int sgc_set_max_rounds(sgc_state* st, int32_t rounds);
 
 /* Number of kernel launches the last sgc_step / sgc_step_group enqueued for this state. */
