@@ -1869,6 +1869,7 @@ static cudaError_t recover_batches(sgc_state* const* sts, float* const* weights,
         args[0].half_n = st0->pass_n_half / 2;
         args[0].rows_wide = args[0].rows_narrow = st0->pass_n_half;
         n_rounds = n_rounds + 1 < kMaxRounds ? n_rounds + 1 : kMaxRounds;
+        if (st0->max_rounds > 0 && n_rounds > st0->max_rounds) n_rounds = st0->max_rounds;
     }
     PassWide wide;
     if (two_level) {
