@@ -193,13 +193,14 @@ def test_speculative_recovery_with_redrawn_supports_and_alpha(sgc):
     assert all(fb == 0 for _, fb, _ in stats), stats
 
 
-@pytest.mark.parametrize("max_rounds", [1, 2, 3])
-def test_lockstep_finishes_what_a_bounded_number_of_rounds_leaves_open(sgc, max_rounds):
+@pytest.mark.parametrize("d,k,s,max_rounds", [(150_000, 256, 32, 1), (150_000, 256, 32, 2), (150_000, 256, 32, 3),
+                                              (100_000, 768, 96, 2)])
+def test_lockstep_finishes_what_a_bounded_number_of_rounds_leaves_open(sgc, d, k, s, max_rounds):
     # Two steady steps, then a new support every step, so that every later step needs several rounds of speculation and
     # its first refuted pick gets a prescribed column.  With the rounds bounded, the lock-step path takes over from a
-    # state that the Gram-matrix speculation left behind -- stored columns, F, coefficients and the prescribed pick
-    # included -- and must still end with Algorithm 3's supports and update.
-    d, k, s, seed = 150_000, 256, 32, 3
+    # state that the speculation left behind -- stored columns, F, coefficients and the prescribed pick included -- and
+    # must still end with Algorithm 3's supports and update.  (s = 96: the bounded steps screen in half-width passes.)
+    seed = 3
     hp = inputs.ADAM
     st = sgc.Sgc(d, k, s, seed, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"])
     st.set_mode(sgc.MODE_SPECULATIVE)
