@@ -229,27 +229,15 @@ __device__ void pick_block(PickSmem& sm, const float* __restrict__ grad, unsigne
         }
     }
     __syncthreads();
-    // ascending index order: bitonic sort of the slots in use, rounded up to a power of two (unused slots hold
-    // 0xFFFFFFFF and sink to the end)
-    unsigned int span = 2;
-    while (span < s) span <<= 1;
-    for (unsigned int size = 2; size <= span; size <<= 1) {
-        for (unsigned int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (unsigned int i = threadIdx.x; i < span; i += NT) {
-                const unsigned int j = i ^ stride;
-                if (j > i && j < span) {
-                    const uint32_t a = sm.picked[i], b = sm.picked[j];
-                    const bool up = ((i & size) == 0);
-                    if ((a > b) == up) { sm.picked[i] = b; sm.picked[j] = a; }
-                }
-            }
-            __syncthreads();
-        }
-    }
+    // ascending index order: the indices are distinct, so the rank of one among the s kept is its place in the output (every
+    // thread reads the same slot at the same time: a broadcast); exactly s slots are in use, the radix selection having
+    // stopped on a threshold that s keys reach
     for (unsigned int i = threadIdx.x; i < s; i += NT) {
         const uint32_t idx = sm.picked[i];
-        sel_idx[i] = idx;
-        sel_val[i] = grad[idx];
+        unsigned int rank = 0;
+        for (unsigned int q = 0; q < s; ++q) rank += sm.picked[q] < idx ? 1u : 0u;
+        sel_idx[rank] = idx;
+        sel_val[rank] = grad[idx];
     }
 }
 
@@ -354,20 +342,22 @@ k_select_fast(const float* __restrict__ grad, unsigned long long d, unsigned int
     for (int u = 0; u < per; ++u) { const unsigned int c = __ldcg(&hist[threadIdx.x * per + u]); sh_hist[threadIdx.x * per + u] = c; mine += c; }
     const unsigned int count = __ldcg(&cnt->sel_count);
     const bool hit = count >= s && count <= (unsigned int)kSelCap;
-    part[threadIdx.x] = mine;
     if (threadIdx.x == 0) next_bin = floor_bin;         // when even the whole histogram holds fewer than `want`: its floor
     __syncthreads();
     {
-        // keys in the bins of higher threads: suffix sum by a Hillis-Steele scan over the reversed order
-        const int rt = kFastThreads - 1 - threadIdx.x;
+        // keys in the bins of this and of higher threads: suffix sum, first inside each warp (shuffles), then over the warps
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         unsigned int incl = mine;
-        for (int o = 1; o < kFastThreads; o <<= 1) {
-            __syncthreads();
-            const unsigned int add = (rt >= o) ? part[threadIdx.x + o] : 0u;
-            __syncthreads();
-            incl += add;
-            part[threadIdx.x] = incl;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int v = __shfl_down_sync(0xffffffffu, incl, o);
+            if (lane + o < 32) incl += v;
         }
+        if (lane == 0) part[warp] = incl;                   // the warp's total
+        __syncthreads();
+        unsigned int higher = 0;
+        for (int w = warp + 1; w < kFastThreads / 32; ++w) higher += part[w];
+        incl += higher;
         const unsigned int above = incl - mine;
         if (above < want && want <= incl) {              // exactly one thread
             unsigned int acc = above;
