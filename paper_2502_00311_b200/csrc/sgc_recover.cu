@@ -325,19 +325,36 @@ __device__ void corr_candidates(const OmpArgs& a, int n_cand, Top2 (*wtop)[32], 
         float dm = 0.0f, dv = 0.0f, n2 = 0.0f;
         uint32_t h = key.ck + (uint32_t)lane * key.mk;
         const uint32_t step = 32u * key.mk;
+        if ((k & 1) == 0) {
+            // both residual pairs of a generated word in one 16-byte read: consecutive lanes, consecutive banks
+            const float4* r4 = reinterpret_cast<const float4*>(r32);
 #pragma unroll 4
-        for (int row = 2 * lane; row < k; row += 64) {              // one generated word = two rows
-            const float2 z = half2_bits_to_float2(z_pair_from_word(h));
-            h += step;
-            const float2 r0 = r32[row];
-            dm = __fmaf_rn(z.x, r0.x, dm);
-            dv = __fmaf_rn(z.x, r0.y, dv);
-            n2 = __fmaf_rn(z.x, z.x, n2);
-            if (row + 1 < k) {
-                const float2 r1 = r32[row + 1];
-                dm = __fmaf_rn(z.y, r1.x, dm);
-                dv = __fmaf_rn(z.y, r1.y, dv);
+            for (int pr = lane; pr < (k >> 1); pr += 32) {
+                const float2 z = half2_bits_to_float2(z_pair_from_word(h));
+                h += step;
+                const float4 rr = r4[pr];
+                dm = __fmaf_rn(z.x, rr.x, dm);
+                dv = __fmaf_rn(z.x, rr.y, dv);
+                n2 = __fmaf_rn(z.x, z.x, n2);
+                dm = __fmaf_rn(z.y, rr.z, dm);
+                dv = __fmaf_rn(z.y, rr.w, dv);
                 n2 = __fmaf_rn(z.y, z.y, n2);
+            }
+        } else {
+#pragma unroll 4
+            for (int row = 2 * lane; row < k; row += 64) {              // one generated word = two rows
+                const float2 z = half2_bits_to_float2(z_pair_from_word(h));
+                h += step;
+                const float2 r0 = r32[row];
+                dm = __fmaf_rn(z.x, r0.x, dm);
+                dv = __fmaf_rn(z.x, r0.y, dv);
+                n2 = __fmaf_rn(z.x, z.x, n2);
+                if (row + 1 < k) {
+                    const float2 r1 = r32[row + 1];
+                    dm = __fmaf_rn(z.y, r1.x, dm);
+                    dv = __fmaf_rn(z.y, r1.y, dv);
+                    n2 = __fmaf_rn(z.y, z.y, n2);
+                }
             }
         }
         dm = warp_sum(dm); dv = warp_sum(dv); n2 = warp_sum(n2);
